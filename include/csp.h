@@ -1,0 +1,198 @@
+/*
+ * csp.h -- C interface of the B200 (sm_100a) library for the scoring-and-compaction pass of
+ * Cross-Self Pruning (CSP), the KV-cache pruning method of "Cross-Self KV Cache Pruning for
+ * Efficient Vision-Language Inference".
+ *
+ * One call handles one layer: every sequence b < batch and every KV head h < n_kv_heads is an
+ * independent unit.  For each unit the path is
+ *
+ *   score    logits of the last W queries against every cached key (Eq. 5), each row normalised
+ *            by n-softmax over all keys it can see (Eq. 7), the last R key columns dropped
+ *            (Section 3.2, "A[-O:, :-R]"), rows averaged over the query heads of the KV group,
+ *            then summed over the query axis separately for queries with the same modality
+ *            label as the key (intra, "self") and a different one (inter, "cross") (Eq. 1);
+ *   select   a top-K over each of the two score vectors (Eq. 2), the two masks combined (Eq. 3),
+ *            the kept positions listed in ascending order followed by the last R positions;
+ *   compact  K, V and the labels gathered by that list (Eq. 4).
+ *
+ * Algorithm 1 is `csp_prune_layer`; a cache shorter than its budget T is passed through.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless its name ends in `_host`.  The caller owns every
+ *    buffer.  The library never allocates or frees device memory and, except for
+ *    csp_device_status and csp_prune_layer_host, never synchronises: work is enqueued on the
+ *    given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
+ *  - Inputs are read-only.  Outputs must not overlap inputs or each other.
+ *  - Tensors are described by a base pointer and ELEMENT strides; the innermost (head_dim)
+ *    axis is contiguous.  Base pointers and row starts must be 16-byte aligned (every stride
+ *    times the element size a multiple of 16 bytes).
+ *  - Errors the host can see (null pointer, unsupported shape, misalignment, workspace too
+ *    small, wrong GPU) are returned at once and nothing is enqueued.  Conditions only the
+ *    device can see are OR-ed into a status word at the start of the workspace
+ *    (CSP_DEV_* bits) and read back with csp_device_status; kernels never trap and every wait
+ *    inside them is bounded.
+ *  - Labels: modality[b, (h,) t] is a small integer; 0 is text, anything else is visual;
+ *    "intra" means equal labels.  After a prune the labels differ per head, so they carry a
+ *    head stride (0 when all heads of a sequence share one row of labels).
+ */
+#ifndef CSP_H
+#define CSP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CSP_OK = 0,
+    CSP_ERR_INVALID_ARG = 1,  /* null pointer, negative size */
+    CSP_ERR_UNSUPPORTED = 2,  /* shape, dtype, stride or mode this build has no kernel for */
+    CSP_ERR_WORKSPACE = 3,    /* workspace missing or smaller than csp_workspace_bytes */
+    CSP_ERR_ARCH = 4,         /* the current device is not compute capability 10.x */
+    CSP_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed (launch, copy, descriptor) */
+    CSP_ERR_TIMEOUT = 6       /* a bounded wait inside a kernel expired (from csp_device_status) */
+} csp_status;
+
+typedef enum { CSP_F32 = 0, CSP_BF16 = 1 } csp_dtype;
+
+/* Eq. 3 prints M = M^s AND M^c; Sections 3.2 and 5.1 describe the kept set as both selections
+ * together, with overlap saving budget.  OR is the default reading, AND the printed one. */
+typedef enum { CSP_COMBINE_OR = 0, CSP_COMBINE_AND = 1 } csp_combine;
+
+/* SEGMENTED: four budgets per sequence, a top-K of the intra score and of the inter score among
+ * the text keys and among the visual keys.  GLOBAL: the paper's literal K^s and K^c over all keys. */
+typedef enum { CSP_SELECT_SEGMENTED = 0, CSP_SELECT_GLOBAL = 1 } csp_select_mode;
+
+/* PER_KV: one selection per KV head from the mean over its query-head group.
+ * MEAN_ALL: one selection per sequence from the mean over every head (Section 3.2). */
+typedef enum { CSP_HEADS_PER_KV = 0, CSP_HEADS_MEAN_ALL = 1 } csp_head_reduce;
+
+/* bits of the device status word */
+enum {
+    CSP_DEV_K_CLAMPED = 1,  /* a budget exceeded its candidate count (or was negative) and was clamped */
+    CSP_DEV_CAPACITY = 2,   /* a unit's kept rows did not fit out_capacity; its n_out is -1 */
+    CSP_DEV_TIMEOUT = 4,    /* a bounded wait expired; outputs of that call are not valid */
+    CSP_DEV_BAD_LEN = 8     /* a sequence length was negative or above max_len; unit skipped, n_out -1 */
+};
+
+typedef struct {
+    void* ptr;
+    int64_t stride_b, stride_h, stride_t; /* in elements; the head_dim axis has stride 1 */
+} csp_tensor;
+
+typedef struct {
+    int32_t batch;        /* B  sequences                                                     */
+    int32_t n_q_heads;    /* H_q, a multiple of n_kv_heads; group size G = H_q / H_kv <= 8     */
+    int32_t n_kv_heads;   /* H_kv                                                             */
+    int32_t head_dim;     /* d; row bytes d*sizeof(elem) must be 128, 256 or 512               */
+    int32_t window;       /* W (the paper's O): 1..32 last queries are the observation window */
+    int32_t recent;       /* R: last R keys are always kept and never scored                  */
+    int32_t max_len;      /* padded key length of k, v, modality and the score vectors        */
+    int32_t out_capacity; /* rows per head available in keep_idx, k_out, v_out, mod_out       */
+    int32_t dtype;        /* csp_dtype: element type of q_win, k, v, k_out, v_out             */
+    float n;              /* the n of n-softmax (Eq. 7); the paper uses 1; 0 gives softmax    */
+    float scale;          /* logit scale; 0 means 1/sqrt(head_dim) (Eq. 5)                    */
+    int32_t combine;      /* csp_combine                                                      */
+    int32_t select_mode;  /* csp_select_mode                                                  */
+    int32_t head_reduce;  /* csp_head_reduce; MEAN_ALL requires shared labels (mod_stride_h == 0) */
+} csp_params;
+
+/* Bytes of scratch that csp_score (MEAN_ALL) and csp_prune_layer need; also holds the status
+ * word.  The first 256 bytes must be zero before first use (csp_workspace_reset). */
+size_t csp_workspace_bytes(const csp_params* p);
+
+/* Enqueue the zeroing of the workspace's status area. */
+csp_status csp_workspace_reset(void* workspace, void* cuda_stream);
+
+/*
+ * Eq. 5, Eq. 7, the window/recent trim and Eq. 1.
+ *   q_win      [B, H_q, W, d]      queries of the last W positions (position L_b-W+w), read-only
+ *   k          [B, H_kv, max_len, d] cached keys; rows >= L_b are ignored
+ *   modality   labels, uint8, element (b,h,t) at modality[b*mod_stride_b + h*mod_stride_h + t]
+ *   seq_lens   [B] int32: L_b.  A sequence with L_b < W or L_b < R is skipped here (and passed
+ *              through unchanged by csp_select)
+ *   lse_or_null [B, H_q, W] fp32: natural log of sum_t exp(logit) over the keys each window row
+ *              sees, if an upstream attention kernel has it; NULL makes the library compute it
+ *   score_self, score_cross [B, H_kv, max_len] fp32 outputs; entries t >= L_b - R are not written
+ * A query at position p sees keys t <= p.  The n-softmax denominator runs over ALL visible keys,
+ * including the last R; only then are those columns dropped.
+ */
+csp_status csp_score(const csp_params* p, csp_tensor q_win, csp_tensor k,
+                     const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                     const int32_t* seq_lens, const float* lse_or_null,
+                     float* score_self, float* score_cross,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Eq. 2, Eq. 3 and the index list of Eq. 4.
+ *   budgets    int32. SEGMENTED: [B,4] = k_self_text, k_self_visual, k_cross_text, k_cross_visual.
+ *              GLOBAL: [B,2] = k_self, k_cross.  Each is clamped to [0, candidates] (flagged).
+ *   total_budget_or_null [B] int32 = T of Algorithm 1: a sequence with L_b < T keeps everything.
+ *   keep_idx   [B, H_kv, out_capacity] int32: kept positions ascending, then L_b-R .. L_b-1
+ *   n_out      [B, H_kv] int32: length of that list; -1 if it would exceed out_capacity (flagged,
+ *              keep_idx of that unit untouched)
+ * Order of a top-K: higher score first; among equal scores the lower position wins (-0 == +0).
+ * Scores must not be NaN.
+ */
+csp_status csp_select(const csp_params* p, const float* score_self, const float* score_cross,
+                      const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                      const int32_t* seq_lens, const int32_t* budgets,
+                      const int32_t* total_budget_or_null,
+                      int32_t* keep_idx, int32_t* n_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Eq. 4: k_out[b,h,j,:] = k[b,h,keep_idx[b,h,j],:] for j < n_out[b,h]; same for v and the labels.
+ *   k_out, v_out [B, H_kv, out_capacity, d] (strided); mod_out [B, H_kv, out_capacity] dense, may
+ *   be NULL.  Rows j >= n_out are left as they were; units with n_out <= 0 are skipped.
+ */
+csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v,
+                       const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                       const int32_t* keep_idx, const int32_t* n_out,
+                       csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, void* cuda_stream);
+
+/*
+ * Algorithm 1, one invocation for one layer: csp_score, csp_select, csp_compact back to back on
+ * one stream.  score_self / score_cross / keep_idx may be NULL, in which case they live in the
+ * workspace; n_out is required.
+ */
+csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
+                           const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                           const int32_t* seq_lens, const int32_t* budgets,
+                           const int32_t* total_budget_or_null, const float* lse_or_null,
+                           csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
+                           float* score_self_or_null, float* score_cross_or_null,
+                           int32_t* keep_idx_or_null,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of device staging that csp_prune_layer_host needs for these parameters. */
+size_t csp_host_staging_bytes(const csp_params* p);
+
+/*
+ * Algorithm 1 for a caller whose cache lives in HOST memory (pinned memory makes the copies
+ * asynchronous): copies the dense inputs into `staging` (device, caller-owned,
+ * >= csp_host_staging_bytes), runs csp_prune_layer there, copies k_out, v_out, mod_out, n_out
+ * back and waits for the stream.  All *_host tensors are dense: q [B,H_q,W,d],
+ * k, v [B,H_kv,max_len,d], modality [B,max_len] (mod_per_head == 0) or [B,H_kv,max_len],
+ * outputs [B,H_kv,out_capacity,(d)].  dev_status_host (may be NULL) receives the status word.
+ */
+csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const void* k_host,
+                                const void* v_host, const uint8_t* modality_host, int mod_per_head,
+                                const int32_t* seq_lens_host, const int32_t* budgets_host,
+                                const int32_t* total_budget_host_or_null,
+                                void* k_out_host, void* v_out_host, uint8_t* mod_out_host,
+                                int32_t* n_out_host, int32_t* dev_status_host,
+                                void* staging, size_t staging_bytes, void* cuda_stream);
+
+/* Waits for the stream, copies the status word to *host_out (may be NULL), clears it, and returns
+ * CSP_ERR_TIMEOUT if CSP_DEV_TIMEOUT was set, else CSP_OK. */
+csp_status csp_device_status(void* workspace, void* cuda_stream, int32_t* host_out);
+
+const char* csp_status_string(csp_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

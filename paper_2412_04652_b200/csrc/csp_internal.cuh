@@ -1,0 +1,79 @@
+// Internal declarations shared by the translation units of libcsp (not part of the C interface).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "csp.h"
+
+namespace csp {
+
+// ---- workspace layout -------------------------------------------------------------------
+// [0, 256)            status area (word 0 = OR of CSP_DEV_* bits)
+// then, each rounded up to 256 bytes:
+//   score_self  fp32 [B, Hkv, max_len]     (prune_layer when the caller passes NULL)
+//   score_cross fp32 [B, Hkv, max_len]
+//   part_self   fp32 [B, Hkv, max_len]     (MEAN_ALL: per-KV-head partial sums)
+//   part_cross  fp32 [B, Hkv, max_len]
+//   keep_idx    int32 [B, Hkv, out_capacity]
+constexpr size_t kStatusBytes = 256;
+
+struct WorkspaceLayout {
+    size_t score_self, score_cross, part_self, part_cross, keep_idx, total;
+};
+
+inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+inline WorkspaceLayout workspace_layout(const csp_params& p) {
+    WorkspaceLayout w;
+    const size_t units = size_t(p.batch) * size_t(p.n_kv_heads);
+    const size_t sc = round256(units * size_t(p.max_len) * 4);
+    w.score_self = kStatusBytes;
+    w.score_cross = w.score_self + sc;
+    w.part_self = w.score_cross + sc;
+    w.part_cross = w.part_self + sc;
+    w.keep_idx = w.part_cross + sc;
+    w.total = w.keep_idx + round256(units * size_t(p.out_capacity) * 4);
+    return w;
+}
+
+// ---- arguments handed to the kernels ------------------------------------------------------
+struct ScoreArgs {
+    const void* q; int64_t q_sb, q_sh, q_st;        // element strides
+    const uint8_t* modality; int64_t mod_sb, mod_sh;
+    const int32_t* seq_lens;
+    const float* lse;                                // may be null
+    float* score_self; float* score_cross;           // [B, Hkv, max_len]
+    int32_t* status;
+    int32_t n_kv_heads, group, window, recent, max_len;
+    float n, scale_log2, weight;                     // weight = 1/G or 1/Hq
+};
+
+struct SelectArgs {
+    const float* score_self; const float* score_cross;
+    const uint8_t* modality; int64_t mod_sb, mod_sh;
+    const int32_t* seq_lens; const int32_t* budgets; const int32_t* total_budget;
+    int32_t* keep_idx; int32_t* n_out; int32_t* status;
+    int32_t n_kv_heads, window, recent, max_len, out_capacity;
+    int32_t combine_and, global_mode;
+};
+
+struct CompactArgs {
+    const void* k; const void* v; void* k_out; void* v_out;
+    int64_t k_sb, k_sh, k_st, v_sb, v_sh, v_st;      // in 16-byte units
+    int64_t ko_sb, ko_sh, ko_st, vo_sb, vo_sh, vo_st;
+    const uint8_t* modality; int64_t mod_sb, mod_sh; uint8_t* mod_out;
+    const int32_t* keep_idx; const int32_t* n_out;
+    int32_t n_kv_heads, max_len, out_capacity, chunks_per_row;
+};
+
+// ---- host-side launchers (defined next to their kernels) ----------------------------------
+csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s);
+csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,
+                            float* score_self, float* score_cross, const int32_t* seq_lens,
+                            cudaStream_t s);
+csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t s);
+csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_t s);
+
+}  // namespace csp
