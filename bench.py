@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the CSP scoring-and-compaction pass.
+
+A step is one pass of the whole path (score -> select -> compact, i.e. csp_prune_layer) over
+every layer of one synthetic multimodal KV cache.  The reported metric is KV tokens pruned per
+second per layer: (sum of sequence lengths) / (time of one layer's prune).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
+
+With N > 1 (launched under torch.distributed.run) every rank prunes its own replica of the
+workload; there is no exchange step on this path, so the job throughput is the sum.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import csp_synth as synth  # noqa: E402
+
+METRIC = "kv_tokens_pruned_per_sec_per_layer"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------------------------ helpers
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.sm_max = None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def _sample(self):
+        nv = self.nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+        try:
+            r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        except Exception:
+            r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+        for bit, name in names.items():
+            if r & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self._sample()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": []}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def algorithmic_bytes(cfg, n_out_total: int):
+    """Per-layer algorithmic bytes of each kernel (every tensor touched exactly once)."""
+    es = 2 if cfg.dtype == torch.bfloat16 else 4
+    d, Hkv, Hq, W = cfg.head_dim, cfg.n_kv_heads, cfg.n_q_heads, cfg.window
+    sum_l = int(cfg.seq_lens.sum())
+    sum_n = int((cfg.seq_lens - cfg.recent).clip(min=0).sum())
+    score = sum_l * Hkv * d * es + cfg.batch * Hq * W * d * es + sum_l + 2 * 4 * sum_n * Hkv
+    select = 2 * 4 * sum_n * Hkv + sum_n * Hkv + 4 * n_out_total
+    compact = 4 * n_out_total + 2 * 2 * n_out_total * d * es + 2 * n_out_total
+    return {"score": score, "select": select, "compact": compact, "total": score + select + compact}
+
+
+class LayerBuffers:
+    def __init__(self, csp, cfg, p, layer, device):
+        self.q, self.k, self.v = synth.make_layer(cfg, layer, device)
+        B, H, cap, d = cfg.batch, cfg.n_kv_heads, p.out_capacity, cfg.head_dim
+        self.k_out = torch.empty((B, H, cap, d), dtype=cfg.dtype, device=device)
+        self.v_out = torch.empty((B, H, cap, d), dtype=cfg.dtype, device=device)
+        self.mod_out = torch.empty((B, H, cap), dtype=torch.uint8, device=device)
+        self.n_out = torch.zeros((B, H), dtype=torch.int32, device=device)
+        self.ss = torch.empty((B, H, cfg.max_len), dtype=torch.float32, device=device)
+        self.sc = torch.empty((B, H, cfg.max_len), dtype=torch.float32, device=device)
+        self.idx = torch.empty((B, H, cap), dtype=torch.int32, device=device)
+
+
+# ------------------------------------------------------------------------------------ reference arm
+
+def run_reference(args, rank, world):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload."""
+    if rank != 0:
+        return
+    from oracle import csp_oracle as orc
+    orc.build()
+    cfg = synth.config(args.config)
+    G = cfg.group
+    n_units = min(args.ref_units, cfg.n_kv_heads)
+    b = int(np.argmax(cfg.seq_lens)) if cfg.batch > 1 else 0
+    L = int(cfg.seq_lens[b])
+    q, k, v = synth.make_layer(cfg, 0, "cpu")
+    qs = q[b:b + 1, :n_units * G].contiguous()
+    ks, vs = k[b:b + 1, :n_units, :L].contiguous(), v[b:b + 1, :n_units, :L].contiguous()
+    mod = cfg.modality()[b:b + 1, :L]
+    op = orc.Params(1, n_units * G, n_units, cfg.head_dim, cfg.window, cfg.recent, L, cfg.out_capacity(),
+                    dtype=orc.F32 if cfg.dtype == torch.float32 else orc.BF16)
+    tb = None if cfg.total_budget is None else cfg.total_budget[b:b + 1]
+
+    def step():
+        orc.prune_layer(op, qs, ks, vs, mod, np.array([L], np.int32), cfg.budgets[b:b + 1], tb)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    # one sample = n_units of the H_kv heads of one sequence of one layer
+    value = L * n_units / cfg.n_kv_heads / dt
+    sample = f"{n_units} of {cfg.n_kv_heads} KV heads of sequence {b} (L={L}) of one layer per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"configs[{args.config}] {cfg.name}", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ CUDA arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--ref-units", type=int, default=8, help="KV heads per reference-arm step")
+    ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
+    ap.add_argument("--launch", default="graph", choices=["graph", "stream"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-baseline-units", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.steps == 300:
+            args.steps, args.warmup = 5, 1
+        run_reference(args, rank, world)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    from paper_2412_04652_b200 import binding as csp
+    csp.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = synth.config(args.config, budget_pct=args.budget_pct) if args.config == 4 else synth.config(args.config)
+    n_layers = cfg.n_layers
+    n_buf = n_layers if args.layers <= 0 else min(args.layers, n_layers)
+    cap = cfg.out_capacity()
+    p = csp.Params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.recent, cfg.max_len,
+                   cap, dtype=csp.F32 if cfg.dtype == torch.float32 else csp.BF16)
+    mod = torch.from_numpy(cfg.modality()).to(dev)
+    lens = torch.from_numpy(cfg.seq_lens).to(dev)
+    bud = torch.from_numpy(cfg.budgets).to(dev)
+    tot = None if cfg.total_budget is None else torch.from_numpy(cfg.total_budget).to(dev)
+    ws = csp.new_workspace(p, dev)
+    layers = [LayerBuffers(csp, cfg, p, i, dev) for i in range(n_buf)]
+    sum_l = int(cfg.seq_lens.sum())
+
+    def prune(lb):
+        csp.prune_layer(p, lb.q, lb.k, lb.v, mod, lens, bud, lb.k_out, lb.v_out, lb.mod_out, lb.n_out, ws,
+                        total_budget=tot)
+
+    def step():
+        for i in range(n_layers):
+            prune(layers[i % n_buf])
+
+    stream = torch.cuda.Stream(dev)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            step()
+        stream.synchronize()
+        graph = None
+        if args.launch == "graph":
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            for _ in range(3):
+                graph.replay()
+            stream.synchronize()
+        run_step = graph.replay if graph is not None else step
+
+        status = csp.device_status(ws)
+        n_out_total = int(layers[0].n_out.clamp(min=0).sum().item())
+
+        # ---- timed region: K steps, device resident ----
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            run_step()
+        e1.record(stream)
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        ms_total = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms_total], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_total = float(t.item())
+        ms_step = ms_total / args.steps
+        value = world * sum_l * n_layers / (ms_step * 1e-3)
+
+        # ---- per-kernel durations, live, with events on the launching stream ----
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_layers)]
+        reps = 3
+        per = {"score": 0.0, "select": 0.0, "compact": 0.0}
+        for _ in range(reps):
+            for i in range(n_layers):
+                lb = layers[i % n_buf]
+                evs[i][0].record(stream)
+                csp.score(p, lb.q, lb.k, mod, lens, lb.ss, lb.sc, ws)
+                evs[i][1].record(stream)
+                csp.select(p, lb.ss, lb.sc, mod, lens, bud, lb.idx, lb.n_out, ws, total_budget=tot)
+                evs[i][2].record(stream)
+                csp.compact(p, lb.k, lb.v, mod, lb.idx, lb.n_out, lb.k_out, lb.v_out, lb.mod_out)
+                evs[i][3].record(stream)
+            stream.synchronize()
+            for i in range(n_layers):
+                per["score"] += evs[i][0].elapsed_time(evs[i][1])
+                per["select"] += evs[i][1].elapsed_time(evs[i][2])
+                per["compact"] += evs[i][2].elapsed_time(evs[i][3])
+        per = {k_: v_ / (reps * n_layers) for k_, v_ in per.items()}   # ms per launch
+        status |= csp.device_status(ws)
+
+    peak, peak_kind = measured_peaks()
+    ab = algorithmic_bytes(cfg, n_out_total)
+    dominant = max(per, key=per.get)
+    achieved = ab[dominant] / (per[dominant] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": ab[dominant], "us_per_launch": per[dominant] * 1e3}
+    path = {"algorithmic_bytes_per_layer": ab["total"], "us_per_layer": ms_step * 1e3 / n_layers,
+            "achieved_gbs": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9,
+            "frac_of_hbm_peak": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9 / peak,
+            "kernel_us": {k_: v_ * 1e3 for k_, v_ in per.items()},
+            "kernel_gbs": {k_: ab[k_] / (per[k_] * 1e-3) / 1e9 for k_ in per}}
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) ----
+    e2e = None
+    if args.e2e_steps > 0:
+        n_host = min(n_buf, 4)
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        host = []
+        for i in range(n_host):
+            lb = layers[i]
+            host.append(dict(q=pin(lb.q), k=pin(lb.k), v=pin(lb.v), k_out=pin(lb.k_out), v_out=pin(lb.v_out),
+                             mod_out=pin(lb.mod_out), n_out=pin(lb.n_out)))
+        h_mod, h_lens, h_bud = pin(mod), pin(lens), pin(bud)
+        h_tot = None if tot is None else pin(tot)
+        staging = torch.empty(csp.host_staging_bytes(p), dtype=torch.uint8, device=dev)
+
+        def host_step():
+            for i in range(n_layers):
+                hb = host[i % n_host]
+                csp.prune_layer_host(p, hb["q"], hb["k"], hb["v"], h_mod, h_lens, h_bud, hb["k_out"], hb["v_out"],
+                                     hb["mod_out"], hb["n_out"], staging, total_budget=h_tot)
+
+        with torch.cuda.stream(stream):
+            host_step()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.e2e_steps):
+                host_step()
+            e1.record(stream)
+            stream.synchronize()
+            ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        hb = host[0]
+        h2d = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("q", "k", "v")) + \
+            n_layers * (h_mod.numel() + 4 * h_lens.numel() + 4 * h_bud.numel())
+        d2h = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("k_out", "v_out", "mod_out", "n_out"))
+        e2e = {"value": world * sum_l * n_layers / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "api": "csp_prune_layer_host"}
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N=1 only ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import csp_oracle as orc
+        orc.build()
+        G = cfg.group
+        b = int(np.argmax(cfg.seq_lens)) if cfg.batch > 1 else 0
+        L = int(cfg.seq_lens[b])
+        n_units = min(args.cpu_baseline_units, cfg.n_kv_heads)
+        lb = layers[0]
+        qs = lb.q[b:b + 1, :n_units * G].cpu().contiguous()
+        ks, vs = lb.k[b:b + 1, :n_units, :L].cpu().contiguous(), lb.v[b:b + 1, :n_units, :L].cpu().contiguous()
+        op = orc.Params(1, n_units * G, n_units, cfg.head_dim, cfg.window, cfg.recent, L, cap,
+                        dtype=orc.F32 if cfg.dtype == torch.float32 else orc.BF16)
+        t0 = time.perf_counter()
+        reps_cpu = 0
+        while reps_cpu < 1 or (time.perf_counter() - t0 < 10.0 and reps_cpu < 50):
+            orc.prune_layer(op, qs, ks, vs, cfg.modality()[b:b + 1, :L], np.array([L], np.int32),
+                            cfg.budgets[b:b + 1], None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
+            reps_cpu += 1
+        dt = (time.perf_counter() - t0) / reps_cpu
+        cpu_baseline = {"value": L * n_units / cfg.n_kv_heads / dt, "unit": UNIT, "cores": orc.num_threads(),
+                        "kind": "oracle",
+                        "sample": f"{n_units} of {cfg.n_kv_heads} KV heads of sequence {b} (L={L}) of layer 0, "
+                                  f"{reps_cpu} repetitions, {dt:.3f} s each"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == torch.bfloat16 else "f32",
+                "data": "synthetic",
+                "config": {"workload": f"configs[{args.config}] {cfg.name}", "layers": n_layers,
+                           "distinct_layer_buffers": n_buf, "batch": cfg.batch, "kv_heads": cfg.n_kv_heads,
+                           "q_heads": cfg.n_q_heads, "head_dim": cfg.head_dim, "sum_seq_len": sum_l,
+                           "window": cfg.window, "recent": cfg.recent, "kept_rows_per_layer": n_out_total,
+                           "launch": "cuda_graph of one step" if graph is not None else "stream",
+                           "l2": "inputs larger than L2: every layer has its own K/V buffers"
+                                 if n_buf * ab["score"] > 2 * 126e6 else "inputs smaller than L2",
+                           "replicas": "one independent replica per GPU, no collective"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * n_layers * 3,
+                "roofline": roofline, "path": path, "cpu_baseline": cpu_baseline, "device_status": status}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,221 @@
+"""Thin ctypes binding of libcsp.so: same names as the C interface, argument marshalling only.
+
+Every step of the path runs inside the CUDA library; PyTorch is used for device memory and for
+the current stream.  There is no CPU fallback: if the library is missing, import of the symbols
+fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcsp.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
+F32, BF16 = 0, 1
+COMBINE_OR, COMBINE_AND = 0, 1
+SELECT_SEGMENTED, SELECT_GLOBAL = 0, 1
+HEADS_PER_KV, HEADS_MEAN_ALL = 0, 1
+DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
+
+EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_select", "csp_compact",
+           "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
+           "csp_status_string")
+
+
+class CspError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (csp_status {code})")
+
+
+class CTensor(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
+
+
+class CParams(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("window", C.c_int32), ("recent", C.c_int32),
+                ("max_len", C.c_int32), ("out_capacity", C.c_int32), ("dtype", C.c_int32),
+                ("n", C.c_float), ("scale", C.c_float), ("combine", C.c_int32),
+                ("select_mode", C.c_int32), ("head_reduce", C.c_int32)]
+
+
+@dataclass
+class Params:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    window: int
+    recent: int
+    max_len: int
+    out_capacity: int
+    dtype: int = BF16
+    n: float = 1.0
+    scale: float = 0.0
+    combine: int = COMBINE_OR
+    select_mode: int = SELECT_SEGMENTED
+    head_reduce: int = HEADS_PER_KV
+
+    def c(self) -> CParams:
+        return CParams(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.window,
+                       self.recent, self.max_len, self.out_capacity, self.dtype, self.n, self.scale,
+                       self.combine, self.select_mode, self.head_reduce)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libcsp.so; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2412_04652_b200.build`")
+        l = C.CDLL(LIB_PATH)
+        P = C.POINTER(CParams)
+        vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+        l.csp_workspace_bytes.restype = sz
+        l.csp_workspace_bytes.argtypes = [P]
+        l.csp_workspace_reset.restype = C.c_int
+        l.csp_workspace_reset.argtypes = [vp, vp]
+        l.csp_score.restype = C.c_int
+        l.csp_score.argtypes = [P, CTensor, CTensor, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp]
+        l.csp_select.restype = C.c_int
+        l.csp_select.argtypes = [P, vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        l.csp_compact.restype = C.c_int
+        l.csp_compact.argtypes = [P, CTensor, CTensor, vp, i64, i64, vp, vp, CTensor, CTensor, vp, vp]
+        l.csp_prune_layer.restype = C.c_int
+        l.csp_prune_layer.argtypes = [P, CTensor, CTensor, CTensor, vp, i64, i64, vp, vp, vp, vp,
+                                      CTensor, CTensor, vp, vp, vp, vp, vp, vp, sz, vp]
+        l.csp_host_staging_bytes.restype = sz
+        l.csp_host_staging_bytes.argtypes = [P]
+        l.csp_prune_layer_host.restype = C.c_int
+        l.csp_prune_layer_host.argtypes = [P, vp, vp, vp, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp,
+                                           vp, sz, vp]
+        l.csp_device_status.restype = C.c_int
+        l.csp_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+        l.csp_status_string.restype = C.c_char_p
+        l.csp_status_string.argtypes = [C.c_int]
+        _lib = l
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().csp_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise CspError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def tensor4(t: torch.Tensor) -> CTensor:
+    """[B, H, T, d] tensor -> (pointer, element strides); the last axis must be contiguous."""
+    assert t.dim() == 4 and (t.stride(3) == 1 or t.shape[3] == 1), "head_dim axis must be contiguous"
+    return CTensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _mod_strides(modality: torch.Tensor):
+    """[B, L] (shared by the heads) or [B, H, L] labels -> (stride_b, stride_h)."""
+    assert modality.dtype == torch.uint8 and modality.stride(-1) == 1
+    if modality.dim() == 2:
+        return modality.stride(0), 0
+    return modality.stride(0), modality.stride(1)
+
+
+def workspace_bytes(p: Params) -> int:
+    cp = p.c()
+    return int(lib().csp_workspace_bytes(C.byref(cp)))
+
+
+def new_workspace(p: Params, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and zeroes a workspace for these parameters."""
+    n = workspace_bytes(p)
+    if n == 0:
+        raise CspError(ERR_UNSUPPORTED, "csp_workspace_bytes")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def workspace_reset(ws: torch.Tensor):
+    _check(lib().csp_workspace_reset(_ptr(ws), _stream()), "csp_workspace_reset")
+
+
+def score(p: Params, q_win, k, modality, seq_lens, score_self, score_cross, ws, lse=None):
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_score(C.byref(cp), tensor4(q_win), tensor4(k), _ptr(modality), sb, sh, _ptr(seq_lens),
+                           _ptr(lse), _ptr(score_self), _ptr(score_cross), _ptr(ws), ws.numel(), _stream()),
+           "csp_score")
+
+
+def select(p: Params, score_self, score_cross, modality, seq_lens, budgets, keep_idx, n_out, ws,
+           total_budget=None):
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_select(C.byref(cp), _ptr(score_self), _ptr(score_cross), _ptr(modality), sb, sh,
+                            _ptr(seq_lens), _ptr(budgets), _ptr(total_budget), _ptr(keep_idx), _ptr(n_out),
+                            _ptr(ws), ws.numel(), _stream()), "csp_select")
+
+
+def compact(p: Params, k, v, modality, keep_idx, n_out, k_out, v_out, mod_out=None):
+    cp = p.c()
+    sb, sh = _mod_strides(modality) if modality is not None else (0, 0)
+    _check(lib().csp_compact(C.byref(cp), tensor4(k), tensor4(v), _ptr(modality), sb, sh, _ptr(keep_idx),
+                             _ptr(n_out), tensor4(k_out), tensor4(v_out), _ptr(mod_out), _stream()),
+           "csp_compact")
+
+
+def prune_layer(p: Params, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, mod_out, n_out, ws,
+                total_budget=None, lse=None, score_self=None, score_cross=None, keep_idx=None):
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_prune_layer(C.byref(cp), tensor4(q_win), tensor4(k), tensor4(v), _ptr(modality), sb, sh,
+                                 _ptr(seq_lens), _ptr(budgets), _ptr(total_budget), _ptr(lse),
+                                 tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
+                                 _ptr(score_self), _ptr(score_cross), _ptr(keep_idx),
+                                 _ptr(ws), ws.numel(), _stream()), "csp_prune_layer")
+
+
+def host_staging_bytes(p: Params) -> int:
+    cp = p.c()
+    return int(lib().csp_host_staging_bytes(C.byref(cp)))
+
+
+def prune_layer_host(p: Params, q, k, v, modality, seq_lens, budgets, k_out, v_out, mod_out, n_out,
+                     staging: torch.Tensor, total_budget=None) -> int:
+    """All tensors but `staging` are dense CPU tensors (pinned for asynchronous copies).
+    Returns the device status word."""
+    cp = p.c()
+    for t in (q, k, v, modality, seq_lens, budgets, k_out, v_out, n_out):
+        assert t.device.type == "cpu" and t.is_contiguous()
+    word = C.c_int32(0)
+    _check(lib().csp_prune_layer_host(C.byref(cp), _ptr(q), _ptr(k), _ptr(v), _ptr(modality),
+                                      int(modality.dim() == 3), _ptr(seq_lens), _ptr(budgets),
+                                      _ptr(total_budget), _ptr(k_out), _ptr(v_out), _ptr(mod_out),
+                                      _ptr(n_out), C.addressof(word), _ptr(staging), staging.numel(),
+                                      _stream()), "csp_prune_layer_host")
+    return int(word.value)
+
+
+def device_status(ws: torch.Tensor) -> int:
+    """Waits for the current stream, returns the status word (CSP_DEV_* bits) and clears it."""
+    word = C.c_int32(0)
+    rc = lib().csp_device_status(_ptr(ws), _stream(), C.byref(word))
+    if rc not in (OK, ERR_TIMEOUT):
+        raise CspError(rc, "csp_device_status")
+    return int(word.value)

@@ -1,0 +1,156 @@
+"""Helpers shared by the GPU parity tests: run the CUDA library and the CPU oracle on the same
+bytes and compare under the stated tolerances."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+REL_TOL = 2e-3      # scores: |gpu - oracle| <= REL_TOL * |oracle| + ABS_FRAC * max|oracle score of the unit|
+ABS_FRAC = 1e-6
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    """Raw element bits of a CPU/GPU tensor (bf16 -> uint16, fp32 -> uint32)."""
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    if t.dtype == torch.float32:
+        return t.view(torch.int32).numpy().view(np.uint32)
+    return t.numpy()
+
+
+def gpu_params(csp, cfg, cap=None, **kw):
+    return csp.Params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.recent,
+                      cfg.max_len, cap if cap is not None else cfg.out_capacity(),
+                      dtype=csp.F32 if cfg.dtype == torch.float32 else csp.BF16, **kw)
+
+
+def orc_params(orc, cfg, cap=None, **kw):
+    return orc.Params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.recent,
+                      cfg.max_len, cap if cap is not None else cfg.out_capacity(),
+                      dtype=orc.F32 if cfg.dtype == torch.float32 else orc.BF16, **kw)
+
+
+def assert_scores_close(got: np.ndarray, want: np.ndarray, seq_lens, recent, what=""):
+    """got, want: [B, H, max_len]; compared on the candidates t < L_b - R of every unit."""
+    B, H, _ = want.shape
+    for b in range(B):
+        N = int(seq_lens[b]) - recent
+        if N <= 0:
+            continue
+        for h in range(H):
+            w, g = want[b, h, :N].astype(np.float64), got[b, h, :N].astype(np.float64)
+            tol = REL_TOL * np.abs(w) + ABS_FRAC * np.abs(w).max()
+            bad = np.abs(g - w) > tol
+            assert not bad.any(), (f"{what} unit ({b},{h}): {bad.sum()} of {N} scores off; worst at "
+                                   f"t={np.argmax(np.abs(g - w) - tol)} got {g[np.argmax(np.abs(g - w) - tol)]} "
+                                   f"want {w[np.argmax(np.abs(g - w) - tol)]}")
+            zero = w == 0.0
+            assert (g[zero] == 0.0).all(), f"{what} unit ({b},{h}): structural zeros must be exactly 0"
+
+
+def assert_index_sets_match(gpu_idx, gpu_n, ref, modality, seq_lens, recent, global_mode=False):
+    """Kept sets must be identical except for keys whose oracle score lies within REL_TOL of the
+    K-th (boundary) score of a top-K problem the key takes part in.  Returns the number of
+    boundary-band differences that were tolerated."""
+    B, H = ref["n_out"].shape
+    tolerated = 0
+    for b in range(B):
+        L = int(seq_lens[b])
+        for h in range(H):
+            n_ref, n_gpu = int(ref["n_out"][b, h]), int(gpu_n[b, h])
+            if n_ref < 0:
+                assert n_gpu == -1
+                continue
+            got = gpu_idx[b, h, :n_gpu]
+            want = ref["keep_idx"][b, h, :n_ref]
+            assert (np.diff(got) > 0).all(), "kept positions must be strictly ascending"
+            if ref["flags"][b, h] & 4:      # identity
+                np.testing.assert_array_equal(got, want)
+                continue
+            np.testing.assert_array_equal(got[-recent:] if recent else got[:0], np.arange(L - recent, L))
+            diff = set(got.tolist()) ^ set(want.tolist())
+            if not diff:
+                continue
+            mod = modality[b, h] if modality.ndim == 3 else modality[b]
+            mg = ref["margins"][b, h]
+            for t in diff:
+                vis = int(mod[t] != 0)
+                probs = [(0, ref["score_self"]), (1, ref["score_cross"])] if global_mode else \
+                        [(vis, ref["score_self"]), (2 + vis, ref["score_cross"])]
+                ok = False
+                for pidx, sc in probs:
+                    kth = float(mg[pidx, 0])
+                    if np.isnan(kth):
+                        continue
+                    s = float(sc[b, h, t])
+                    if abs(s - kth) <= REL_TOL * abs(kth) + ABS_FRAC * float(np.abs(sc[b, h, :L - recent]).max()):
+                        ok = True
+                assert ok, f"unit ({b},{h}) key {t} differs and is not at a top-K boundary"
+                tolerated += 1
+    return tolerated
+
+
+class GpuRun:
+    """Device copies of one layer's inputs plus freshly allocated outputs."""
+
+    def __init__(self, csp, p, q, k, v, modality, seq_lens, budgets, total_budget=None, lse=None):
+        dev = "cuda"
+        self.csp, self.p = csp, p
+        self.q, self.k, self.v = q.to(dev), k.to(dev), v.to(dev)
+        self.mod = torch.as_tensor(np.ascontiguousarray(modality)).to(dev)
+        self.lens = torch.as_tensor(np.asarray(seq_lens, np.int32)).to(dev)
+        self.bud = torch.as_tensor(np.ascontiguousarray(np.asarray(budgets, np.int32))).to(dev)
+        self.tot = None if total_budget is None else torch.as_tensor(np.asarray(total_budget, np.int32)).to(dev)
+        self.lse = None if lse is None else torch.as_tensor(np.asarray(lse, np.float32)).to(dev)
+        B, H, cap, d = p.batch, p.n_kv_heads, p.out_capacity, p.head_dim
+        self.ss = torch.full((B, H, p.max_len), -7.0, device=dev)
+        self.sc = torch.full((B, H, p.max_len), -7.0, device=dev)
+        self.idx = torch.full((B, H, cap), -1, dtype=torch.int32, device=dev)
+        self.n_out = torch.full((B, H), -99, dtype=torch.int32, device=dev)
+        self.k_out = torch.zeros((B, H, cap, d), dtype=self.k.dtype, device=dev)
+        self.v_out = torch.zeros((B, H, cap, d), dtype=self.k.dtype, device=dev)
+        self.mod_out = torch.zeros((B, H, cap), dtype=torch.uint8, device=dev)
+        self.ws = csp.new_workspace(p)
+
+    def score(self):
+        self.csp.score(self.p, self.q, self.k, self.mod, self.lens, self.ss, self.sc, self.ws, lse=self.lse)
+        return self
+
+    def select(self):
+        self.csp.select(self.p, self.ss, self.sc, self.mod, self.lens, self.bud, self.idx, self.n_out, self.ws,
+                        total_budget=self.tot)
+        return self
+
+    def compact(self):
+        self.csp.compact(self.p, self.k, self.v, self.mod, self.idx, self.n_out, self.k_out, self.v_out,
+                         self.mod_out)
+        return self
+
+    def prune(self, with_optional=True):
+        kw = dict(score_self=self.ss, score_cross=self.sc, keep_idx=self.idx) if with_optional else {}
+        self.csp.prune_layer(self.p, self.q, self.k, self.v, self.mod, self.lens, self.bud, self.k_out,
+                             self.v_out, self.mod_out, self.n_out, self.ws, total_budget=self.tot,
+                             lse=self.lse, **kw)
+        return self
+
+    def status(self) -> int:
+        return self.csp.device_status(self.ws)
+
+
+def assert_compaction_exact(run: GpuRun, modality):
+    """k_out/v_out/mod_out must be the rows named by the GPU's own index list, bit for bit."""
+    idx, n_out = run.idx.cpu().numpy(), run.n_out.cpu().numpy()
+    kb, vb = bits(run.k), bits(run.v)
+    ko, vo, mo = bits(run.k_out), bits(run.v_out), run.mod_out.cpu().numpy()
+    B, H = n_out.shape
+    for b in range(B):
+        for h in range(H):
+            n = int(n_out[b, h])
+            if n <= 0:
+                continue
+            ii = idx[b, h, :n]
+            np.testing.assert_array_equal(ko[b, h, :n], kb[b, h][ii])
+            np.testing.assert_array_equal(vo[b, h, :n], vb[b, h][ii])
+            mod = modality[b, h] if modality.ndim == 3 else modality[b]
+            np.testing.assert_array_equal(mo[b, h, :n], mod[ii])

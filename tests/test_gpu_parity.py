@@ -1,0 +1,460 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, on the same seeded
+inputs, through the C interface.  Sizes span several 128-key tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import csp_synth as synth
+from parity_util import (GpuRun, assert_compaction_exact, assert_index_sets_match, assert_scores_close,
+                         bits, gpu_params, orc_params)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def csp():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2412_04652_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _layout(L, n_img, img_len, seed):
+    rng = np.random.RandomState(seed)
+    img_len = max(1, min(img_len, (L - 40) // n_img))
+    text = L - n_img * img_len
+    assert text >= 40
+    cuts = np.sort(rng.randint(0, text - 40 + 1, size=n_img))
+    spans = np.diff(np.concatenate([[0], cuts, [text - 40]])).tolist()
+    spans[-1] += 40
+    return synth.interleaved_layout(spans, img_len)
+
+
+def _case(lens, n_q, n_kv, d, W, R, dtype=torch.bfloat16, seed=0, img=(2, 50), **kw):
+    lays = [_layout(L, img[0], img[1], seed + i) for i, L in enumerate(lens)]
+    return synth.small_config("case", lays, n_q, n_kv, d, W, R, dtype=dtype, seed=seed, **kw)
+
+
+def _run_score(csp, oracle, cfg, modality=None, gpu_kw=None, orc_kw=None, q_gain=1.0, lse=None):
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    if q_gain != 1.0:
+        q = (q.float() * q_gain).to(cfg.dtype)
+    mod = cfg.modality() if modality is None else modality
+    p = gpu_params(csp, cfg, **(gpu_kw or {}))
+    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, cfg.budgets, lse=lse).score()
+    assert run.status() == 0
+    op = orc_params(oracle, cfg, **(orc_kw or {}))
+    s, c = oracle.score(op, q.cpu(), k.cpu(), mod, cfg.seq_lens, lse=lse)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent, "self")
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent, "cross")
+    return run, s, c
+
+
+# ------------------------------------------------------------------ score
+
+@pytest.mark.parametrize("lens,n_q,n_kv,d,W,R,dtype", [
+    ((300,), 2, 2, 128, 32, 32, torch.bfloat16),            # MHA, 3 tiles, ragged tail
+    ((517, 130, 1029), 4, 4, 128, 32, 32, torch.bfloat16),  # ragged batch
+    ((700,), 4, 2, 128, 32, 32, torch.bfloat16),            # GQA G=2
+    ((700, 257), 12, 4, 128, 32, 32, torch.bfloat16),       # G=3
+    ((390,), 4, 1, 128, 32, 32, torch.bfloat16),            # G=4
+    ((450,), 5, 1, 64, 32, 32, torch.bfloat16),             # G=5, 128-byte rows
+    ((1300, 640), 7, 1, 128, 32, 32, torch.bfloat16),       # G=7 (the GQA benchmark shape)
+    ((333,), 8, 1, 128, 16, 16, torch.bfloat16),            # G=8, narrow window
+    ((1024,), 4, 4, 64, 16, 16, torch.float32),             # fp32 (3xTF32)
+    ((500,), 4, 2, 128, 32, 32, torch.float32),             # fp32, 512-byte rows, G=2
+    ((400,), 2, 2, 256, 32, 32, torch.bfloat16),            # 512-byte bf16 rows
+    ((260,), 2, 2, 128, 5, 9, torch.bfloat16),              # odd window, R > W
+    ((260,), 2, 2, 128, 32, 7, torch.bfloat16),             # R < W: causal mask cuts into candidates
+    ((129,), 1, 1, 128, 32, 0, torch.bfloat16),             # R = 0
+    ((128,), 2, 2, 128, 32, 32, torch.bfloat16),            # exactly one tile
+    ((64,), 2, 2, 128, 32, 32, torch.bfloat16),             # less than a tile
+])
+def test_score_matches_oracle(csp, oracle, lens, n_q, n_kv, d, W, R, dtype):
+    _run_score(csp, oracle, _case(lens, n_q, n_kv, d, W, R, dtype=dtype, seed=len(lens) + n_q))
+
+
+def test_score_mixed_modality_window_and_per_head_labels(csp, oracle):
+    cfg = _case((600, 350), 4, 2, 128, 32, 32, seed=5)
+    rng = np.random.RandomState(0)
+    mod = (rng.rand(2, 2, cfg.max_len) < 0.5).astype(np.uint8)      # per head, random incl. the window
+    _run_score(csp, oracle, cfg, modality=mod)
+    mod3 = (rng.randint(0, 3, size=(2, cfg.max_len))).astype(np.uint8)  # three labels
+    _run_score(csp, oracle, cfg, modality=mod3)
+
+
+@pytest.mark.parametrize("n", [0.0, 1.0, 100.0])
+def test_score_n_sensitive(csp, oracle, n):
+    # logits ~ 8 * N(0,1) - 20: the exponential mass is comparable to or far below n
+    cfg = _case((200, 64), 2, 2, 128, 32, 32, seed=7)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    q = (q.float() * 8).to(cfg.dtype)
+    q[..., 0] = 1.0
+    k[..., 0] = -20.0 * np.sqrt(128)
+    p = gpu_params(csp, cfg, n=n)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).score()
+    assert run.status() == 0
+    s, c = oracle.score(orc_params(oracle, cfg, n=n), q.cpu(), k.cpu(), cfg.modality(), cfg.seq_lens)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent)
+
+
+def test_score_large_logits_and_explicit_scale(csp, oracle):
+    cfg = _case((300,), 2, 2, 128, 32, 32, seed=8)
+    _run_score(csp, oracle, cfg, q_gain=6.0)
+    _run_score(csp, oracle, cfg, gpu_kw=dict(scale=0.25), orc_kw=dict(scale=0.25))
+
+
+def test_score_all_zero_queries_closed_form(csp, oracle):
+    cfg = _case((300,), 2, 2, 128, 32, 32, seed=9)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    q.zero_()
+    mod = cfg.modality()
+    run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod, cfg.seq_lens, cfg.budgets).score()
+    L, W = 300, 32
+    want = sum(1.0 / (1.0 + (L - W + w) + 1) for w in range(W))   # every window row is text here
+    s, c = run.ss.cpu().numpy()[0, 0, :L - 32], run.sc.cpu().numpy()[0, 0, :L - 32]
+    text = mod[0, :L - 32] == 0
+    np.testing.assert_allclose(s[text], want, rtol=1e-5)
+    np.testing.assert_allclose(c[~text], want, rtol=1e-5)
+    assert (s[~text] == 0).all() and (c[text] == 0).all()
+
+
+def test_score_with_supplied_lse(csp, oracle):
+    cfg = _case((500, 200), 4, 2, 128, 32, 32, seed=10)
+    q, k, v = synth.make_layer(cfg, 0, "cpu")
+    G = 2
+    lse = np.zeros((2, 4, 32))
+    for b in range(2):
+        L = int(cfg.seq_lens[b])
+        for hq in range(4):
+            o = (q[b, hq].double() @ k[b, hq // G, :L].double().T / np.sqrt(128)).numpy()
+            for w in range(32):
+                lse[b, hq, w] = np.log(np.exp(o[w, :L - 32 + w + 1]).sum())
+    p = gpu_params(csp, cfg)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets, lse=lse).score()
+    s, c = oracle.score(orc_params(oracle, cfg), q, k, cfg.modality(), cfg.seq_lens)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent)
+
+
+def test_score_mean_over_all_heads(csp, oracle):
+    cfg = _case((420, 300), 8, 4, 128, 32, 32, seed=11)
+    _run_score(csp, oracle, cfg, gpu_kw=dict(head_reduce=csp.HEADS_MEAN_ALL),
+               orc_kw=dict(head_reduce=oracle.HEADS_MEAN_ALL))
+
+
+def test_score_strided_views_and_padding_ignored(csp, oracle):
+    cfg = _case((300, 200), 4, 2, 128, 32, 32, seed=12)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    big = torch.full((2, 2, cfg.max_len + 24, 256), float("nan"), dtype=k.dtype, device="cuda")
+    big[:, :, 8:8 + cfg.max_len, 128:] = k
+    kview = big[:, :, 8:8 + cfg.max_len, 128:]
+    kview[1, :, 200:] = float("nan")                      # padding rows hold NaN
+    p = gpu_params(csp, cfg)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets)
+    run.k = kview
+    run.score()
+    assert run.status() == 0
+    s, c = oracle.score(orc_params(oracle, cfg), q.cpu(), k.cpu(), cfg.modality(), cfg.seq_lens)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent)
+
+
+def test_score_is_bit_reproducible(csp, oracle):
+    cfg = _case((900, 400), 7, 1, 128, 32, 32, seed=13)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    runs = [GpuRun(csp, gpu_params(csp, cfg), q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).score()
+            for _ in range(2)]
+    for b, L in enumerate(cfg.seq_lens):
+        assert torch.equal(runs[0].ss[b, :, :L - 32], runs[1].ss[b, :, :L - 32])
+        assert torch.equal(runs[0].sc[b, :, :L - 32], runs[1].sc[b, :, :L - 32])
+
+
+# ------------------------------------------------------------------ select (bit-exact on equal fp32 scores)
+
+def _select_case(csp, oracle, B, H, lens, R, budgets, quantise=None, seed=0, total=None, cap=None, **mode):
+    rng = np.random.RandomState(seed)
+    Lm = max(lens)
+    s = rng.rand(B, H, Lm).astype(np.float32)
+    c = rng.rand(B, H, Lm).astype(np.float32)
+    if quantise:
+        s, c = np.floor(s * quantise) / quantise, np.floor(c * quantise) / quantise
+    mod = (rng.rand(B, Lm) < 0.6).astype(np.uint8)
+    cap = cap if cap is not None else Lm
+    kw = dict(combine=mode.get("combine", 0), select_mode=mode.get("select_mode", 0))
+    p = csp.Params(B, H, H, 128, min(32, min(lens)) if min(lens) > 0 else 1, R, Lm, cap, **kw)
+    dummy = torch.zeros(B, H, 1, 128, dtype=torch.bfloat16)
+    run = GpuRun(csp, p, dummy, dummy, dummy, mod, lens, budgets, total_budget=total)
+    run.ss, run.sc = torch.from_numpy(s).cuda(), torch.from_numpy(c).cuda()
+    run.select()
+    op = oracle.Params(B, H, H, 128, p.window, R, Lm, cap, **kw)
+    idx, n_out, flags, _ = oracle.select(op, s, c, mod, np.array(lens, np.int32), np.array(budgets, np.int32),
+                                         None if total is None else np.array(total, np.int32))
+    gi, gn = run.idx.cpu().numpy(), run.n_out.cpu().numpy()
+    np.testing.assert_array_equal(gn, n_out)
+    for b in range(B):
+        for h in range(H):
+            n = n_out[b, h]
+            if n > 0:
+                np.testing.assert_array_equal(gi[b, h, :n], idx[b, h, :n])
+    return run.status(), flags
+
+
+@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1), dict(select_mode=1, combine=1)])
+def test_select_matches_oracle_exactly(csp, oracle, mode):
+    lens = (3000, 1500, 777)
+    nb = 2 if mode.get("select_mode") else 4
+    budgets = np.random.RandomState(1).randint(0, 400, size=(3, nb))
+    _select_case(csp, oracle, 3, 2, lens, 32, budgets, seed=1, **mode)
+    _select_case(csp, oracle, 3, 2, lens, 32, budgets, quantise=16, seed=2, **mode)   # heavy ties
+
+
+def test_select_all_equal_scores_and_extreme_budgets(csp, oracle):
+    lens = (2100, 40)
+    st, flags = _select_case(csp, oracle, 2, 1, lens, 8, [[5, 7, 0, 0], [0, 0, 0, 0]], quantise=1, seed=3)
+    assert st == 0
+    st, flags = _select_case(csp, oracle, 2, 1, lens, 8, [[100000, 100000, 3, -4], [1, 1, 1, 1]], seed=4)
+    assert st == csp.DEV_K_CLAMPED and (flags[0] & oracle.FLAG_K_CLAMPED).all()
+
+
+def test_select_identity_capacity_and_short_sequences(csp, oracle):
+    st, flags = _select_case(csp, oracle, 3, 2, (500, 20, 0), 32, [[10, 10, 10, 10]] * 3, seed=5, total=[501, 0, 0])
+    assert st == 0 and (flags & oracle.FLAG_IDENTITY).all()
+    st, flags = _select_case(csp, oracle, 2, 1, (500, 300), 32, [[40, 40, 40, 40], [2, 2, 2, 2]], seed=6, cap=64)
+    assert st == csp.DEV_CAPACITY and (flags[0] & oracle.FLAG_CAPACITY).all() and not flags[1].any()
+
+
+def test_select_long_sequence(csp, oracle):
+    _select_case(csp, oracle, 1, 2, (32768,), 32, [[1626, 0, 0, 4301]], seed=7)
+    _select_case(csp, oracle, 1, 1, (32768,), 32, [[1626, 3, 9, 4301]], quantise=64, seed=8)
+
+
+def test_select_negative_and_signed_zero_scores(csp, oracle):
+    rng = np.random.RandomState(9)
+    s = rng.randn(1, 1, 700).astype(np.float32)
+    s[0, 0, ::7] = 0.0
+    s[0, 0, 3::7] = -0.0
+    c = -s
+    mod = np.zeros((1, 700), np.uint8)
+    p = csp.Params(1, 1, 1, 128, 32, 32, 700, 700, select_mode=1)
+    dummy = torch.zeros(1, 1, 1, 128, dtype=torch.bfloat16)
+    run = GpuRun(csp, p, dummy, dummy, dummy, mod, [700], [[300, 250]])
+    run.ss, run.sc = torch.from_numpy(s).cuda(), torch.from_numpy(c).cuda()
+    run.select()
+    idx, n_out, _, _ = oracle.select(oracle.Params(1, 1, 1, 128, 32, 32, 700, 700, select_mode=1), s, c, mod,
+                                     np.array([700], np.int32), np.array([[300, 250]], np.int32))
+    n = int(n_out[0, 0])
+    assert int(run.n_out[0, 0]) == n
+    np.testing.assert_array_equal(run.idx.cpu().numpy()[0, 0, :n], idx[0, 0, :n])
+
+
+# ------------------------------------------------------------------ compact
+
+def test_compact_is_bit_exact_with_strides(csp, oracle):
+    cfg = _case((400, 250), 4, 2, 128, 32, 32, seed=20)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    p = gpu_params(csp, cfg, cap=300)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets)
+    rng = np.random.RandomState(0)
+    idx = np.full((2, 2, 300), -1, np.int32)
+    n_out = np.array([[300, 17], [0, -1]], np.int32)
+    for b in range(2):
+        for h in range(2):
+            n = max(int(n_out[b, h]), 0)
+            idx[b, h, :n] = np.sort(rng.choice(int(cfg.seq_lens[b]), n, replace=False))
+    run.idx, run.n_out = torch.from_numpy(idx).cuda(), torch.from_numpy(n_out).cuda()
+    wide = torch.zeros(2, 2, 300, 256, dtype=k.dtype, device="cuda")
+    run.k_out = wide[..., :128]
+    run.v_out = wide[..., 128:]
+    run.compact()
+    assert_compaction_exact(run, cfg.modality())
+    ko, vo, mo = oracle.compact(orc_params(oracle, cfg, cap=300), k.cpu(), v.cpu(), cfg.modality(), idx, n_out)
+    np.testing.assert_array_equal(bits(run.k_out), ko)
+    np.testing.assert_array_equal(bits(run.v_out), vo)
+    np.testing.assert_array_equal(run.mod_out.cpu().numpy(), mo)
+
+
+# ------------------------------------------------------------------ Algorithm 1 end to end
+
+def _run_prune(csp, oracle, cfg, layer=0, with_optional=True, **mode):
+    q, k, v = synth.make_layer(cfg, layer, "cuda")
+    p = gpu_params(csp, cfg, **mode)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget)
+    run.prune(with_optional)
+    ref = oracle.prune_layer(orc_params(oracle, cfg, **mode), q.cpu(), k.cpu(), v.cpu(), cfg.modality(),
+                             cfg.seq_lens, cfg.budgets, cfg.total_budget)
+    return run, ref
+
+
+@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1)])
+def test_prune_layer_small(csp, oracle, mode):
+    cfg = _case((900, 300, 517), 4, 2, 128, 32, 32, seed=30, visual_pct=25, text_pct=50)
+    if mode.get("select_mode"):
+        cfg.budgets = cfg.budgets[:, [0, 3]].copy()
+    run, ref = _run_prune(csp, oracle, cfg, **mode)
+    assert run.status() == 0
+    assert_scores_close(run.ss.cpu().numpy(), ref["score_self"], cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, cfg.recent)
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens,
+                            cfg.recent, global_mode=bool(mode.get("select_mode")))
+    assert_compaction_exact(run, cfg.modality())
+    if not mode:
+        np.testing.assert_array_equal(run.n_out.cpu().numpy(), ref["n_out"])
+
+
+def test_prune_layer_without_optional_outputs_and_twice_identical(csp, oracle):
+    cfg = _case((700, 450), 4, 4, 128, 32, 32, seed=31)
+    run, ref = _run_prune(csp, oracle, cfg, with_optional=False)
+    np.testing.assert_array_equal(run.n_out.cpu().numpy(), ref["n_out"])
+    first = (run.k_out.clone(), run.v_out.clone(), run.n_out.clone())
+    run.prune(with_optional=False)
+    assert torch.equal(first[0], run.k_out) and torch.equal(first[1], run.v_out) and torch.equal(first[2], run.n_out)
+    # compare with the run that exposes the index list
+    run2, _ = _run_prune(csp, oracle, cfg)
+    assert torch.equal(run2.k_out, run.k_out) and torch.equal(run2.mod_out, run.mod_out)
+
+
+def test_full_budget_is_identity_and_below_total_passthrough(csp, oracle):
+    cfg = _case((300, 200), 2, 2, 128, 32, 32, seed=32, visual_pct=100, text_pct=100)
+    run, ref = _run_prune(csp, oracle, cfg)
+    for b, L in enumerate(cfg.seq_lens):
+        assert (run.n_out[b] == int(L)).all()
+        np.testing.assert_array_equal(bits(run.k_out)[b, :, :L], bits(run.k)[b, :, :L])
+        np.testing.assert_array_equal(bits(run.v_out)[b, :, :L], bits(run.v)[b, :, :L])
+    cfg = _case((300, 200), 2, 2, 128, 32, 32, seed=33)
+    cfg.total_budget = np.array([301, 100], np.int32)
+    cap = 300
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    run = GpuRun(csp, gpu_params(csp, cfg, cap=cap), q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets,
+                 total_budget=cfg.total_budget).prune()
+    assert (run.n_out[0] == 300).all() and (run.n_out[1] < 200).all()
+    np.testing.assert_array_equal(bits(run.k_out)[0, :, :300], bits(run.k)[0, :, :300])
+
+
+def test_config0_full(csp, oracle):
+    cfg = synth.config(0)
+    run, ref = _run_prune(csp, oracle, cfg)
+    assert run.status() == 0
+    assert_scores_close(run.ss.cpu().numpy(), ref["score_self"], cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, cfg.recent)
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens, 16)
+    assert_compaction_exact(run, cfg.modality())
+    assert (run.n_out.cpu().numpy() == 520).all()
+
+
+def test_config1_one_layer_full(csp, oracle):
+    cfg = synth.config(1)
+    run, ref = _run_prune(csp, oracle, cfg, layer=3)
+    assert run.status() == 0
+    assert_scores_close(run.ss.cpu().numpy(), ref["score_self"], cfg.seq_lens, cfg.recent)
+    assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, cfg.recent)
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens, 32)
+    assert_compaction_exact(run, cfg.modality())
+    assert (run.n_out.cpu().numpy() == 1027).all()
+
+
+def _sampled_units_check(csp, oracle, cfg, units, layer=0):
+    """Full-size GPU run in the launch configuration the bench uses; the oracle recomputes sampled
+    (sequence, KV head) units one by one from the bytes the GPU read."""
+    q, k, v = synth.make_layer(cfg, layer, "cuda")
+    p = gpu_params(csp, cfg)
+    mod = cfg.modality()
+    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget).prune()
+    # budgets above the candidate count are clamped (and flagged); everything else must be clean
+    want = np.zeros(cfg.batch, np.int64)
+    clamped = False
+    for b, lay in enumerate(cfg.layouts):
+        n_text, n_vis = synth.candidate_counts(lay, cfg.recent)
+        ks, kc = int(cfg.budgets[b, 0]), int(cfg.budgets[b, 3])
+        clamped |= ks > n_text or kc > n_vis
+        want[b] = min(ks, n_text) + min(kc, n_vis) + cfg.recent
+    assert run.status() == (csp.DEV_K_CLAMPED if clamped else 0)
+    G = cfg.group
+    for b, h in units:
+        L = int(cfg.seq_lens[b])
+        op = oracle.Params(1, G, 1, cfg.head_dim, cfg.window, cfg.recent, L, p.out_capacity)
+        ref = oracle.prune_layer(op, q[b:b + 1, h * G:(h + 1) * G].cpu(), k[b:b + 1, h:h + 1, :L].cpu(),
+                                 v[b:b + 1, h:h + 1, :L].cpu(), mod[b:b + 1, :L], np.array([L], np.int32),
+                                 cfg.budgets[b:b + 1],
+                                 None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
+        assert_scores_close(run.ss[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_self"], [L], cfg.recent)
+        assert_scores_close(run.sc[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], cfg.recent)
+        assert_index_sets_match(run.idx[b:b + 1, h:h + 1].cpu().numpy(), run.n_out[b:b + 1, h:h + 1].cpu().numpy(),
+                                ref, mod[b:b + 1, :L], [L], cfg.recent)
+    assert_compaction_exact(run, mod)
+    # properties that hold at any size
+    assert (run.n_out.cpu().numpy() == want[:, None]).all()
+
+
+def test_config2_sampled_units(csp, oracle):
+    _sampled_units_check(csp, oracle, synth.config(2), [(0, 0), (0, 17), (0, 31)])
+
+
+def test_config3_sampled_units(csp, oracle):
+    _sampled_units_check(csp, oracle, synth.config(3), [(0, 1), (3, 2)])
+
+
+def test_config4_sampled_units(csp, oracle):
+    cfg = synth.config(4, budget_pct=20)
+    rng = np.random.RandomState(0)
+    units = [(int(rng.randint(32)), int(rng.randint(32))) for _ in range(4)]
+    _sampled_units_check(csp, oracle, cfg, units)
+
+
+def test_host_buffer_entry_point(csp, oracle):
+    cfg = _case((600, 340), 4, 2, 128, 32, 32, seed=40)
+    q, k, v = synth.make_layer(cfg, 0, "cpu")
+    p = gpu_params(csp, cfg)
+    cap = p.out_capacity
+    pin = lambda t: t.contiguous().pin_memory()
+    mod, lens, bud = (pin(torch.from_numpy(cfg.modality())), pin(torch.from_numpy(cfg.seq_lens)),
+                      pin(torch.from_numpy(cfg.budgets)))
+    k_out = pin(torch.zeros(2, 2, cap, 128, dtype=k.dtype))
+    v_out = pin(torch.zeros(2, 2, cap, 128, dtype=k.dtype))
+    mod_out = pin(torch.zeros(2, 2, cap, dtype=torch.uint8))
+    n_out = pin(torch.zeros(2, 2, dtype=torch.int32))
+    staging = torch.empty(csp.host_staging_bytes(p), dtype=torch.uint8, device="cuda")
+    status = csp.prune_layer_host(p, pin(q), pin(k), pin(v), mod, lens, bud, k_out, v_out, mod_out, n_out, staging)
+    assert status == 0
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).prune()
+    assert torch.equal(n_out, run.n_out.cpu())
+    for b in range(2):
+        for h in range(2):
+            n = int(n_out[b, h])
+            assert torch.equal(k_out[b, h, :n], run.k_out[b, h, :n].cpu())
+            assert torch.equal(v_out[b, h, :n], run.v_out[b, h, :n].cpu())
+            assert torch.equal(mod_out[b, h, :n], run.mod_out[b, h, :n].cpu())
+
+
+def test_bad_lengths_are_flagged_not_faulted(csp, oracle):
+    cfg = _case((300, 200), 2, 2, 128, 32, 32, seed=41)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, cfg.modality(), [5000, -3], cfg.budgets).prune()
+    assert run.status() & csp.DEV_BAD_LEN
+    assert (run.n_out.cpu().numpy() == -1).all()
+
+
+def test_reprune_round_with_per_head_labels(csp, oracle):
+    """Second invocation of Algorithm 1: the compacted cache of round one plus appended decode
+    tokens is pruned again; labels now differ per head."""
+    cfg = _case((800,), 4, 2, 128, 32, 32, seed=42, visual_pct=30, text_pct=40)
+    run, ref = _run_prune(csp, oracle, cfg)
+    n1 = int(run.n_out[0, 0])
+    assert (run.n_out == n1).all()
+    add, L2 = 64, n1 + 64
+    g = torch.Generator(device="cuda").manual_seed(5)
+    k2 = torch.cat([run.k_out[:, :, :n1], torch.randn(1, 2, add, 128, device="cuda", generator=g).to(torch.bfloat16)], 2)
+    v2 = torch.cat([run.v_out[:, :, :n1], torch.randn(1, 2, add, 128, device="cuda", generator=g).to(torch.bfloat16)], 2)
+    mod2 = torch.cat([run.mod_out[:, :, :n1], torch.zeros(1, 2, add, dtype=torch.uint8, device="cuda")], 2).contiguous()
+    q2 = torch.randn(1, 4, 32, 128, device="cuda", generator=g).to(torch.bfloat16)
+    bud = np.array([[60, 0, 0, 20]], np.int32)
+    p2 = csp.Params(1, 4, 2, 128, 32, 32, L2, 162)
+    run2 = GpuRun(csp, p2, q2, k2.contiguous(), v2.contiguous(), mod2.cpu().numpy(), [L2], bud).prune()
+    assert run2.status() == 0
+    ref2 = oracle.prune_layer(oracle.Params(1, 4, 2, 128, 32, 32, L2, 162), q2.cpu(), k2.cpu(), v2.cpu(),
+                              mod2.cpu().numpy(), np.array([L2], np.int32), bud)
+    assert_scores_close(run2.ss.cpu().numpy(), ref2["score_self"], [L2], 32)
+    assert_scores_close(run2.sc.cpu().numpy(), ref2["score_cross"], [L2], 32)
+    assert_index_sets_match(run2.idx.cpu().numpy(), run2.n_out.cpu().numpy(), ref2, mod2.cpu().numpy(), [L2], 32)
+    assert_compaction_exact(run2, mod2.cpu().numpy())
