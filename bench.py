@@ -177,7 +177,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"])
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-baseline-units", type=int, default=16)
+    ap.add_argument("--cpu-baseline-units", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
     args = ap.parse_args()
@@ -362,7 +362,7 @@ def main():
                         dtype=orc.F32 if cfg.dtype == torch.float32 else orc.BF16)
         t0 = time.perf_counter()
         reps_cpu = 0
-        while reps_cpu < 1 or (time.perf_counter() - t0 < 10.0 and reps_cpu < 50):
+        while reps_cpu < 1 or (time.perf_counter() - t0 < 12.0 and reps_cpu < 5000):
             orc.prune_layer(op, qs, ks, vs, cfg.modality()[b:b + 1, :L], np.array([L], np.int32),
                             cfg.budgets[b:b + 1], None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
             reps_cpu += 1

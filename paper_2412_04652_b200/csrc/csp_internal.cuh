@@ -68,8 +68,16 @@ struct CompactArgs {
     int32_t n_kv_heads, max_len, out_capacity, chunks_per_row;
 };
 
+// cluster size: the largest power of two (<= 8) that still fits every cluster on the 148 SMs at once
+inline int pick_cluster(int units, int max_tiles) {
+    int c = 1;
+    while (c < 8 && units * (c * 2) <= 148 && c * 2 <= max_tiles) c *= 2;
+    return c;
+}
+
 // ---- host-side launchers (defined next to their kernels) ----------------------------------
 csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s);
+csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s);
 csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,
                             float* score_self, float* score_cross, const int32_t* seq_lens,
                             cudaStream_t s);

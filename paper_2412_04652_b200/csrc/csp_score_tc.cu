@@ -1,0 +1,505 @@
+// Scoring kernel for bf16 caches on the 5th-generation tensor cores (tcgen05 + tensor memory):
+// window logits (Eq. 5), n-softmax rows (Eq. 7), recent trim, head-group mean and the intra/inter
+// query-axis sums (Eq. 1), for one layer.
+//
+// One thread-block cluster of C CTAs owns one (sequence, KV head) unit; 128-key tiles of K are
+// dealt round-robin to its CTAs.  Inside a CTA
+//   warp 8      TMA producer: K tiles -> ring of 128B-swizzled shared-memory stages
+//   warp 9      one thread issues tcgen05.mma: D[128 keys x 32G queries] = K_tile . Q^T, fp32
+//               accumulators in tensor memory, several tiles in flight (ring of TMEM buffers)
+//   warps 0-7   epilogue, two groups of four warps taking alternate tiles, reading TMEM
+// The same tile stream runs twice:
+//   pass 1  all tiles of the unit: per window row a running (max, sum of 2^(x-max)); merged over
+//           lanes, warps and - through distributed shared memory - the CTAs of the cluster
+//   pass 2  candidate tiles again (L2 hits): one thread per key reads its row of logits,
+//           weight = 2^(x*scale + c_w) with c_w = log2(1 / (G (n 2^-m + Z))) - m, added to the key's
+//           intra or inter sum by label equality; no cross-thread reduction is left, and the two
+//           score vectors are written fully coalesced.
+// Summation orders are fixed: results are bit-reproducible run to run.
+#include "csp_device.cuh"
+#include "csp_internal.cuh"
+
+namespace csp {
+namespace {
+using namespace dev;
+
+constexpr int kTcThreads = 320;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kMaxStages = 8;
+constexpr int kMaxTmemBufs = 4;
+
+// ---- tcgen05 wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// one row (TMEM lane) per thread, 32 consecutive fp32 columns
+__device__ __forceinline__ void tc_ld_row32(uint32_t (&v)[32], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+// 16 rows x 32 columns spread over the warp like an mma accumulator: thread (lane) holds, for each
+// 8-column block i, regs 4i..4i+3 = (row lane/4, cols 2(lane%4)+{0,1}), (row lane/4+8, same cols)
+__device__ __forceinline__ void tc_ld_16x32(uint32_t (&v)[16], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t sw128_desc(uint32_t smem_addr) {
+    uint64_t d = uint64_t((smem_addr & 0x3FFFFu) >> 4);
+    d |= uint64_t(1) << 16;                // leading byte offset (unused for swizzled K-major)
+    d |= uint64_t(1024 >> 4) << 32;        // stride byte offset
+    d |= uint64_t(1) << 46;                // descriptor version
+    d |= uint64_t(2) << 61;                // SWIZZLE_128B
+    return d;
+}
+__device__ __forceinline__ float lg2f(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int G> struct TmemPlan {
+    static constexpr int kCols = 32 * G;                                   // accumulator columns per tile
+    static constexpr int kBufs = (512 / kCols) >= kMaxTmemBufs ? kMaxTmemBufs : (512 / kCols);
+    static constexpr int kNeeded = kCols * kBufs;
+    static constexpr int kAlloc = kNeeded <= 32 ? 32 : kNeeded <= 64 ? 64 : kNeeded <= 128 ? 128
+                                  : kNeeded <= 256 ? 256 : 512;
+};
+
+struct TcSmemPlan {   // byte offsets from the 1024-aligned base
+    uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
+};
+__host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
+    TcSmemPlan s;
+    uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
+    s.q = off;        off += uint32_t(nh) * uint32_t(g) * 32u * 128u;
+    s.wstats = off;   off += 8u * uint32_t(g) * 32u * 8u;
+    s.cstats = off;   off += uint32_t(g) * 32u * 8u;
+    s.cvec = off;     off += uint32_t(g) * 32u * 4u;
+    s.dq_mask = off;  off += 32u * 4u;
+    s.dq_val = off;   off += 32u * 4u;
+    s.bars = off;     off += (2u * kMaxStages + 2u * kMaxTmemBufs + 1u) * 8u;
+    s.misc = off;     off += 16u;                       // tmem base, abort flag, n distinct query labels
+    s.total = off;
+    return s;
+}
+
+template <int NH, int G>
+__global__ void __launch_bounds__(kTcThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages) {
+    constexpr int KS = NH * 4;                          // MMAs (K = 16 elements = 32 bytes) per tile
+    constexpr int NC = TmemPlan<G>::kCols;
+    constexpr int NB = TmemPlan<G>::kBufs;
+    constexpr uint32_t kStageBytes = NH * kBlockBytes;
+    // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, M = 128, N = NC
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NC >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const TcSmemPlan sp = tc_smem_plan(NH, G, n_stages);
+    const uint32_t q_s = base + sp.q;
+    float2* const wstats = reinterpret_cast<float2*>(base_ptr + sp.wstats);
+    float2* const cstats = reinterpret_cast<float2*>(base_ptr + sp.cstats);
+    float* const cvec = reinterpret_cast<float*>(base_ptr + sp.cvec);
+    uint32_t* const dq_mask = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_mask);
+    uint32_t* const dq_val = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_val);
+    const uint32_t full_k = base + sp.bars;
+    const uint32_t empty_k = full_k + 8 * kMaxStages;
+    const uint32_t tmem_full = empty_k + 8 * kMaxStages;
+    const uint32_t tmem_empty = tmem_full + 8 * kMaxTmemBufs;
+    const uint32_t q_ready = tmem_empty + 8 * kMaxTmemBufs;
+    volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + sp.misc);
+    volatile int* const abort_flag = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 4);
+    volatile int* const n_dq = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 8);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const uint32_t rank = cluster_rank(), csize = cluster_size();
+
+    int L = a.seq_lens[b];
+    const bool bad_len = L < 0 || L > a.max_len;
+    const bool skip = bad_len || L < a.window || L < a.recent;
+    if (bad_len && tid == 0 && rank == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
+    if (skip) L = 0;
+    const int W = a.window;
+    const int N = skip ? 0 : L - a.recent;
+    const int tiles_all = a.lse ? 0 : (L + kTileKeys - 1) / kTileKeys;
+    const int tiles_cand = (N + kTileKeys - 1) / kTileKeys;
+    const int my_all = tiles_all > int(rank) ? (tiles_all - int(rank) + int(csize) - 1) / int(csize) : 0;
+    const int my_cand = tiles_cand > int(rank) ? (tiles_cand - int(rank) + int(csize) - 1) / int(csize) : 0;
+    const int total = my_all + my_cand;
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
+        for (int i = 0; i < NB; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
+        mbar_init(q_ready, 8);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TmemPlan<G>::kAlloc);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == kProducerWarp) {
+        // =============================== TMA producer ===============================
+        cluster_arrive();                         // cluster barrier 1: nothing of ours to publish
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            for (int it = 0; it < total; ++it) {
+                const int slot = it % n_stages;
+                const uint32_t round = uint32_t(it / n_stages);
+                const int tile = (it < my_all ? it : it - my_all) * int(csize) + int(rank);
+                mbar_wait(empty_k + 8 * slot, (round & 1u) ^ 1u, abort_flag);
+                if (*abort_flag) break;
+                mbar_expect_tx(full_k + 8 * slot, kStageBytes);
+#pragma unroll
+                for (int hb = 0; hb < NH; ++hb)
+                    tma_load_4d(base + slot * kStageBytes + hb * kBlockBytes, &tmap, full_k + 8 * slot,
+                                hb * 64, tile * kTileKeys, h, b);
+            }
+            if (*abort_flag) {
+                // let copies that were issued land before the CTA's shared memory is given up
+                const int issued = total < n_stages ? total : n_stages;
+                for (int s = 0; s < issued; ++s) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_k + 8 * s, 0) && !mbar_try_wait(full_k + 8 * s, 1) &&
+                           global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+        __syncwarp();
+        cluster_wait();
+    } else if (warp == kMmaWarp) {
+        // =============================== MMA issuer ===============================
+        cluster_arrive();
+        if (lane == 0) {
+            mbar_wait(q_ready, 0, abort_flag);
+            for (int it = 0; it < total; ++it) {
+                const int slot = it % n_stages, buf = it % NB;
+                mbar_wait(full_k + 8 * slot, uint32_t(it / n_stages) & 1u, abort_flag);
+                mbar_wait(tmem_empty + 8 * buf, (uint32_t(it / NB) & 1u) ^ 1u, abort_flag);
+                if (*abort_flag) break;
+                tc_fence_after();
+                const uint32_t stage_addr = base + slot * kStageBytes;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const uint64_t ad = sw128_desc(stage_addr + uint32_t(ks >> 2) * kBlockBytes + uint32_t(ks & 3) * 32u);
+                    const uint64_t bd = sw128_desc(q_s + uint32_t(ks >> 2) * (NC * 128u) + uint32_t(ks & 3) * 32u);
+                    tc_mma_bf16(tmem_base + uint32_t(buf * NC), ad, bd, kIdesc, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(empty_k + 8 * slot);    // stage may be refilled once these MMAs have read it
+                tc_commit(tmem_full + 8 * buf);   // accumulator ready for the epilogue
+            }
+        }
+        __syncwarp();
+        cluster_wait();
+    } else {
+        // =============================== epilogue warps ===============================
+        const int quarter = warp & 3, group = warp >> 2;
+        const int lq = lane & 3, lr = lane >> 2;
+        const uint8_t* modp = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
+
+        // stage Q of this KV group: row (g*32 + w), 128-byte column blocks, 16-byte chunks XOR-swizzled
+        if (!skip) {
+            const uint8_t* qb = static_cast<const uint8_t*>(a.q);
+            constexpr int kChunksPerRow = NH * 8;
+            for (int i = tid; i < G * 32 * kChunksPerRow; i += kConsumerThreads) {
+                const int r = i / kChunksPerRow, c = i % kChunksPerRow;
+                const int g = r >> 5, w = r & 31;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (w < W) {
+                    const int64_t e = int64_t(b) * a.q_sb + int64_t(h * G + g) * a.q_sh + int64_t(w) * a.q_st;
+                    v = *reinterpret_cast<const uint4*>(qb + e * 2 + c * 16);
+                }
+                const uint32_t off = uint32_t(c >> 3) * (NC * 128) + uint32_t(r) * 128 + (uint32_t((c & 7) ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4*>(base_ptr + sp.q + off) = v;
+            }
+        } else {
+            for (int i = tid; i < NH * NC * 8; i += kConsumerThreads)
+                *reinterpret_cast<uint4*>(base_ptr + sp.q + i * 16) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make Q visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(q_ready);
+
+        // table of the distinct labels of the window queries and the columns carrying each
+        if (warp == 0) {
+            const uint32_t ql = (lane < W && !skip) ? modp[L - W + lane] : 0xFFFFFFFFu;
+            int count = 0;
+            for (int j = 0; j < W; ++j) {
+                const uint32_t vj = __shfl_sync(0xffffffffu, ql, j);
+                const uint32_t same = __ballot_sync(0xffffffffu, ql == vj);
+                const bool first = (same & ((1u << j) - 1u)) == 0u;       // no earlier column has this label
+                if (first) {
+                    if (lane == 0) { dq_val[count] = vj; dq_mask[count] = same; }
+                    ++count;
+                }
+            }
+            if (lane == 0) *n_dq = skip ? 0 : count;
+        }
+
+        const float scale2 = a.scale_log2;
+        const int first_masked_key = L - W;       // keys beyond this may be hidden from some window row
+
+        // ---------------------------------- pass 1 ----------------------------------
+        float m_run[G][8], z_run[G][8];
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) { m_run[g][jj] = kNeg; z_run[g][jj] = 0.f; }
+
+        for (int it = group; it < my_all; it += 2) {
+            const int buf = it % NB;
+            const int tile = it * int(csize) + int(rank);
+            mbar_wait(tmem_full + 8 * buf, uint32_t(it / NB) & 1u, abort_flag);
+            tc_fence_after();
+            const bool masked = (tile + 1) * kTileKeys > first_masked_key;
+            const int t_base = tile * kTileKeys + quarter * 32 + lr;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                uint32_t v0[16], v1[16];
+                const uint32_t col = uint32_t(buf * NC + g * 32);
+                tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
+                tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
+                tc_wait_ld();
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int jj = nt * 2 + e;
+                        float x[4] = {__uint_as_float(v0[nt * 4 + e]) * scale2, __uint_as_float(v0[nt * 4 + 2 + e]) * scale2,
+                                      __uint_as_float(v1[nt * 4 + e]) * scale2, __uint_as_float(v1[nt * 4 + 2 + e]) * scale2};
+                        if (!masked) {
+                            const float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+                            if (mx > m_run[g][jj] + kLazy) { z_run[g][jj] *= ex2f(m_run[g][jj] - mx); m_run[g][jj] = mx; }
+                            const float mm = m_run[g][jj];
+                            z_run[g][jj] += (ex2f(x[0] - mm) + ex2f(x[1] - mm)) + (ex2f(x[2] - mm) + ex2f(x[3] - mm));
+                        } else {
+                            const int colw = nt * 8 + lq * 2 + e;
+                            bool vis[4];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                const int t = t_base + (r & 1) * 8 + (r >> 1) * 16;
+                                vis[r] = colw < W && t <= first_masked_key + colw;   // key <= query position
+                                x[r] = vis[r] ? x[r] : kNeg;
+                            }
+                            const float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+                            if (mx > m_run[g][jj] + kLazy) { z_run[g][jj] *= ex2f(m_run[g][jj] - mx); m_run[g][jj] = mx; }
+                            const float mm = m_run[g][jj];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) z_run[g][jj] += vis[r] ? ex2f(x[r] - mm) : 0.f;
+                        }
+                    }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+        }
+
+        // merge the running statistics: lanes holding the same columns, then warps, then CTAs
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+#pragma unroll
+                for (int d = 4; d <= 16; d <<= 1) {
+                    const float om = __shfl_xor_sync(0xffffffffu, m_run[g][jj], d);
+                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[g][jj], d);
+                    merge_stats(m_run[g][jj], z_run[g][jj], om, oz);
+                }
+                if (lr == 0) wstats[(warp * G + g) * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[g][jj], z_run[g][jj]);
+            }
+        consumer_sync();
+        if (tid < G * 32) {
+            float m = kNeg, z = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                const float2 s = wstats[w * (G * 32) + tid];
+                merge_stats(m, z, s.x, s.y);
+            }
+            cstats[tid] = make_float2(m, z);
+        }
+        cluster_arrive();
+        cluster_wait();
+        if (tid < G * 32) {
+            const int g = tid >> 5, col = tid & 31;
+            float m, z;
+            if (a.lse) {
+                // caller-supplied natural-log row sums: use them as (max, sum) = (lse, 1)
+                m = (col < W && !skip)
+                        ? a.lse[(int64_t(b) * (a.n_kv_heads * G) + h * G + g) * W + col] * 1.4426950408889634f
+                        : 0.f;
+                z = 1.f;
+            } else {
+                m = kNeg; z = 0.f;
+                for (uint32_t r = 0; r < csize; ++r) {
+                    const float2 s = ld_remote_f2(smem_u32(&cstats[tid]), r);
+                    merge_stats(m, z, s.x, s.y);
+                }
+            }
+            // weight of 2^(x - m) is 1 / (G (n 2^-m + Z)); fold it and -m into one additive constant
+            const float denom = a.n * ex2f(-m) + z;
+            cvec[tid] = col < W ? lg2f(a.weight / denom) - m : -INFINITY;
+        }
+        consumer_sync();
+
+        // ---------------------------------- pass 2 ----------------------------------
+        float* const out_s = a.score_self + (int64_t(b) * a.n_kv_heads + h) * a.max_len;
+        float* const out_c = a.score_cross + (int64_t(b) * a.n_kv_heads + h) * a.max_len;
+        const int ndq = *n_dq;
+        const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
+
+        for (int it = my_all + ((my_all ^ group) & 1); it < total; it += 2) {
+            const int buf = it % NB;
+            const int tile = (it - my_all) * int(csize) + int(rank);
+            const int t = tile * kTileKeys + quarter * 32 + lane;          // this thread's key
+            const uint32_t kmod = t < N ? modp[t] : 0u;
+            mbar_wait(tmem_full + 8 * buf, uint32_t(it / NB) & 1u, abort_flag);
+            tc_fence_after();
+            uint32_t same = 0u;                                            // window columns with the key's label
+            for (int i = 0; i < ndq; ++i) same = dq_val[i] == kmod ? dq_mask[i] : same;
+            const int delta = t - first_masked_key;                        // column w sees the key iff w >= delta
+            const uint32_t vis = delta <= 0 ? wmask : (delta >= 32 ? 0u : (wmask & (0xFFFFFFFFu << delta)));
+            const uint32_t add_s = same & vis, add_c = ~same & vis;
+            float s = 0.f, c = 0.f;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                uint32_t v[32];
+                tc_ld_row32(v, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + g * 32));
+                tc_wait_ld();
+                const float4* cv = reinterpret_cast<const float4*>(cvec + g * 32);
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4) {
+                    const float4 cc = cv[j4];
+                    const float p0 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 0]), scale2, cc.x));
+                    const float p1 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 1]), scale2, cc.y));
+                    const float p2 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 2]), scale2, cc.z));
+                    const float p3 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 3]), scale2, cc.w));
+                    s += (add_s >> (j4 * 4 + 0)) & 1u ? p0 : 0.f; c += (add_c >> (j4 * 4 + 0)) & 1u ? p0 : 0.f;
+                    s += (add_s >> (j4 * 4 + 1)) & 1u ? p1 : 0.f; c += (add_c >> (j4 * 4 + 1)) & 1u ? p1 : 0.f;
+                    s += (add_s >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c += (add_c >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
+                    s += (add_s >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c += (add_c >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+            if (t < N) { out_s[t] = s; out_c[t] = c; }
+        }
+        if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
+    }
+
+    // every warp: give tensor memory back, then keep shared memory alive until the peers are done
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TmemPlan<G>::kAlloc);
+    }
+    cluster_arrive();                             // cluster barrier 2
+    cluster_wait();
+}
+
+template <int NH, int G>
+csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
+    const int fixed = int(tc_smem_plan(NH, G, 0).total) + 1024;
+    int stages = (227 * 1024 - fixed) / (NH * kBlockBytes);
+    if (stages > 6) stages = 6;
+    if (stages < 2) return CSP_ERR_UNSUPPORTED;
+    const size_t smem = tc_smem_plan(NH, G, stages).total + 1024;
+    auto kern = score_tc_kernel<NH, G>;
+    static bool configured[64] = {};   // per instantiation and device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            return CSP_ERR_CUDA;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
+    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages) != cudaSuccess) { cudaGetLastError(); return CSP_ERR_CUDA; }
+    return CSP_OK;
+}
+
+template <int NH>
+csp_status launch_g(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
+    switch (a.group) {
+        case 1: return launch_inst<NH, 1>(p, a, tmap, s);
+        case 2: return launch_inst<NH, 2>(p, a, tmap, s);
+        case 3: return launch_inst<NH, 3>(p, a, tmap, s);
+        case 4: return launch_inst<NH, 4>(p, a, tmap, s);
+        case 5: return launch_inst<NH, 5>(p, a, tmap, s);
+        case 6: return launch_inst<NH, 6>(p, a, tmap, s);
+        case 7: return launch_inst<NH, 7>(p, a, tmap, s);
+        case 8: return launch_inst<NH, 8>(p, a, tmap, s);
+        default: return CSP_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace
+
+csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
+    switch (p.head_dim * 2) {
+        case 128: return launch_g<1>(p, a, tmap, s);
+        case 256: return launch_g<2>(p, a, tmap, s);
+        case 512: return launch_g<4>(p, a, tmap, s);
+        default: return CSP_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace csp

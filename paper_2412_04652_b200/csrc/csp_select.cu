@@ -3,9 +3,9 @@
 //
 // One CTA per (sequence, KV head) unit.  Up to four top-K problems run together (intra/inter score x
 // text/visual keys, or intra/inter over all keys): an MSB-first radix select on the order-preserving
-// integer image of the fp32 scores finds each problem's K-th value, ties at that value are taken in
-// position order with a block-wide prefix count, and a second prefix count over the combined mask
-// places the kept positions in ascending order.  The result equals the first K entries of a stable
+// integer image of the fp32 scores (staged once in shared memory) finds each problem's K-th value,
+// ties at that value are taken in position order with a block-wide prefix count, and a second
+// prefix count over the combined mask places the kept positions in ascending order.  The result equals the first K entries of a stable
 // descending sort, exactly.
 #include "csp_internal.cuh"
 
@@ -14,6 +14,13 @@ namespace {
 
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kPasses = 3;                              // radix digits of 11, 11 and 10 bits
+constexpr int kBins = 2048;
+constexpr int kHistRow = kBins + kBins / 32;           // one pad word per 32 bins: conflict-free lane-strided scans
+__device__ __forceinline__ int hpad(int bin) { return bin + (bin >> 5); }
+constexpr int kBytesPerCached = 9;                      // two 32-bit keys and the label of one position
+__device__ __constant__ int kDigitShift[kPasses] = {21, 10, 0};
+__device__ __constant__ int kDigitBits[kPasses] = {11, 11, 10};
 
 __device__ __forceinline__ uint32_t order_key(float f) {
     uint32_t b = __float_as_uint(f);
@@ -48,8 +55,13 @@ __device__ __forceinline__ V block_exclusive_scan(V v, V* warp_tot, V* total_out
     return warp_tot[warp] + inc - v;
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs a) {
-    __shared__ uint32_t hist[4][256];
+__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs a, const int n_cached_max) {
+    // dynamic: hist[4][kBins], then the cached keys of the first n_cached positions
+    extern __shared__ __align__(16) uint8_t sel_smem[];
+    uint32_t (*hist)[kHistRow] = reinterpret_cast<uint32_t (*)[kHistRow]>(sel_smem);
+    uint32_t* const cache_s = reinterpret_cast<uint32_t*>(sel_smem + 4 * kHistRow * 4);
+    uint32_t* const cache_c = cache_s + n_cached_max;
+    uint8_t* const cache_m = reinterpret_cast<uint8_t*>(cache_c + n_cached_max);
     __shared__ uint32_t prefix[4];
     __shared__ int32_t krem[4];
     __shared__ int32_t act[4];
@@ -85,6 +97,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
     const int nprob = a.global_mode ? 2 : 4;
     const int32_t* const bud = a.budgets + int64_t(b) * nprob;
 
+    // stage the order-preserving keys and labels on chip once; every later pass reads them from there
+    const int n_cached = min(N, n_cached_max);
+    for (int t = tid; t < n_cached; t += kSelThreads) {
+        cache_s[t] = order_key(ss[t]);
+        cache_c[t] = order_key(sc[t]);
+        cache_m[t] = mod[t];
+    }
+    auto key_s = [&](int t) { return t < n_cached ? cache_s[t] : order_key(ss[t]); };
+    auto key_c = [&](int t) { return t < n_cached ? cache_c[t] : order_key(sc[t]); };
+    auto label = [&](int t) { return t < n_cached ? cache_m[t] : mod[t]; };
+
     if (tid < 4) {
         prefix[tid] = 0;
         const int32_t k = tid < nprob ? bud[tid] : 0;
@@ -93,25 +116,25 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
         if (k < 0) atomicOr(a.status, CSP_DEV_K_CLAMPED);
     }
 
-    // ---- radix select, 8 bits per pass, most significant first
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        for (int i = tid; i < 4 * 256; i += kSelThreads) (&hist[0][0])[i] = 0;
+    // ---- radix select, most significant digit first
+    for (int pass = 0; pass < kPasses; ++pass) {
+        const int shift = kDigitShift[pass], nbins = 1 << kDigitBits[pass];
+        for (int i = tid; i < 4 * kHistRow; i += kSelThreads) (&hist[0][0])[i] = 0;
         __syncthreads();
         for (int t = tid; t < N; t += kSelThreads) {
-            const int vis = a.global_mode ? 0 : (mod[t] != 0);
+            const int vis = a.global_mode ? 0 : (label(t) != 0);
             const int ps = vis, pc = a.global_mode ? 1 : 2 + vis;
-            const uint32_t ks = order_key(ss[t]), kc = order_key(sc[t]);
-            if (act[ps] && (pass == 0 || (ks >> (shift + 8)) == prefix[ps]))
-                atomicAdd(&hist[ps][(ks >> shift) & 255u], 1u);
-            if (act[pc] && (pass == 0 || (kc >> (shift + 8)) == prefix[pc]))
-                atomicAdd(&hist[pc][(kc >> shift) & 255u], 1u);
+            const uint32_t ks = key_s(t), kc = key_c(t);
+            const uint32_t hi_s = pass == 0 ? 0u : ks >> (shift + kDigitBits[pass]);
+            const uint32_t hi_c = pass == 0 ? 0u : kc >> (shift + kDigitBits[pass]);
+            if (act[ps] && hi_s == prefix[ps]) atomicAdd(&hist[ps][hpad((ks >> shift) & (nbins - 1))], 1u);
+            if (act[pc] && hi_c == prefix[pc]) atomicAdd(&hist[pc][hpad((kc >> shift) & (nbins - 1))], 1u);
         }
         __syncthreads();
         if (warp < nprob && act[warp]) {
-            uint32_t bins[8], ls = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { bins[i] = hist[warp][lane * 8 + i]; ls += bins[i]; }
+            const int per_lane = nbins / 32;            // 64 or 32 bins per lane
+            uint32_t ls = 0;
+            for (int i = 0; i < per_lane; ++i) ls += hist[warp][hpad(lane * per_lane + i)];
             uint32_t suf = ls;                          // inclusive suffix sum over lanes
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -133,14 +156,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
                 const uint32_t above = suf - ls;
                 if (above < uint32_t(k) && uint32_t(k) <= suf) {
                     uint32_t cum = above;
-#pragma unroll
-                    for (int i = 7; i >= 0; --i) {
-                        if (cum + bins[i] >= uint32_t(k)) {
-                            prefix[warp] = (prefix[warp] << 8) | uint32_t(lane * 8 + i);
+                    for (int i = per_lane - 1; i >= 0; --i) {
+                        const uint32_t c = hist[warp][hpad(lane * per_lane + i)];
+                        if (cum + c >= uint32_t(k)) {
+                            prefix[warp] = (prefix[warp] << kDigitBits[pass]) | uint32_t(lane * per_lane + i);
                             krem[warp] = k - int32_t(cum);
                             break;
                         }
-                        cum += bins[i];
+                        cum += c;
                     }
                 }
             }
@@ -155,10 +178,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
     // ---- ties: rank of each threshold-valued key among its equals, in position order
     unsigned long long eq_self = 0, eq_cross = 0;       // two 32-bit counters each: [text | visual]
     for (int t = t_beg; t < t_end; ++t) {
-        const int vis = a.global_mode ? 0 : (mod[t] != 0);
+        const int vis = a.global_mode ? 0 : (label(t) != 0);
         const int ps = vis, pc = a.global_mode ? 1 : 2 + vis;
-        if (act[ps] && order_key(ss[t]) == prefix[ps]) eq_self += 1ull << (32 * vis);
-        if (act[pc] && order_key(sc[t]) == prefix[pc]) eq_cross += 1ull << (32 * vis);
+        if (act[ps] && key_s(t) == prefix[ps]) eq_self += 1ull << (32 * vis);
+        if (act[pc] && key_c(t) == prefix[pc]) eq_cross += 1ull << (32 * vis);
     }
     const unsigned long long ex_self = block_exclusive_scan(eq_self, scan_ws, &scan_total[0]);
     const unsigned long long ex_cross = block_exclusive_scan(eq_cross, scan_ws, &scan_total[1]);
@@ -167,9 +190,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
         uint32_t rank_s[2] = {uint32_t(ex_self), uint32_t(ex_self >> 32)};
         uint32_t rank_c[2] = {uint32_t(ex_cross), uint32_t(ex_cross >> 32)};
         for (int t = t_beg; t < t_end; ++t) {
-            const int vis = a.global_mode ? 0 : (mod[t] != 0);
+            const int vis = a.global_mode ? 0 : (label(t) != 0);
             const int ps = vis, pc = a.global_mode ? 1 : 2 + vis;
-            const uint32_t ks = order_key(ss[t]), kc = order_key(sc[t]);
+            const uint32_t ks = key_s(t), kc = key_c(t);
             bool sel_s = false, sel_c = false;
             if (act[ps]) {
                 if (ks > prefix[ps]) sel_s = true;
@@ -201,7 +224,23 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
 csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t s) {
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
-    select_kernel<<<units, kSelThreads, 0, s>>>(a);
+    // cache as many positions on chip as one CTA's shared memory allows (the rest is read from L2)
+    const size_t fixed = 4 * kHistRow * 4;
+    size_t n_cached = size_t(p.max_len);
+    const size_t limit = (200 * 1024 - fixed) / kBytesPerCached;
+    if (n_cached > limit) n_cached = limit;
+    n_cached = (n_cached + 3) & ~size_t(3);
+    const size_t smem = fixed + n_cached * kBytesPerCached;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
+            cudaSuccess)
+            return CSP_ERR_CUDA;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    select_kernel<<<units, kSelThreads, smem, s>>>(a, int(n_cached));
     return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
 }
 
