@@ -108,9 +108,16 @@ def algorithmic_bytes(cfg, n_out_total: int):
 
 
 class LayerBuffers:
-    def __init__(self, csp, cfg, p, layer, device):
-        self.q, self.k, self.v = synth.make_layer(cfg, layer, device)
-        B, H, cap, d = cfg.batch, cfg.n_kv_heads, p.out_capacity, cfg.head_dim
+    """Inputs and outputs of one library call: one layer, or `n_fold` layers stacked on the batch axis."""
+
+    def __init__(self, csp, cfg, p, layer, device, n_fold=1):
+        if n_fold == 1:
+            self.q, self.k, self.v = synth.make_layer(cfg, layer, device)
+        else:
+            parts = [synth.make_layer(cfg, layer + i, device) for i in range(n_fold)]
+            self.q, self.k, self.v = (torch.cat([x[j] for x in parts], 0) for j in range(3))
+            del parts
+        B, H, cap, d = cfg.batch * n_fold, cfg.n_kv_heads, p.out_capacity, cfg.head_dim
         self.k_out = torch.empty((B, H, cap, d), dtype=cfg.dtype, device=device)
         self.v_out = torch.empty((B, H, cap, d), dtype=cfg.dtype, device=device)
         self.mod_out = torch.empty((B, H, cap), dtype=torch.uint8, device=device)
@@ -176,6 +183,9 @@ def main():
     ap.add_argument("--ref-units", type=int, default=8, help="KV heads per reference-arm step")
     ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"])
+    ap.add_argument("--streams", type=int, default=8, help="concurrent layer chains inside the step graph")
+    ap.add_argument("--fold-layers", action="store_true",
+                    help="one call for all layers: the layer axis of a [layers*B, H, L, d] cache is passed as batch")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-baseline-units", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -213,17 +223,50 @@ def main():
     lens = torch.from_numpy(cfg.seq_lens).to(dev)
     bud = torch.from_numpy(cfg.budgets).to(dev)
     tot = None if cfg.total_budget is None else torch.from_numpy(cfg.total_budget).to(dev)
-    ws = csp.new_workspace(p, dev)
-    layers = [LayerBuffers(csp, cfg, p, i, dev) for i in range(n_buf)]
     sum_l = int(cfg.seq_lens.sum())
 
-    def prune(lb):
-        csp.prune_layer(p, lb.q, lb.k, lb.v, mod, lens, bud, lb.k_out, lb.v_out, lb.mod_out, lb.n_out, ws,
-                        total_budget=tot)
+    # One entry per library call of a step: (params, buffers, labels, lengths, budgets, totals, layers covered)
+    if args.fold_layers:
+        import copy
+        pf = copy.copy(p)
+        pf.batch = cfg.batch * n_layers
+        calls = [(pf, LayerBuffers(csp, cfg, pf, 0, dev, n_fold=n_layers), mod.repeat(n_layers, 1),
+                  lens.repeat(n_layers), bud.repeat(n_layers, 1), None if tot is None else tot.repeat(n_layers),
+                  n_layers)]
+        n_buf, n_chains = n_layers, 1
+    else:
+        layers = [LayerBuffers(csp, cfg, p, i, dev) for i in range(n_buf)]
+        calls = [(p, layers[i % n_buf], mod, lens, bud, tot, 1) for i in range(n_layers)]
+        n_chains = max(1, min(args.streams, n_layers)) if args.launch == "graph" else 1
+    wss = [csp.new_workspace(calls[0][0], dev) for _ in range(n_chains)]   # one scratch area per concurrent chain
+    first_lb = calls[0][1]
+
+    def prune(call, w):
+        cp, lb, cmod, clens, cbud, ctot, _ = call
+        csp.prune_layer(cp, lb.q, lb.k, lb.v, cmod, clens, cbud, lb.k_out, lb.v_out, lb.mod_out, lb.n_out, w,
+                        total_budget=ctot)
 
     def step():
-        for i in range(n_layers):
-            prune(layers[i % n_buf])
+        for call in calls:
+            prune(call, wss[0])
+
+    side = [torch.cuda.Stream(dev) for _ in range(n_chains - 1)]
+
+    def step_chains(main_stream):
+        # layers are independent: chain c prunes calls c, c + n_chains, ... on its own stream
+        fork = torch.cuda.Event()
+        fork.record(main_stream)
+        for c in range(n_chains):
+            st = main_stream if c == 0 else side[c - 1]
+            if c:
+                st.wait_event(fork)
+            with torch.cuda.stream(st):
+                for i in range(c, len(calls), n_chains):
+                    prune(calls[i], wss[c])
+            if c:
+                join = torch.cuda.Event()
+                join.record(st)
+                main_stream.wait_event(join)
 
     stream = torch.cuda.Stream(dev)
     torch.cuda.synchronize()
@@ -235,14 +278,16 @@ def main():
         if args.launch == "graph":
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
-                step()
+                step_chains(stream)
             for _ in range(3):
                 graph.replay()
             stream.synchronize()
         run_step = graph.replay if graph is not None else step
 
-        status = csp.device_status(ws)
-        n_out_total = int(layers[0].n_out.clamp(min=0).sum().item())
+        status = 0
+        for w in wss:
+            status |= csp.device_status(w)
+        n_out_total = int(first_lb.n_out.clamp(min=0).sum().item()) // calls[0][6]      # kept rows per layer
 
         # ---- timed region: K steps, device resident ----
         if dist is not None:
@@ -268,44 +313,59 @@ def main():
         ms_step = ms_total / args.steps
         value = world * sum_l * n_layers / (ms_step * 1e-3)
 
-        # ---- per-kernel durations, live, with events on the launching stream ----
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_layers)]
-        reps = 3
-        per = {"score": 0.0, "select": 0.0, "compact": 0.0}
-        for _ in range(reps):
-            for i in range(n_layers):
-                lb = layers[i % n_buf]
-                evs[i][0].record(stream)
-                csp.score(p, lb.q, lb.k, mod, lens, lb.ss, lb.sc, ws)
-                evs[i][1].record(stream)
-                csp.select(p, lb.ss, lb.sc, mod, lens, bud, lb.idx, lb.n_out, ws, total_budget=tot)
-                evs[i][2].record(stream)
-                csp.compact(p, lb.k, lb.v, mod, lb.idx, lb.n_out, lb.k_out, lb.v_out, lb.mod_out)
-                evs[i][3].record(stream)
+        # ---- per-kernel durations, live: one CUDA graph per kernel holding that kernel's launch for
+        # every call of a step, replayed back to back and timed with events on the launching stream ----
+        ws = wss[0]
+
+        def score_all():
+            for cp, lb, cmod, clens, cbud, ctot, _ in calls:
+                csp.score(cp, lb.q, lb.k, cmod, clens, lb.ss, lb.sc, ws)
+
+        def select_all():
+            for cp, lb, cmod, clens, cbud, ctot, _ in calls:
+                csp.select(cp, lb.ss, lb.sc, cmod, clens, cbud, lb.idx, lb.n_out, ws, total_budget=ctot)
+
+        def compact_all():
+            for cp, lb, cmod, clens, cbud, ctot, _ in calls:
+                csp.compact(cp, lb.k, lb.v, cmod, lb.idx, lb.n_out, lb.k_out, lb.v_out, lb.mod_out)
+
+        per = {}
+        reps = max(3, min(50, args.steps))
+        for name, fn in (("score", score_all), ("select", select_all), ("compact", compact_all)):
+            fn()
             stream.synchronize()
-            for i in range(n_layers):
-                per["score"] += evs[i][0].elapsed_time(evs[i][1])
-                per["select"] += evs[i][1].elapsed_time(evs[i][2])
-                per["compact"] += evs[i][2].elapsed_time(evs[i][3])
-        per = {k_: v_ / (reps * n_layers) for k_, v_ in per.items()}   # ms per launch
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+            g.replay()
+            stream.synchronize()
+            k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            k0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            k1.record(stream)
+            stream.synchronize()
+            per[name] = k0.elapsed_time(k1) / (reps * len(calls))       # ms per launch
         status |= csp.device_status(ws)
 
     peak, peak_kind = measured_peaks()
     ab = algorithmic_bytes(cfg, n_out_total)
+    layers_per_launch = calls[0][6]
+    ab_launch = {k_: v_ * layers_per_launch for k_, v_ in ab.items()}
     dominant = max(per, key=per.get)
-    achieved = ab[dominant] / (per[dominant] * 1e-3) / 1e9
+    achieved = ab_launch[dominant] / (per[dominant] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
-                "algorithmic_bytes_per_launch": ab[dominant], "us_per_launch": per[dominant] * 1e3}
+                "algorithmic_bytes_per_launch": ab_launch[dominant], "us_per_launch": per[dominant] * 1e3}
     path = {"algorithmic_bytes_per_layer": ab["total"], "us_per_layer": ms_step * 1e3 / n_layers,
             "achieved_gbs": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9,
             "frac_of_hbm_peak": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9 / peak,
-            "kernel_us": {k_: v_ * 1e3 for k_, v_ in per.items()},
-            "kernel_gbs": {k_: ab[k_] / (per[k_] * 1e-3) / 1e9 for k_ in per}}
+            "kernel_us_per_launch": {k_: v_ * 1e3 for k_, v_ in per.items()},
+            "kernel_gbs": {k_: ab_launch[k_] / (per[k_] * 1e-3) / 1e9 for k_ in per}}
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) ----
     e2e = None
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and not args.fold_layers:
         n_host = min(n_buf, 4)
         pin = lambda t: t.cpu().contiguous().pin_memory()
         host = []
@@ -355,7 +415,7 @@ def main():
         b = int(np.argmax(cfg.seq_lens)) if cfg.batch > 1 else 0
         L = int(cfg.seq_lens[b])
         n_units = min(args.cpu_baseline_units, cfg.n_kv_heads)
-        lb = layers[0]
+        lb = first_lb
         qs = lb.q[b:b + 1, :n_units * G].cpu().contiguous()
         ks, vs = lb.k[b:b + 1, :n_units, :L].cpu().contiguous(), lb.v[b:b + 1, :n_units, :L].cpu().contiguous()
         op = orc.Params(1, n_units * G, n_units, cfg.head_dim, cfg.window, cfg.recent, L, cap,
@@ -373,6 +433,9 @@ def main():
                                   f"{reps_cpu} repetitions, {dt:.3f} s each"}
 
     if rank == 0:
+        launch = ("one csp_prune_layer call for all layers (layer axis folded into the batch axis)" if args.fold_layers
+                  else f"cuda graph of one step, {n_chains} concurrent layer chains" if graph is not None
+                  else "one stream, one csp_prune_layer call per layer")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == torch.bfloat16 else "f32",
@@ -381,11 +444,11 @@ def main():
                            "distinct_layer_buffers": n_buf, "batch": cfg.batch, "kv_heads": cfg.n_kv_heads,
                            "q_heads": cfg.n_q_heads, "head_dim": cfg.head_dim, "sum_seq_len": sum_l,
                            "window": cfg.window, "recent": cfg.recent, "kept_rows_per_layer": n_out_total,
-                           "launch": "cuda_graph of one step" if graph is not None else "stream",
+                           "launch": launch,
                            "l2": "inputs larger than L2: every layer has its own K/V buffers"
                                  if n_buf * ab["score"] > 2 * 126e6 else "inputs smaller than L2",
                            "replicas": "one independent replica per GPU, no collective"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * n_layers * 3,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(calls) * 3,
                 "roofline": roofline, "path": path, "cpu_baseline": cpu_baseline, "device_status": status}
         print(json.dumps(line), flush=True)
     if dist is not None:

@@ -68,10 +68,14 @@ struct CompactArgs {
     int32_t n_kv_heads, max_len, out_capacity, chunks_per_row;
 };
 
-// cluster size: the largest power of two (<= 8) that still fits every cluster on the 148 SMs at once
-inline int pick_cluster(int units, int max_tiles) {
+// Cluster size (CTAs per unit, a power of two <= 8).  At least enough CTAs to occupy the 148 SMs when
+// there are few units; more when that lets every CTA keep all of its tiles' logits on chip
+// (`tiles_kept` tiles per CTA; 0 if the kernel keeps none), which removes the second pass over K.
+inline int pick_cluster(int units, int max_tiles, int tiles_kept) {
     int c = 1;
     while (c < 8 && units * (c * 2) <= 148 && c * 2 <= max_tiles) c *= 2;
+    if (tiles_kept > 0)
+        while (c < 8 && (max_tiles + c - 1) / c > tiles_kept) c *= 2;
     return c;
 }
 
@@ -82,6 +86,8 @@ csp_status launch_head_mean(const csp_params& p, const float* part_self, const f
                             float* score_self, float* score_cross, const int32_t* seq_lens,
                             cudaStream_t s);
 csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t s);
+constexpr int kSelectClusterMaxLen = 8 * 1024 * 8;   // longest cache the register-resident cluster select takes
+csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaStream_t s);
 csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_t s);
 
 }  // namespace csp

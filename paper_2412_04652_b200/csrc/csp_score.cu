@@ -467,7 +467,7 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
-    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles);
+    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles, 0);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
     cfg.blockDim = dim3(kThreads);

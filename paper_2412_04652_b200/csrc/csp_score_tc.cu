@@ -11,7 +11,8 @@
 // The same tile stream runs twice:
 //   pass 1  all tiles of the unit: per window row a running (max, sum of 2^(x-max)); merged over
 //           lanes, warps and - through distributed shared memory - the CTAs of the cluster
-//   pass 2  candidate tiles again (L2 hits): one thread per key reads its row of logits,
+//   pass 2  candidate tiles again - from tensor memory where the logits were kept, else recomputed
+//           from K (L2 hits): one thread per key reads its row of logits,
 //           weight = 2^(x*scale + c_w) with c_w = log2(1 / (G (n 2^-m + Z))) - m, added to the key's
 //           intra or inter sum by label equality; no cross-thread reduction is left, and the two
 //           score vectors are written fully coalesced.
@@ -27,7 +28,7 @@ constexpr int kTcThreads = 320;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kMaxStages = 8;
-constexpr int kMaxTmemBufs = 4;
+constexpr int kMaxTmemBufs = 16;
 
 // ---- tcgen05 wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -96,12 +97,15 @@ __device__ __forceinline__ float lg2f(float x) {
     return y;
 }
 
+// Tensor memory (512 columns x 128 lanes of fp32) holds one accumulator of 32G columns per key tile.
+// If all tiles of the CTA fit they simply stay there after pass 1 and pass 2 reads them back: no
+// second pass over K.  Otherwise the first kBufs - kStream tiles stay and the rest cycle through
+// kStream streaming buffers in both passes.
 template <int G> struct TmemPlan {
-    static constexpr int kCols = 32 * G;                                   // accumulator columns per tile
-    static constexpr int kBufs = (512 / kCols) >= kMaxTmemBufs ? kMaxTmemBufs : (512 / kCols);
-    static constexpr int kNeeded = kCols * kBufs;
-    static constexpr int kAlloc = kNeeded <= 32 ? 32 : kNeeded <= 64 ? 64 : kNeeded <= 128 ? 128
-                                  : kNeeded <= 256 ? 256 : 512;
+    static constexpr int kCols = 32 * G;               // accumulator columns per tile
+    static constexpr int kBufs = 512 / kCols;          // 16, 8, 5, 4, 3, 2, 2, 2 for G = 1..8
+    static constexpr int kStream = kBufs >= 8 ? 4 : 2;
+    static constexpr int kAlloc = 512;
 };
 
 struct TcSmemPlan {   // byte offsets from the 1024-aligned base
@@ -127,7 +131,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages) {
     constexpr int KS = NH * 4;                          // MMAs (K = 16 elements = 32 bytes) per tile
     constexpr int NC = TmemPlan<G>::kCols;
-    constexpr int NB = TmemPlan<G>::kBufs;
+    constexpr int TB = TmemPlan<G>::kBufs;
+    constexpr int NS = TmemPlan<G>::kStream;
     constexpr uint32_t kStageBytes = NH * kBlockBytes;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, M = 128, N = NC
     constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NC >> 3) << 17) | (uint32_t(128 >> 4) << 24);
@@ -166,12 +171,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     const int tiles_cand = (N + kTileKeys - 1) / kTileKeys;
     const int my_all = tiles_all > int(rank) ? (tiles_all - int(rank) + int(csize) - 1) / int(csize) : 0;
     const int my_cand = tiles_cand > int(rank) ? (tiles_cand - int(rank) + int(csize) - 1) / int(csize) : 0;
-    const int total = my_all + my_cand;
+    // tiles [0, kept) of this CTA keep their logits in tensor memory between the passes
+    const int kept = my_all <= TB ? my_all : TB - NS;
+    const int streamed1 = my_all - kept;                               // streamed tiles of pass 1
+    const int streamed2 = my_cand > kept ? my_cand - kept : 0;         // tiles recomputed in pass 2
+    const int total = my_all + streamed2;                              // K tiles loaded by this CTA
+    // TMEM buffer and mbarrier parity of tile i of pass `second`
+    auto buf_of = [&](int i, int second) { return i < kept ? i : kept + ((second ? streamed1 : 0) + i - kept) % NS; };
+    auto par_of = [&](int i, int second) {
+        return i < kept ? 0u : uint32_t(((second ? streamed1 : 0) + i - kept) / NS) & 1u;
+    };
 
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
-        for (int i = 0; i < NB; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
+        for (int i = 0; i < TB; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
         mbar_init(q_ready, 8);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -193,7 +207,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             for (int it = 0; it < total; ++it) {
                 const int slot = it % n_stages;
                 const uint32_t round = uint32_t(it / n_stages);
-                const int tile = (it < my_all ? it : it - my_all) * int(csize) + int(rank);
+                const int tile = (it < my_all ? it : it - my_all + kept) * int(csize) + int(rank);
                 mbar_wait(empty_k + 8 * slot, (round & 1u) ^ 1u, abort_flag);
                 if (*abort_flag) break;
                 mbar_expect_tx(full_k + 8 * slot, kStageBytes);
@@ -220,9 +234,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         if (lane == 0) {
             mbar_wait(q_ready, 0, abort_flag);
             for (int it = 0; it < total; ++it) {
-                const int slot = it % n_stages, buf = it % NB;
+                const int slot = it % n_stages;
+                const int second = it >= my_all;
+                const int i = second ? it - my_all + kept : it;        // tile index within its pass
+                const int buf = buf_of(i, second);
                 mbar_wait(full_k + 8 * slot, uint32_t(it / n_stages) & 1u, abort_flag);
-                mbar_wait(tmem_empty + 8 * buf, (uint32_t(it / NB) & 1u) ^ 1u, abort_flag);
+                if (i >= kept) mbar_wait(tmem_empty + 8 * buf, par_of(i, second) ^ 1u, abort_flag);
                 if (*abort_flag) break;
                 tc_fence_after();
                 const uint32_t stage_addr = base + slot * kStageBytes;
@@ -293,10 +310,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) { m_run[g][jj] = kNeg; z_run[g][jj] = 0.f; }
 
-        for (int it = group; it < my_all; it += 2) {
-            const int buf = it % NB;
-            const int tile = it * int(csize) + int(rank);
-            mbar_wait(tmem_full + 8 * buf, uint32_t(it / NB) & 1u, abort_flag);
+        for (int i = group; i < my_all; i += 2) {
+            const int buf = buf_of(i, 0);
+            const int tile = i * int(csize) + int(rank);
+            mbar_wait(tmem_full + 8 * buf, par_of(i, 0), abort_flag);
             tc_fence_after();
             const bool masked = (tile + 1) * kTileKeys > first_masked_key;
             const int t_base = tile * kTileKeys + quarter * 32 + lr;
@@ -336,9 +353,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                         }
                     }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+            if (i >= kept) {                      // streaming buffer: hand it back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+            }
         }
 
         // merge the running statistics: lanes holding the same columns, then warps, then CTAs
@@ -394,12 +413,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         const int ndq = *n_dq;
         const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
 
-        for (int it = my_all + ((my_all ^ group) & 1); it < total; it += 2) {
-            const int buf = it % NB;
-            const int tile = (it - my_all) * int(csize) + int(rank);
+        for (int i = group; i < my_cand; i += 2) {
+            const int buf = buf_of(i, 1);
+            const int tile = i * int(csize) + int(rank);
             const int t = tile * kTileKeys + quarter * 32 + lane;          // this thread's key
             const uint32_t kmod = t < N ? modp[t] : 0u;
-            mbar_wait(tmem_full + 8 * buf, uint32_t(it / NB) & 1u, abort_flag);
+            mbar_wait(tmem_full + 8 * buf, par_of(i, 1), abort_flag);
             tc_fence_after();
             uint32_t same = 0u;                                            // window columns with the key's label
             for (int i = 0; i < ndq; ++i) same = dq_val[i] == kmod ? dq_mask[i] : same;
@@ -426,9 +445,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                     s += (add_s >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c += (add_c >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+            if (i >= kept) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+            }
             if (t < N) { out_s[t] = s; out_c[t] = c; }
         }
         if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
@@ -462,7 +483,7 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
-    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles);
+    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles, TmemPlan<G>::kBufs);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
     cfg.blockDim = dim3(kTcThreads);

@@ -1,4 +1,5 @@
-// Selection kernel: the two top-K masks (Eq. 2), their combination (Eq. 3) and the ascending list
+// Selection kernel for caches longer than 65536 positions (shorter ones take csp_select_cluster.cu):
+// the two top-K masks (Eq. 2), their combination (Eq. 3) and the ascending list
 // of kept positions followed by the recent block (index side of Eq. 4).
 //
 // One CTA per (sequence, KV head) unit.  Up to four top-K problems run together (intra/inter score x
@@ -224,6 +225,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
 csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t s) {
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
+    if (p.max_len <= kSelectClusterMaxLen) return launch_select_cluster(p, a, s);
+    // very long caches: one CTA per unit, keys staged in shared memory as far as it reaches
     // cache as many positions on chip as one CTA's shared memory allows (the rest is read from L2)
     const size_t fixed = 4 * kHistRow * 4;
     size_t n_cached = size_t(p.max_len);
