@@ -97,15 +97,17 @@ __device__ __forceinline__ float lg2f(float x) {
     return y;
 }
 
-// Tensor memory (512 columns x 128 lanes of fp32) holds one accumulator of 32G columns per key tile.
-// If all tiles of the CTA fit they simply stay there after pass 1 and pass 2 reads them back: no
-// second pass over K.  Otherwise the first kBufs - kStream tiles stay and the rest cycle through
-// kStream streaming buffers in both passes.
+// Tensor memory (512 columns x 128 lanes of fp32 per SM) holds one accumulator of 32G columns per key
+// tile.  If all tiles of the CTA fit into its share they simply stay there after pass 1 and pass 2
+// reads them back: no second pass over K.  Otherwise all but 2-4 buffers keep the first tiles and the
+// rest cycle through the remaining "streaming" buffers in both passes.
+// A CTA either owns the SM (512 columns, up to 6 K stages) or shares it with a second CTA (256
+// columns, 3 stages, MHA only), so that one CTA's barrier and epilogue phases overlap the other's
+// streaming.
 template <int G> struct TmemPlan {
     static constexpr int kCols = 32 * G;               // accumulator columns per tile
-    static constexpr int kBufs = 512 / kCols;          // 16, 8, 5, 4, 3, 2, 2, 2 for G = 1..8
-    static constexpr int kStream = kBufs >= 8 ? 4 : 2;
-    static constexpr int kAlloc = 512;
+    static constexpr int kBufs = 512 / kCols;          // buffers when the CTA owns the SM
+    static constexpr int kBufsShared = 256 / kCols;    // buffers when two CTAs share the SM
 };
 
 struct TcSmemPlan {   // byte offsets from the 1024-aligned base
@@ -128,11 +130,12 @@ __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
 
 template <int NH, int G>
 __global__ void __launch_bounds__(kTcThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages) {
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages,
+                const int tmem_cols) {
     constexpr int KS = NH * 4;                          // MMAs (K = 16 elements = 32 bytes) per tile
     constexpr int NC = TmemPlan<G>::kCols;
-    constexpr int TB = TmemPlan<G>::kBufs;
-    constexpr int NS = TmemPlan<G>::kStream;
+    const int TB = tmem_cols / NC;                      // accumulator buffers this CTA owns
+    const int NS = TB >= 8 ? 4 : 2;                     // of which streaming buffers when not all tiles fit
     constexpr uint32_t kStageBytes = NH * kBlockBytes;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, M = 128, N = NC
     constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NC >> 3) << 17) | (uint32_t(128 >> 4) << 24);
@@ -191,7 +194,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == kMmaWarp) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TmemPlan<G>::kAlloc);
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), uint32_t(tmem_cols));
         tmem_relinquish();
     }
     tc_fence_before();
@@ -413,11 +416,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         const int ndq = *n_dq;
         const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
 
+        // this thread's key of tile i is t_of(i); its label is fetched one tile ahead
+        auto t_of = [&](int i) { return (i * int(csize) + int(rank)) * kTileKeys + quarter * 32 + lane; };
+        uint32_t kmod_next = (group < my_cand && t_of(group) < N) ? modp[t_of(group)] : 0u;
         for (int i = group; i < my_cand; i += 2) {
             const int buf = buf_of(i, 1);
-            const int tile = i * int(csize) + int(rank);
-            const int t = tile * kTileKeys + quarter * 32 + lane;          // this thread's key
-            const uint32_t kmod = t < N ? modp[t] : 0u;
+            const int t = t_of(i);
+            const uint32_t kmod = kmod_next;
+            kmod_next = (i + 2 < my_cand && t_of(i + 2) < N) ? modp[t_of(i + 2)] : 0u;
             mbar_wait(tmem_full + 8 * buf, par_of(i, 1), abort_flag);
             tc_fence_after();
             uint32_t same = 0u;                                            // window columns with the key's label
@@ -460,7 +466,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     __syncthreads();
     if (warp == kMmaWarp) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TmemPlan<G>::kAlloc);
+        tmem_dealloc(tmem_base, uint32_t(tmem_cols));
     }
     cluster_arrive();                             // cluster barrier 2
     cluster_wait();
@@ -468,8 +474,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
 
 template <int NH, int G>
 csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
+    const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
+    const int units = p.batch * p.n_kv_heads;
+    // Two CTAs per SM when (MHA) every CTA can still keep all its tiles in its half of tensor memory.
+    bool shared_sm = false;
+    int c = pick_cluster(units, max_tiles, TmemPlan<G>::kBufs);
+    if (G == 1 && NH <= 2) {
+        const int c2 = pick_cluster(units, max_tiles, TmemPlan<G>::kBufsShared);
+        if ((max_tiles + c2 - 1) / c2 <= TmemPlan<G>::kBufsShared) { shared_sm = true; c = c2; }
+    }
     const int fixed = int(tc_smem_plan(NH, G, 0).total) + 1024;
-    int stages = (227 * 1024 - fixed) / (NH * kBlockBytes);
+    int stages = ((shared_sm ? 113 : 227) * 1024 - fixed) / (NH * kBlockBytes);
     if (stages > 6) stages = 6;
     if (stages < 2) return CSP_ERR_UNSUPPORTED;
     const size_t smem = tc_smem_plan(NH, G, stages).total + 1024;
@@ -482,8 +497,6 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
             return CSP_ERR_CUDA;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
-    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles, TmemPlan<G>::kBufs);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
     cfg.blockDim = dim3(kTcThreads);
@@ -493,7 +506,10 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages) != cudaSuccess) { cudaGetLastError(); return CSP_ERR_CUDA; }
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages, shared_sm ? 256 : 512) != cudaSuccess) {
+        cudaGetLastError();
+        return CSP_ERR_CUDA;
+    }
     return CSP_OK;
 }
 
