@@ -1,8 +1,8 @@
 // Selection kernel for caches up to 65536 positions: the two top-K masks (Eq. 2), their combination
 // (Eq. 3) and the ascending list of kept positions followed by the recent block (index side of Eq. 4).
 //
-// A cluster of 1-8 CTAs (1024 threads) owns one (sequence, KV head) unit.  Every thread keeps E (4 or
-// 8) of the unit's keys in registers for the whole kernel (the order-preserving integer images of
+// A cluster of 1-8 CTAs (512 or 1024 threads) owns one (sequence, KV head) unit.  Every thread keeps E (4
+// or 8) of the unit's keys in registers for the whole kernel (the order-preserving integer images of
 // both scores plus a label bit); a warp covers 32 E consecutive positions, lane l holding positions
 // base + 32 e + l, so loads are coalesced and "position order" inside a warp is (e, lane) order,
 // which ballots enumerate for free.  Many warps with little code each hide the latencies of the
@@ -24,8 +24,6 @@ namespace csp {
 namespace {
 using namespace dev;
 
-constexpr int kCsThreads = 1024;
-constexpr int kCsWarps = kCsThreads / 32;
 constexpr uint32_t kFull = 0xffffffffu;
 
 // barrier over the whole cluster; a cluster of one CTA only needs the CTA barrier
@@ -35,8 +33,9 @@ __device__ __forceinline__ void cluster_sync_all(uint32_t csize) {
     cluster_wait();
 }
 
-template <int E>
+template <int kCsThreads, int E>
 __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const SelectArgs a) {
+    constexpr int kCsWarps = kCsThreads / 32;
     __shared__ __align__(16) uint32_t hist[2][4][256];   // ping-pong: a round never zeroes what peers still read
     __shared__ uint32_t chosen[4];                       // digit of the K-th value decided in the last round
     __shared__ int32_t krem[4];                          // how many are still to be taken among the live keys
@@ -328,7 +327,7 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Sel
     if (csize > 1) cluster_wait();                       // peers are done reading this CTA's shared memory
 }
 
-template <int E>
+template <int kCsThreads, int E>
 csp_status launch_e(const csp_params& p, const SelectArgs& a, int cs, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cs, p.batch * p.n_kv_heads, 1);
@@ -339,7 +338,7 @@ csp_status launch_e(const csp_params& p, const SelectArgs& a, int cs, cudaStream
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, select_cluster_kernel<E>, a) != cudaSuccess) { cudaGetLastError(); return CSP_ERR_CUDA; }
+    if (cudaLaunchKernelEx(&cfg, select_cluster_kernel<kCsThreads, E>, a) != cudaSuccess) { cudaGetLastError(); return CSP_ERR_CUDA; }
     return CSP_OK;
 }
 
@@ -349,11 +348,15 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     if (units > 65535) return CSP_ERR_UNSUPPORTED;
-    // 4 keys per thread while a cluster of at most 8 CTAs covers the cache, else 8
-    const int e = p.max_len <= 8 * kCsThreads * 4 ? 4 : 8;
+    // A CTA covers 4096 keys (8192 for caches above 32768 positions).  With few units the kernel is
+    // latency-bound: 1024 threads x 4 keys, many warps with little code each.  With many units it is
+    // throughput-bound: 512 threads x 8 keys, two CTAs per SM overlapping each other's barriers.
+    const int per_cta = p.max_len <= 8 * 4096 ? 4096 : 8192;
     int cs = 1;
-    while (cs < 8 && cs * kCsThreads * e < p.max_len) cs *= 2;
-    return e == 4 ? launch_e<4>(p, a, cs, s) : launch_e<8>(p, a, cs, s);
+    while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
+    if (per_cta == 8192) return launch_e<1024, 8>(p, a, cs, s);
+    if (units * cs >= 2 * 148) return launch_e<512, 8>(p, a, cs, s);
+    return launch_e<1024, 4>(p, a, cs, s);
 }
 
 }  // namespace csp
