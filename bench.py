@@ -95,6 +95,20 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the job is done when every replica is."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, tokens_per_layer: int, n_layers: int, ms_step: float) -> float:
+    """Whole-job metric: every rank prunes its own replica (no exchange step), so the units add up."""
+    return world * tokens_per_layer * n_layers / (ms_step * 1e-3)
+
+
 def algorithmic_bytes(cfg, n_out_total: int):
     """Per-layer algorithmic bytes of each kernel (every tensor touched exactly once)."""
     es = 2 if cfg.dtype == torch.bfloat16 else 4
@@ -305,13 +319,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
         clocks = sampler.stop()
-        ms_total = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms_total], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_total = float(t.item())
+        ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
         ms_step = ms_total / args.steps
-        value = world * sum_l * n_layers / (ms_step * 1e-3)
+        value = job_throughput(world, sum_l, n_layers, ms_step)
 
         # ---- per-kernel durations, live: one CUDA graph per kernel holding that kernel's launch for
         # every call of a step, replayed back to back and timed with events on the launching stream ----
@@ -395,15 +405,12 @@ def main():
             e1.record(stream)
             stream.synchronize()
             ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, dist, dev)
         hb = host[0]
         h2d = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("q", "k", "v")) + \
             n_layers * (h_mod.numel() + 4 * h_lens.numel() + 4 * h_bud.numel())
         d2h = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("k_out", "v_out", "mod_out", "n_out"))
-        e2e = {"value": world * sum_l * n_layers / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": job_throughput(world, sum_l, n_layers, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "api": "csp_prune_layer_host"}
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N=1 only ----
