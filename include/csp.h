@@ -186,6 +186,36 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
                                 int32_t* n_out_host, int32_t* dev_status_host,
                                 void* staging, size_t staging_bytes, void* cuda_stream);
 
+/*
+ * No counterpart in the paper: a convenience of this library.  Algorithm 1 exactly as
+ * csp_prune_layer computes it, for callers that have no way to obtain scratch memory: code that runs
+ * after a serving engine has claimed all device memory for its own pool, plug-ins that are handed
+ * tensors but no allocator, or latency-critical loops where a cudaMalloc (which stalls the device)
+ * is not acceptable.  The scratch (status word, score vectors, index list) is a fixed array inside
+ * the library, csp_static_workspace_limit() bytes (8 MiB) on every GPU that loads it, held until
+ * the process exits.  The call allocates and frees nothing.
+ *   - Shapes whose csp_workspace_bytes exceeds the limit are refused with CSP_ERR_WORKSPACE and
+ *     nothing is enqueued (8 MiB covers e.g. 32 KV heads x 4096 positions; use csp_prune_layer with
+ *     your own workspace beyond that).
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array, which still holds the previous call's contents; the status
+ *     area is cleared on the stream at the start of every call.  Two calls whose GPU work can
+ *     overlap (different streams, several host threads) race on it: serialise them.
+ *   - dev_status_out_or_null: DEVICE pointer to one int32 that receives the CSP_DEV_* status word
+ *     of this call (copied on the stream); per-unit failures also show as n_out == -1.
+ * Inputs, outputs and all other rules are those of csp_prune_layer.
+ */
+csp_status csp_prune_layer_static(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
+                                  const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                                  const int32_t* seq_lens, const int32_t* budgets,
+                                  const int32_t* total_budget_or_null, const float* lse_or_null,
+                                  csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
+                                  int32_t* dev_status_out_or_null, void* cuda_stream);
+
+/* Size in bytes of the built-in scratch array used by csp_prune_layer_static. */
+size_t csp_static_workspace_limit(void);
+
 /* Waits for the stream, copies the status word to *host_out (may be NULL), clears it, and returns
  * CSP_ERR_TIMEOUT if CSP_DEV_TIMEOUT was set, else CSP_OK. */
 csp_status csp_device_status(void* workspace, void* cuda_stream, int32_t* host_out);

@@ -25,7 +25,7 @@ DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
 
 EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_select", "csp_compact",
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
-           "csp_status_string")
+           "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit")
 
 
 class CspError(RuntimeError):
@@ -99,6 +99,11 @@ def lib() -> C.CDLL:
         l.csp_prune_layer_host.restype = C.c_int
         l.csp_prune_layer_host.argtypes = [P, vp, vp, vp, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp,
                                            vp, sz, vp]
+        l.csp_prune_layer_static.restype = C.c_int
+        l.csp_prune_layer_static.argtypes = [P, CTensor, CTensor, CTensor, vp, i64, i64, vp, vp, vp, vp,
+                                             CTensor, CTensor, vp, vp, vp, vp]
+        l.csp_static_workspace_limit.restype = sz
+        l.csp_static_workspace_limit.argtypes = []
         l.csp_device_status.restype = C.c_int
         l.csp_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         l.csp_status_string.restype = C.c_char_p
@@ -189,6 +194,22 @@ def prune_layer(p: Params, q_win, k, v, modality, seq_lens, budgets, k_out, v_ou
                                  tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
                                  _ptr(score_self), _ptr(score_cross), _ptr(keep_idx),
                                  _ptr(ws), ws.numel(), _stream()), "csp_prune_layer")
+
+
+def static_workspace_limit() -> int:
+    return int(lib().csp_static_workspace_limit())
+
+
+def prune_layer_static(p: Params, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, mod_out, n_out,
+                       total_budget=None, lse=None, dev_status_out=None):
+    """csp_prune_layer without a caller workspace: the library's built-in scratch array is used, so
+    nothing is allocated.  Raises CspError(ERR_WORKSPACE) for shapes beyond static_workspace_limit()."""
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_prune_layer_static(C.byref(cp), tensor4(q_win), tensor4(k), tensor4(v), _ptr(modality), sb, sh,
+                                        _ptr(seq_lens), _ptr(budgets), _ptr(total_budget), _ptr(lse),
+                                        tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
+                                        _ptr(dev_status_out), _stream()), "csp_prune_layer_static")
 
 
 def host_staging_bytes(p: Params) -> int:
