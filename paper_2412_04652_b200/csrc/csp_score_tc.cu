@@ -72,6 +72,15 @@ __device__ __forceinline__ void tc_ld_row32(uint32_t (&v)[32], uint32_t taddr) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+// one row (TMEM lane) per thread, 16 consecutive fp32 columns
+__device__ __forceinline__ void tc_ld_row16(uint32_t (&v)[16], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
 // 16 rows x 32 columns spread over the warp like an mma accumulator: thread (lane) holds, for each
 // 8-column block i, regs 4i..4i+3 = (row lane/4, cols 2(lane%4)+{0,1}), (row lane/4+8, same cols)
 __device__ __forceinline__ void tc_ld_16x32(uint32_t (&v)[16], uint32_t taddr) {
@@ -129,7 +138,7 @@ __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
 }
 
 template <int NH, int G>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, (G == 1 && NH <= 2) ? 2 : 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages,
                 const int tmem_cols) {
     constexpr int KS = NH * 4;                          // MMAs (K = 16 elements = 32 bytes) per tile
@@ -427,30 +436,37 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             mbar_wait(tmem_full + 8 * buf, par_of(i, 1), abort_flag);
             tc_fence_after();
             uint32_t same = 0u;                                            // window columns with the key's label
-            for (int i = 0; i < ndq; ++i) same = dq_val[i] == kmod ? dq_mask[i] : same;
+            for (int q = 0; q < ndq; ++q) same = dq_val[q] == kmod ? dq_mask[q] : same;
             const int delta = t - first_masked_key;                        // column w sees the key iff w >= delta
             const uint32_t vis = delta <= 0 ? wmask : (delta >= 32 ? 0u : (wmask & (0xFFFFFFFFu << delta)));
             const uint32_t add_s = same & vis, add_c = ~same & vis;
-            float s = 0.f, c = 0.f;
+            // the row of 32 G logits is read in chunks of 16 columns; the load of the next chunk is in
+            // flight while the current one is turned into weights (two accumulators per score)
+            float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
+            const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
+            uint32_t va[16], vb[16];
+            tc_ld_row16(va, row_addr);
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                uint32_t v[32];
-                tc_ld_row32(v, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + g * 32));
+            for (int ch = 0; ch < 2 * G; ++ch) {
                 tc_wait_ld();
-                const float4* cv = reinterpret_cast<const float4*>(cvec + g * 32);
+                uint32_t (&cur)[16] = (ch & 1) ? vb : va;
+                if (ch + 1 < 2 * G) tc_ld_row16((ch & 1) ? va : vb, row_addr + uint32_t((ch + 1) * 16));
+                const float4* cv = reinterpret_cast<const float4*>(cvec + ch * 16);
+                const uint32_t as = add_s >> ((ch & 1) * 16), ac = add_c >> ((ch & 1) * 16);
 #pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
+                for (int j4 = 0; j4 < 4; ++j4) {
                     const float4 cc = cv[j4];
-                    const float p0 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 0]), scale2, cc.x));
-                    const float p1 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 1]), scale2, cc.y));
-                    const float p2 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 2]), scale2, cc.z));
-                    const float p3 = ex2f(fmaf(__uint_as_float(v[j4 * 4 + 3]), scale2, cc.w));
-                    s += (add_s >> (j4 * 4 + 0)) & 1u ? p0 : 0.f; c += (add_c >> (j4 * 4 + 0)) & 1u ? p0 : 0.f;
-                    s += (add_s >> (j4 * 4 + 1)) & 1u ? p1 : 0.f; c += (add_c >> (j4 * 4 + 1)) & 1u ? p1 : 0.f;
-                    s += (add_s >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c += (add_c >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
-                    s += (add_s >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c += (add_c >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
+                    const float p0 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                    const float p1 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                    const float p2 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                    const float p3 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                    s0 += (as >> (j4 * 4 + 0)) & 1u ? p0 : 0.f; c0 += (ac >> (j4 * 4 + 0)) & 1u ? p0 : 0.f;
+                    s1 += (as >> (j4 * 4 + 1)) & 1u ? p1 : 0.f; c1 += (ac >> (j4 * 4 + 1)) & 1u ? p1 : 0.f;
+                    s0 += (as >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c0 += (ac >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
+                    s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                 }
             }
+            const float s = s0 + s1, c = c0 + c1;
             if (i >= kept) {
                 tc_fence_before();
                 __syncwarp();
