@@ -197,7 +197,7 @@ def main():
     ap.add_argument("--ref-units", type=int, default=8, help="KV heads per reference-arm step")
     ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"])
-    ap.add_argument("--streams", type=int, default=8, help="concurrent layer chains inside the step graph")
+    ap.add_argument("--streams", type=int, default=32, help="concurrent layer chains inside the step graph")
     ap.add_argument("--fold-layers", action="store_true",
                     help="one call for all layers: the layer axis of a [layers*B, H, L, d] cache is passed as batch")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -82,6 +82,8 @@ inline int pick_cluster(int units, int max_tiles, int tiles_kept) {
 // ---- host-side launchers (defined next to their kernels) ----------------------------------
 csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s);
 csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s);
+csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
+                                bool* taken);
 csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,
                             float* score_self, float* score_cross, const int32_t* seq_lens,
                             cudaStream_t s);

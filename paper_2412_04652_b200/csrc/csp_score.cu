@@ -532,7 +532,12 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tenso
                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return CSP_ERR_UNSUPPORTED;
-    return p.dtype == CSP_F32 ? launch_t<float>(p, a, tmap, s) : launch_score_tc(p, a, tmap, s);
+    if (p.dtype == CSP_F32) return launch_t<float>(p, a, tmap, s);
+    // many MHA units: resident clusters that stream unit after unit; otherwise one cluster per unit
+    bool taken = false;
+    const csp_status ps = launch_score_persist(p, a, tmap, s, &taken);
+    if (ps != CSP_OK || taken) return ps;
+    return launch_score_tc(p, a, tmap, s);
 }
 
 csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,

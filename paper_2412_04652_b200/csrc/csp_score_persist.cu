@@ -1,0 +1,467 @@
+// Persistent variant of the bf16 tcgen05 scoring kernel for many MHA units (window logits Eq. 5,
+// n-softmax rows Eq. 7, recent trim, intra/inter query-axis sums Eq. 1).
+//
+// Used when a launch has more (sequence, head) units than clusters fit on the GPU.  A cluster of C
+// CTAs stays resident and walks over units cluster_id, cluster_id + n_clusters, ...  The roles of a
+// CTA are decoupled by mbarriers so that the K stream never stops between units:
+//   warp 8   TMA producer: runs ahead into the next unit's K tiles as soon as ring stages free up
+//   warp 9   MMA issuer: logits of unit j go to half (j & 1) of tensor memory (8 tiles of 32 columns)
+//   warp 10  stages Q and the query-label table of the next unit while the current one is in flight
+//   warps 0-7 epilogue: pass 1 statistics, cluster-wide merge, pass 2 from tensor memory, scores
+// While the epilogue warps finish unit j (statistics exchange, pass 2), the producer and the tensor
+// core already work on unit j + 1 in the other half.  The cluster-wide merge of the row statistics
+// uses an mbarrier per CTA that all CTAs of the cluster arrive on remotely, so only the epilogue
+// warps take part and nobody else is held up.  Every wait is bounded.
+//
+// Precondition (checked by the launcher): G = 1, no caller-supplied LSE, and at most 8 tiles per CTA,
+// so that every tile's logits stay in tensor memory between the passes.
+#include "csp_internal.cuh"
+#include "csp_tc.cuh"
+
+namespace csp {
+namespace {
+using namespace dev;
+
+// barrier over the 256 epilogue threads that also tells everyone whether any of them saw `pred`
+__device__ __forceinline__ bool consumer_any(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "barrier.cta.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(uint32_t(pred)), "n"(kConsumerThreads) : "memory");
+    return r != 0;
+}
+
+constexpr int kPsThreads = 352;                         // 8 epilogue warps, producer, MMA issuer, stager
+constexpr int kPsProducerWarp = 8;
+constexpr int kPsMmaWarp = 9;
+constexpr int kPsStageWarp = 10;
+constexpr int kHalfBufs = 8;                            // tiles whose logits one half of tensor memory holds
+constexpr int kPsMaxStages = 8;
+
+struct PsSmemPlan {   // byte offsets from the 1024-aligned base
+    uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
+};
+__host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
+    PsSmemPlan s;
+    uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
+    s.q = off;        off += 2u * uint32_t(nh) * 32u * 128u;      // two units in flight
+    s.wstats = off;   off += 8u * 32u * 8u;
+    s.cstats = off;   off += 2u * 32u * 8u;                       // ping-pong, read by the peers
+    s.cvec = off;     off += 32u * 4u;
+    s.dq_mask = off;  off += 2u * 32u * 4u;
+    s.dq_val = off;   off += 2u * 32u * 4u;
+    s.bars = off;     off += (2u * kPsMaxStages + 2u * kHalfBufs + 8u) * 8u;
+    s.misc = off;     off += 32u;     // tmem base, abort flag, n distinct query labels [2]
+    s.total = off;
+    return s;
+}
+
+template <int NH>
+__global__ void __launch_bounds__(kPsThreads, 1)
+score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages,
+                        const int n_units, const int n_clusters) {
+    constexpr int KS = NH * 4;
+    constexpr int NC = 32;
+    constexpr uint32_t kStageBytes = NH * kBlockBytes;
+    constexpr uint32_t kQBytes = NH * 32 * 128;
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NC >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const PsSmemPlan sp = ps_smem_plan(NH, n_stages);
+    float2* const wstats = reinterpret_cast<float2*>(base_ptr + sp.wstats);
+    float2* const cstats = reinterpret_cast<float2*>(base_ptr + sp.cstats);
+    float* const cvec = reinterpret_cast<float*>(base_ptr + sp.cvec);
+    uint32_t* const dq_mask = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_mask);
+    uint32_t* const dq_val = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_val);
+    const uint32_t full_k = base + sp.bars;
+    const uint32_t empty_k = full_k + 8 * kPsMaxStages;
+    const uint32_t tmem_full = empty_k + 8 * kPsMaxStages;        // [2][8]
+    const uint32_t half_free = tmem_full + 8 * 2 * kHalfBufs;     // [2] epilogue done with the half
+    const uint32_t q_ready = half_free + 16;                      // [2] Q and label table staged
+    const uint32_t q_free = q_ready + 16;                         // [2] tensor core done reading Q
+    const uint32_t stats_ready = q_free + 16;                     // [2] every CTA of the cluster published its statistics
+    volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + sp.misc);
+    volatile int* const abort_flag = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 4);
+    volatile int* const n_dq = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 8);   // [2]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_rank(), csize = cluster_size();
+    const int cid = int(blockIdx.x / csize);
+    const int W = a.window;
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
+        for (int i = 0; i < 2 * kHalfBufs; ++i) mbar_init(tmem_full + 8 * i, 1);
+        for (int p = 0; p < 2; ++p) {
+            mbar_init(half_free + 8 * p, 8);
+            mbar_init(q_ready + 8 * p, 1);
+            mbar_init(q_free + 8 * p, 1);
+            mbar_init(stats_ready + 8 * p, csize);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == kPsMmaWarp) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512u);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    // peers arrive on this CTA's barriers: nobody may start before every CTA has initialised them
+    cluster_arrive();
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // what every role needs to know about unit u
+    struct Unit { int b, h, L, N, my_all, my_cand; bool skip; };
+    auto unit_of = [&](int u) {
+        Unit x;
+        x.b = u / a.n_kv_heads; x.h = u % a.n_kv_heads;
+        int L = a.seq_lens[x.b];
+        const bool bad = L < 0 || L > a.max_len;
+        x.skip = bad || L < a.window || L < a.recent;
+        if (x.skip) L = 0;
+        x.L = L;
+        x.N = x.skip ? 0 : L - a.recent;
+        const int tiles_all = (L + kTileKeys - 1) / kTileKeys, tiles_cand = (x.N + kTileKeys - 1) / kTileKeys;
+        x.my_all = tiles_all > int(rank) ? (tiles_all - int(rank) + int(csize) - 1) / int(csize) : 0;
+        x.my_cand = tiles_cand > int(rank) ? (tiles_cand - int(rank) + int(csize) - 1) / int(csize) : 0;
+        if (x.my_all > kHalfBufs) x.my_all = kHalfBufs;          // never happens (launcher); keeps indices in range
+        if (x.my_cand > x.my_all) x.my_cand = x.my_all;
+        return x;
+    };
+
+    if (warp == kPsProducerWarp) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            int it = 0;
+            for (int u = cid; u < n_units && !*abort_flag; u += n_clusters) {
+                const Unit x = unit_of(u);
+                for (int i = 0; i < x.my_all; ++i, ++it) {
+                    const int slot = it % n_stages;
+                    mbar_wait(empty_k + 8 * slot, (uint32_t(it / n_stages) & 1u) ^ 1u, abort_flag);
+                    if (*abort_flag) break;
+                    mbar_expect_tx(full_k + 8 * slot, kStageBytes);
+                    const int tile = i * int(csize) + int(rank);
+#pragma unroll
+                    for (int hb = 0; hb < NH; ++hb)
+                        tma_load_4d(base + slot * kStageBytes + hb * kBlockBytes, &tmap, full_k + 8 * slot,
+                                    hb * 64, tile * kTileKeys, x.h, x.b);
+                }
+            }
+            if (*abort_flag) {
+                // let copies that were issued land before the CTA's shared memory is given up
+                for (int s = 0; s < n_stages; ++s) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_k + 8 * s, 0) && !mbar_try_wait(full_k + 8 * s, 1) &&
+                           global_ns() - t0 < kWaitLimitNs / 8) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == kPsMmaWarp) {
+        // =============================== MMA issuer ===============================
+        if (lane == 0) {
+            int it = 0, j = 0;
+            for (int u = cid; u < n_units && !*abort_flag; u += n_clusters, ++j) {
+                const Unit x = unit_of(u);
+                const int p = j & 1;
+                const uint32_t ph = uint32_t(j >> 1) & 1u;
+                mbar_wait(q_ready + 8 * p, ph, abort_flag);             // Q of this unit is in shared memory
+                mbar_wait(half_free + 8 * p, ph ^ 1u, abort_flag);      // the unit two back left this half
+                const uint32_t q_s = base + sp.q + uint32_t(p) * kQBytes;
+                for (int i = 0; i < x.my_all; ++i, ++it) {
+                    const int slot = it % n_stages;
+                    mbar_wait(full_k + 8 * slot, uint32_t(it / n_stages) & 1u, abort_flag);
+                    if (*abort_flag) break;
+                    tc_fence_after();
+                    const uint32_t stage_addr = base + slot * kStageBytes;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const uint64_t ad = sw128_desc(stage_addr + uint32_t(ks >> 2) * kBlockBytes + uint32_t(ks & 3) * 32u);
+                        const uint64_t bd = sw128_desc(q_s + uint32_t(ks >> 2) * (NC * 128u) + uint32_t(ks & 3) * 32u);
+                        tc_mma_bf16(tmem_base + uint32_t((p * kHalfBufs + i) * NC), ad, bd, kIdesc, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(empty_k + 8 * slot);
+                    tc_commit(tmem_full + 8 * (p * kHalfBufs + i));
+                }
+                // buffers this unit does not use still flip once per unit: one parity rule for all of them
+                for (int i = x.my_all; i < kHalfBufs; ++i) mbar_arrive(tmem_full + 8 * (p * kHalfBufs + i));
+                tc_commit(q_free + 8 * p);
+            }
+        }
+        __syncwarp();
+    } else if (warp == kPsStageWarp) {
+        // =============================== Q / label-table stager ===============================
+        int j = 0;
+        for (int u = cid; u < n_units; u += n_clusters, ++j) {
+            if (__any_sync(0xffffffffu, *abort_flag != 0)) break;        // the whole warp leaves together
+            const Unit x = unit_of(u);
+            const int p = j & 1;
+            const uint32_t ph = uint32_t(j >> 1) & 1u;
+            mbar_wait(q_free + 8 * p, ph ^ 1u, abort_flag);
+            mbar_wait(half_free + 8 * p, ph ^ 1u, abort_flag);
+            uint8_t* const q_dst = base_ptr + sp.q + p * kQBytes;
+            const uint8_t* qb = static_cast<const uint8_t*>(a.q);
+            constexpr int kChunksPerRow = NH * 8;
+            for (int i = lane; i < 32 * kChunksPerRow; i += 32) {
+                const int w = i / kChunksPerRow, c = i % kChunksPerRow;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (w < W && !x.skip) {
+                    const int64_t e = int64_t(x.b) * a.q_sb + int64_t(x.h) * a.q_sh + int64_t(w) * a.q_st;
+                    v = *reinterpret_cast<const uint4*>(qb + e * 2 + c * 16);
+                }
+                const uint32_t off = uint32_t(c >> 3) * (NC * 128) + uint32_t(w) * 128 + (uint32_t((c & 7) ^ (w & 7)) << 4);
+                *reinterpret_cast<uint4*>(q_dst + off) = v;
+            }
+            // table of the distinct labels of the window queries and the columns carrying each
+            const uint8_t* modp = a.modality + int64_t(x.b) * a.mod_sb + int64_t(x.h) * a.mod_sh;
+            const uint32_t ql = (lane < W && !x.skip) ? modp[x.L - W + lane] : 0xFFFFFFFFu;
+            int count = 0;
+            for (int jq = 0; jq < W; ++jq) {
+                const uint32_t vj = __shfl_sync(0xffffffffu, ql, jq);
+                const uint32_t same = __ballot_sync(0xffffffffu, ql == vj);
+                if ((same & ((1u << jq) - 1u)) == 0u) {               // no earlier column has this label
+                    if (lane == 0) { dq_val[p * 32 + count] = vj; dq_mask[p * 32 + count] = same; }
+                    ++count;
+                }
+            }
+            if (lane == 0) n_dq[p] = x.skip ? 0 : count;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make Q visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(q_ready + 8 * p);
+        }
+    } else {
+        // =============================== epilogue warps ===============================
+        const int quarter = warp & 3, group = warp >> 2;
+        const int lq = lane & 3, lr = lane >> 2;
+        const float scale2 = a.scale_log2;
+        const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
+        int j = 0;
+        for (int u = cid; u < n_units; u += n_clusters, ++j) {
+            if (consumer_any(*abort_flag != 0)) break;                   // all 256 threads leave together
+            const Unit x = unit_of(u);
+            const int p = j & 1;
+            const uint32_t ph = uint32_t(j >> 1) & 1u;
+            const int first_masked_key = x.L - W;
+            const uint8_t* modp = a.modality + int64_t(x.b) * a.mod_sb + int64_t(x.h) * a.mod_sh;
+            if (tid == 0 && rank == 0) {
+                const int Lraw = a.seq_lens[x.b];
+                if (Lraw < 0 || Lraw > a.max_len) atomicOr(a.status, CSP_DEV_BAD_LEN);
+            }
+
+            // ---------------------------------- pass 1 ----------------------------------
+            float m_run[8], z_run[8];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) { m_run[jj] = kNeg; z_run[jj] = 0.f; }
+            for (int i = group; i < x.my_all; i += 2) {
+                const int buf = p * kHalfBufs + i;
+                const int tile = i * int(csize) + int(rank);
+                mbar_wait(tmem_full + 8 * buf, ph, abort_flag);
+                tc_fence_after();
+                const bool masked = (tile + 1) * kTileKeys > first_masked_key;
+                const int t_base = tile * kTileKeys + quarter * 32 + lr;
+                uint32_t v0[16], v1[16];
+                tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC));
+                tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + uint32_t(buf * NC));
+                tc_wait_ld();
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int jj = nt * 2 + e;
+                        float xv[4] = {__uint_as_float(v0[nt * 4 + e]) * scale2, __uint_as_float(v0[nt * 4 + 2 + e]) * scale2,
+                                       __uint_as_float(v1[nt * 4 + e]) * scale2, __uint_as_float(v1[nt * 4 + 2 + e]) * scale2};
+                        if (!masked) {
+                            const float mx = fmaxf(fmaxf(xv[0], xv[1]), fmaxf(xv[2], xv[3]));
+                            if (mx > m_run[jj] + kLazy) { z_run[jj] *= ex2f(m_run[jj] - mx); m_run[jj] = mx; }
+                            const float mm = m_run[jj];
+                            z_run[jj] += (ex2f(xv[0] - mm) + ex2f(xv[1] - mm)) + (ex2f(xv[2] - mm) + ex2f(xv[3] - mm));
+                        } else {
+                            const int colw = nt * 8 + lq * 2 + e;
+                            bool vis[4];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                const int t = t_base + (r & 1) * 8 + (r >> 1) * 16;
+                                vis[r] = colw < W && t <= first_masked_key + colw;   // key <= query position
+                                xv[r] = vis[r] ? xv[r] : kNeg;
+                            }
+                            const float mx = fmaxf(fmaxf(xv[0], xv[1]), fmaxf(xv[2], xv[3]));
+                            if (mx > m_run[jj] + kLazy) { z_run[jj] *= ex2f(m_run[jj] - mx); m_run[jj] = mx; }
+                            const float mm = m_run[jj];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) z_run[jj] += vis[r] ? ex2f(xv[r] - mm) : 0.f;
+                        }
+                    }
+            }
+            // merge: lanes holding the same columns, then warps, then the CTAs of the cluster
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+#pragma unroll
+                for (int d = 4; d <= 16; d <<= 1) {
+                    const float om = __shfl_xor_sync(0xffffffffu, m_run[jj], d);
+                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[jj], d);
+                    merge_stats(m_run[jj], z_run[jj], om, oz);
+                }
+                if (lr == 0) wstats[warp * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
+            }
+            consumer_sync();
+            if (warp == 0) {
+                float m = kNeg, z = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {
+                    const float2 s = wstats[w * 32 + lane];
+                    merge_stats(m, z, s.x, s.y);
+                }
+                cstats[p * 32 + lane] = make_float2(m, z);
+                __syncwarp();
+                asm volatile("fence.acq_rel.cluster;" ::: "memory");
+                if (lane < int(csize)) mbar_arrive_remote(stats_ready + 8 * p, uint32_t(lane));   // publish to every CTA
+            }
+            mbar_wait_cluster(stats_ready + 8 * p, ph, abort_flag);
+            if (warp == 0) {
+                float m = kNeg, z = 0.f;
+                for (uint32_t r = 0; r < csize; ++r) {
+                    const float2 s = ld_remote_f2(smem_u32(&cstats[p * 32 + lane]), r);
+                    merge_stats(m, z, s.x, s.y);
+                }
+                // weight of 2^(x - m) is 1 / (n 2^-m + Z); fold it and -m into one additive constant
+                const float denom = a.n * ex2f(-m) + z;
+                cvec[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
+            }
+            mbar_wait(q_ready + 8 * p, ph, abort_flag);                  // label table of this unit
+            consumer_sync();
+
+            // ---------------------------------- pass 2 ----------------------------------
+            float* const out_s = a.score_self + (int64_t(x.b) * a.n_kv_heads + x.h) * a.max_len;
+            float* const out_c = a.score_cross + (int64_t(x.b) * a.n_kv_heads + x.h) * a.max_len;
+            const int ndq = n_dq[p];
+            auto t_of = [&](int i) { return (i * int(csize) + int(rank)) * kTileKeys + quarter * 32 + lane; };
+            uint32_t kmod_next = (group < x.my_cand && t_of(group) < x.N) ? modp[t_of(group)] : 0u;
+            for (int i = group; i < x.my_cand; i += 2) {
+                const int buf = p * kHalfBufs + i;
+                const int t = t_of(i);
+                const uint32_t kmod = kmod_next;
+                kmod_next = (i + 2 < x.my_cand && t_of(i + 2) < x.N) ? modp[t_of(i + 2)] : 0u;
+                uint32_t same = 0u;                                        // window columns with the key's label
+                for (int q = 0; q < ndq; ++q) same = dq_val[p * 32 + q] == kmod ? dq_mask[p * 32 + q] : same;
+                const int delta = t - first_masked_key;                    // column w sees the key iff w >= delta
+                const uint32_t vis = delta <= 0 ? wmask : (delta >= 32 ? 0u : (wmask & (0xFFFFFFFFu << delta)));
+                const uint32_t add_s = same & vis, add_c = ~same & vis;
+                float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
+                const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
+                uint32_t va[16], vb[16];
+                tc_ld_row16(va, row_addr);
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    tc_wait_ld();
+                    uint32_t (&cur)[16] = ch ? vb : va;
+                    if (ch == 0) tc_ld_row16(vb, row_addr + 16u);
+                    const float4* cv = reinterpret_cast<const float4*>(cvec + ch * 16);
+                    const uint32_t as = add_s >> (ch * 16), ac = add_c >> (ch * 16);
+#pragma unroll
+                    for (int j4 = 0; j4 < 4; ++j4) {
+                        const float4 cc = cv[j4];
+                        const float p0 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                        const float p1 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                        const float p2 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                        const float p3 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                        s0 += (as >> (j4 * 4 + 0)) & 1u ? p0 : 0.f; c0 += (ac >> (j4 * 4 + 0)) & 1u ? p0 : 0.f;
+                        s1 += (as >> (j4 * 4 + 1)) & 1u ? p1 : 0.f; c1 += (ac >> (j4 * 4 + 1)) & 1u ? p1 : 0.f;
+                        s0 += (as >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c0 += (ac >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
+                        s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
+                    }
+                }
+                if (t < x.N) { out_s[t] = s0 + s1; out_c[t] = c0 + c1; }
+            }
+            // this half of tensor memory, the label table and Q of this parity may now be reused
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(half_free + 8 * p);
+        }
+        if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
+    }
+
+    // every warp: give tensor memory back, then keep shared memory alive until the peers are done
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kPsMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512u);
+    }
+    cluster_arrive();
+    cluster_wait();
+}
+
+template <int NH>
+csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, int c, cudaStream_t s,
+                     bool* taken) {
+    const int units = p.batch * p.n_kv_heads;
+    const int fixed = int(ps_smem_plan(NH, 0).total) + 1024;
+    int stages = (227 * 1024 - fixed) / (NH * kBlockBytes);
+    if (stages > 6) stages = 6;
+    if (stages < 2) return CSP_OK;
+    const size_t smem = ps_smem_plan(NH, stages).total + 1024;
+    auto kern = score_tc_persist_kernel<NH>;
+    static bool configured[64] = {};
+    static int resident[64] = {};      // clusters of this size that fit on the device at once
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return CSP_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kPsThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            return CSP_ERR_CUDA;
+        configured[dev] = true;
+    }
+    static int resident_c[64] = {};
+    if (resident[dev] == 0 || resident_c[dev] != c) {
+        cfg.gridDim = dim3((148 / c) * c, 1, 1);
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = 148 / c / 2; }
+        resident[dev] = n > 0 ? n : 1;
+        resident_c[dev] = c;
+    }
+    const int n_clusters = resident[dev];
+    if (units < 2 * n_clusters) return CSP_OK;           // too few units for a resident loop to pay off
+    cfg.gridDim = dim3(n_clusters * c, 1, 1);
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages, units, n_clusters) != cudaSuccess) {
+        cudaGetLastError();
+        return CSP_ERR_CUDA;
+    }
+    *taken = true;
+    return CSP_OK;
+}
+
+}  // namespace
+
+// Launches the persistent kernel if the shape qualifies; *taken tells whether it did.
+csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
+                                bool* taken) {
+    *taken = false;
+    if (a.group != 1 || a.lse != nullptr) return CSP_OK;
+    const int row_bytes = p.head_dim * 2;
+    if (row_bytes != 128 && row_bytes != 256) return CSP_OK;
+    const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
+    int c = 1;
+    while (c < 8 && (max_tiles + c - 1) / c > kHalfBufs) c *= 2;
+    if ((max_tiles + c - 1) / c > kHalfBufs) return CSP_OK;
+    return row_bytes == 128 ? launch_nh<1>(p, a, tmap, c, s, taken) : launch_nh<2>(p, a, tmap, c, s, taken);
+}
+
+}  // namespace csp

@@ -74,6 +74,20 @@ def test_score_matches_oracle(csp, oracle, lens, n_q, n_kv, d, W, R, dtype):
     _run_score(csp, oracle, _case(lens, n_q, n_kv, d, W, R, dtype=dtype, seed=len(lens) + n_q))
 
 
+@pytest.mark.parametrize("lens_hi,n_seq,heads", [(1000, 40, 8), (2500, 20, 16)])
+def test_score_many_units_resident_clusters(csp, oracle, lens_hi, n_seq, heads):
+    """More MHA units than clusters fit on the GPU: the resident-cluster kernel walks unit after unit
+    (clusters of 1 and of 4 CTAs), ragged lengths, every unit compared."""
+    rng = np.random.RandomState(lens_hi)
+    lens = tuple(int(x) for x in rng.randint(90, lens_hi, size=n_seq))
+    cfg = _case(lens, heads, heads, 128, 32, 32, seed=17)
+    mod = cfg.modality()
+    mod[:, -40:] = (rng.rand(n_seq, 40) < 0.3)          # padding labels and some mixed windows
+    for b, L in enumerate(lens):
+        mod[b, L - 32:L] = (rng.rand(32) < (0.5 if b % 3 == 0 else 0.0))
+    _run_score(csp, oracle, cfg, modality=mod.astype(np.uint8))
+
+
 def test_score_mixed_modality_window_and_per_head_labels(csp, oracle):
     cfg = _case((600, 350), 4, 2, 128, 32, 32, seed=5)
     rng = np.random.RandomState(0)
