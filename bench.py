@@ -109,6 +109,12 @@ def job_throughput(world: int, tokens_per_layer: int, n_layers: int, ms_step: fl
     return world * tokens_per_layer * n_layers / (ms_step * 1e-3)
 
 
+# DRAM bytes (read + write) per launch of each kernel on configs[1], one layer per launch, from the ncu
+# captures summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  Scales with the
+# number of layers a launch covers.  None for workloads that were not captured.
+NCU_DRAM_BYTES_PER_LAYER = {1: {"score": 33.88e6, "select": 1.08e6, "compact": 16.97e6}}
+
+
 def algorithmic_bytes(cfg, n_out_total: int):
     """Per-layer algorithmic bytes of each kernel (every tensor touched exactly once)."""
     es = 2 if cfg.dtype == torch.bfloat16 else 4
@@ -364,8 +370,10 @@ def main():
     ab_launch = {k_: v_ * layers_per_launch for k_, v_ in ab.items()}
     dominant = max(per, key=per.get)
     achieved = ab_launch[dominant] / (per[dominant] * 1e-3) / 1e9
+    traffic = NCU_DRAM_BYTES_PER_LAYER.get(args.config, {}).get(dominant)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "frac": achieved / peak, "traffic": None if traffic is None else traffic * layers_per_launch,
+                "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": ab_launch[dominant], "us_per_launch": per[dominant] * 1e3}
     path = {"algorithmic_bytes_per_layer": ab["total"], "us_per_layer": ms_step * 1e3 / n_layers,
             "achieved_gbs": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9,

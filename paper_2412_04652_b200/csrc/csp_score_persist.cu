@@ -4,10 +4,12 @@
 // Used when a launch has more (sequence, head) units than clusters fit on the GPU.  A cluster of C
 // CTAs stays resident and walks over units cluster_id, cluster_id + n_clusters, ...  The roles of a
 // CTA are decoupled by mbarriers so that the K stream never stops between units:
-//   warp 8   TMA producer: runs ahead into the next unit's K tiles as soon as ring stages free up
-//   warp 9   MMA issuer: logits of unit j go to half (j & 1) of tensor memory (8 tiles of 32 columns)
-//   warp 10  stages Q and the query-label table of the next unit while the current one is in flight
-//   warps 0-7 epilogue: pass 1 statistics, cluster-wide merge, pass 2 from tensor memory, scores
+//   warp 16  TMA producer: runs ahead into the next unit's K tiles as soon as ring stages free up
+//   warp 17  MMA issuer: logits of unit j go to half (j & 1) of tensor memory (8 tiles of 32 columns)
+//   warp 18  stages Q and the query-label table up to two units ahead (ring of three sets)
+//   warps 0-15 two epilogue teams of 8 warps; team p owns half p of tensor memory and every second
+//            unit: pass 1 statistics, cluster-wide merge, pass 2 from tensor memory, scores.  While one
+//            team waits for its peers' statistics the other one computes.
 // While the epilogue warps finish unit j (statistics exchange, pass 2), the producer and the tensor
 // core already work on unit j + 1 in the other half.  The cluster-wide merge of the row statistics
 // uses an mbarrier per CTA that all CTAs of the cluster arrive on remotely, so only the epilogue
@@ -22,24 +24,33 @@ namespace csp {
 namespace {
 using namespace dev;
 
-// barrier over the 256 epilogue threads that also tells everyone whether any of them saw `pred`
-__device__ __forceinline__ bool consumer_any(bool pred) {
+// barrier over `nthreads` threads (barrier id `id`) that also tells everyone whether any of them saw `pred`
+__device__ __forceinline__ bool barrier_any(bool pred, int id, uint32_t nthreads) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %1, 0;\n\t"
-        "barrier.cta.red.or.pred q, 1, %2, p;\n\t"
+        "barrier.cta.red.or.pred q, %3, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"(uint32_t(pred)), "n"(kConsumerThreads) : "memory");
+        : "=r"(r) : "r"(uint32_t(pred)), "r"(nthreads), "r"(id) : "memory");
     return r != 0;
 }
 
-constexpr int kPsThreads = 352;                         // 8 epilogue warps, producer, MMA issuer, stager
-constexpr int kPsProducerWarp = 8;
-constexpr int kPsMmaWarp = 9;
-constexpr int kPsStageWarp = 10;
+constexpr int kTeams = 2;                               // epilogue teams; team p owns tensor-memory half p
+constexpr int kTeamWarps = 8;                           // two groups of four warps (one per TMEM lane quarter)
+constexpr int kTeamThreads = 32 * kTeamWarps;
+constexpr int kEpiWarps = kTeams * kTeamWarps;
+constexpr int kPsProducerWarp = kEpiWarps;
+constexpr int kPsMmaWarp = kEpiWarps + 1;
+constexpr int kPsStageWarp = kEpiWarps + 2;
+constexpr int kPsThreads = 32 * (kEpiWarps + 3);        // epilogue warps, producer, MMA issuer, stager
+// barrier over the 256 threads of one epilogue team
+__device__ __forceinline__ void team_sync(int team) {
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(kTeamThreads) : "memory");
+}
 constexpr int kHalfBufs = 8;                            // tiles whose logits one half of tensor memory holds
 constexpr int kPsMaxStages = 8;
+constexpr int kQSets = 3;                               // Q tiles and label tables staged ahead (ring)
 
 struct PsSmemPlan {   // byte offsets from the 1024-aligned base
     uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
@@ -47,14 +58,14 @@ struct PsSmemPlan {   // byte offsets from the 1024-aligned base
 __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     PsSmemPlan s;
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
-    s.q = off;        off += 2u * uint32_t(nh) * 32u * 128u;      // two units in flight
-    s.wstats = off;   off += 8u * 32u * 8u;
+    s.q = off;        off += uint32_t(kQSets) * uint32_t(nh) * 32u * 128u;   // staged ahead of the tensor core
+    s.wstats = off;   off += 16u * 32u * 8u;                     // [team][warp][column]
     s.cstats = off;   off += 2u * 32u * 8u;                       // ping-pong, read by the peers
-    s.cvec = off;     off += 32u * 4u;
-    s.dq_mask = off;  off += 2u * 32u * 4u;
-    s.dq_val = off;   off += 2u * 32u * 4u;
-    s.bars = off;     off += (2u * kPsMaxStages + 2u * kHalfBufs + 8u) * 8u;
-    s.misc = off;     off += 32u;     // tmem base, abort flag, n distinct query labels [2]
+    s.cvec = off;     off += 2u * 32u * 4u;                      // per team
+    s.dq_mask = off;  off += uint32_t(kQSets) * 32u * 4u;
+    s.dq_val = off;   off += uint32_t(kQSets) * 32u * 4u;
+    s.bars = off;     off += (2u * kPsMaxStages + 4u * kHalfBufs + 3u * kQSets + 2u) * 8u;
+    s.misc = off;     off += 32u;     // tmem base, abort flag, n distinct query labels [kQSets]
     s.total = off;
     return s;
 }
@@ -81,10 +92,11 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     const uint32_t full_k = base + sp.bars;
     const uint32_t empty_k = full_k + 8 * kPsMaxStages;
     const uint32_t tmem_full = empty_k + 8 * kPsMaxStages;        // [2][8]
-    const uint32_t half_free = tmem_full + 8 * 2 * kHalfBufs;     // [2] epilogue done with the half
-    const uint32_t q_ready = half_free + 16;                      // [2] Q and label table staged
-    const uint32_t q_free = q_ready + 16;                         // [2] tensor core done reading Q
-    const uint32_t stats_ready = q_free + 16;                     // [2] every CTA of the cluster published its statistics
+    const uint32_t tmem_empty = tmem_full + 8 * 2 * kHalfBufs;    // [2][8] pass 2 done with the tile's logits
+    const uint32_t unit_done = tmem_empty + 8 * 2 * kHalfBufs;    // [kQSets] epilogue team done with the unit's label table
+    const uint32_t q_ready = unit_done + 8 * kQSets;              // [kQSets] Q and label table staged
+    const uint32_t q_free = q_ready + 8 * kQSets;                 // [kQSets] tensor core done reading Q
+    const uint32_t stats_ready = q_free + 8 * kQSets;             // [2] every CTA of the cluster published its statistics
     volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + sp.misc);
     volatile int* const abort_flag = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 4);
     volatile int* const n_dq = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 8);   // [2]
@@ -97,13 +109,13 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
-        for (int i = 0; i < 2 * kHalfBufs; ++i) mbar_init(tmem_full + 8 * i, 1);
-        for (int p = 0; p < 2; ++p) {
-            mbar_init(half_free + 8 * p, 8);
-            mbar_init(q_ready + 8 * p, 1);
-            mbar_init(q_free + 8 * p, 1);
-            mbar_init(stats_ready + 8 * p, csize);
+        for (int i = 0; i < 2 * kHalfBufs; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
+        for (int q = 0; q < kQSets; ++q) {
+            mbar_init(unit_done + 8 * q, kTeamWarps);
+            mbar_init(q_ready + 8 * q, 1);
+            mbar_init(q_free + 8 * q, 1);
         }
+        for (int p = 0; p < 2; ++p) mbar_init(stats_ready + 8 * p, csize);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -175,12 +187,15 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const Unit x = unit_of(u);
                 const int p = j & 1;
                 const uint32_t ph = uint32_t(j >> 1) & 1u;
-                mbar_wait(q_ready + 8 * p, ph, abort_flag);             // Q of this unit is in shared memory
-                mbar_wait(half_free + 8 * p, ph ^ 1u, abort_flag);      // the unit two back left this half
-                const uint32_t q_s = base + sp.q + uint32_t(p) * kQBytes;
+                const int qs = j % kQSets;
+                const uint32_t qph = uint32_t(j / kQSets) & 1u;
+                mbar_wait(q_ready + 8 * qs, qph, abort_flag);           // Q of this unit is in shared memory
+                const uint32_t q_s = base + sp.q + uint32_t(qs) * kQBytes;
                 for (int i = 0; i < x.my_all; ++i, ++it) {
                     const int slot = it % n_stages;
                     mbar_wait(full_k + 8 * slot, uint32_t(it / n_stages) & 1u, abort_flag);
+                    // the tile that used this buffer two units back has been through pass 2
+                    mbar_wait(tmem_empty + 8 * (p * kHalfBufs + i), ph ^ 1u, abort_flag);
                     if (*abort_flag) break;
                     tc_fence_after();
                     const uint32_t stage_addr = base + slot * kStageBytes;
@@ -194,8 +209,11 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     tc_commit(tmem_full + 8 * (p * kHalfBufs + i));
                 }
                 // buffers this unit does not use still flip once per unit: one parity rule for all of them
-                for (int i = x.my_all; i < kHalfBufs; ++i) mbar_arrive(tmem_full + 8 * (p * kHalfBufs + i));
-                tc_commit(q_free + 8 * p);
+                for (int i = x.my_all; i < kHalfBufs; ++i) {
+                    mbar_wait(tmem_empty + 8 * (p * kHalfBufs + i), ph ^ 1u, abort_flag);
+                    mbar_arrive(tmem_full + 8 * (p * kHalfBufs + i));
+                }
+                tc_commit(q_free + 8 * qs);
             }
         }
         __syncwarp();
@@ -207,20 +225,28 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             const Unit x = unit_of(u);
             const int p = j & 1;
             const uint32_t ph = uint32_t(j >> 1) & 1u;
-            mbar_wait(q_free + 8 * p, ph ^ 1u, abort_flag);
-            mbar_wait(half_free + 8 * p, ph ^ 1u, abort_flag);
-            uint8_t* const q_dst = base_ptr + sp.q + p * kQBytes;
+            const int qs = j % kQSets;
+            const uint32_t qph = uint32_t(j / kQSets) & 1u;
+            mbar_wait(q_free + 8 * qs, qph ^ 1u, abort_flag);            // tensor core done with the unit 3 back
+            mbar_wait(unit_done + 8 * qs, qph ^ 1u, abort_flag);         // and its epilogue with the label table
+            uint8_t* const q_dst = base_ptr + sp.q + qs * kQBytes;
             const uint8_t* qb = static_cast<const uint8_t*>(a.q);
+            // lane w stages window row w: all its 16-byte chunks are loaded before any is stored, so the
+            // global-memory latency is paid once per unit, not once per chunk
             constexpr int kChunksPerRow = NH * 8;
-            for (int i = lane; i < 32 * kChunksPerRow; i += 32) {
-                const int w = i / kChunksPerRow, c = i % kChunksPerRow;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (w < W && !x.skip) {
-                    const int64_t e = int64_t(x.b) * a.q_sb + int64_t(x.h) * a.q_sh + int64_t(w) * a.q_st;
-                    v = *reinterpret_cast<const uint4*>(qb + e * 2 + c * 16);
+            {
+                const int w = lane;
+                uint4 v[kChunksPerRow];
+                const bool have = w < W && !x.skip;
+                const int64_t e = int64_t(x.b) * a.q_sb + int64_t(x.h) * a.q_sh + int64_t(w) * a.q_st;
+                const uint4* src = reinterpret_cast<const uint4*>(qb + e * 2);
+#pragma unroll
+                for (int c = 0; c < kChunksPerRow; ++c) v[c] = have ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int c = 0; c < kChunksPerRow; ++c) {
+                    const uint32_t off = uint32_t(c >> 3) * (NC * 128) + uint32_t(w) * 128 + (uint32_t((c & 7) ^ (w & 7)) << 4);
+                    *reinterpret_cast<uint4*>(q_dst + off) = v[c];
                 }
-                const uint32_t off = uint32_t(c >> 3) * (NC * 128) + uint32_t(w) * 128 + (uint32_t((c & 7) ^ (w & 7)) << 4);
-                *reinterpret_cast<uint4*>(q_dst + off) = v;
             }
             // table of the distinct labels of the window queries and the columns carrying each
             const uint8_t* modp = a.modality + int64_t(x.b) * a.mod_sb + int64_t(x.h) * a.mod_sh;
@@ -230,30 +256,32 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const uint32_t vj = __shfl_sync(0xffffffffu, ql, jq);
                 const uint32_t same = __ballot_sync(0xffffffffu, ql == vj);
                 if ((same & ((1u << jq) - 1u)) == 0u) {               // no earlier column has this label
-                    if (lane == 0) { dq_val[p * 32 + count] = vj; dq_mask[p * 32 + count] = same; }
+                    if (lane == 0) { dq_val[qs * 32 + count] = vj; dq_mask[qs * 32 + count] = same; }
                     ++count;
                 }
             }
-            if (lane == 0) n_dq[p] = x.skip ? 0 : count;
+            if (lane == 0) n_dq[qs] = x.skip ? 0 : count;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make Q visible to the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(q_ready + 8 * p);
+            if (lane == 0) mbar_arrive(q_ready + 8 * qs);
         }
     } else {
         // =============================== epilogue warps ===============================
-        const int quarter = warp & 3, group = warp >> 2;
+        const int team = warp / kTeamWarps, tw = warp % kTeamWarps;   // team-local warp index
+        const int quarter = tw & 3, group = tw >> 2;
         const int lq = lane & 3, lr = lane >> 2;
         const float scale2 = a.scale_log2;
         const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
-        int j = 0;
-        for (int u = cid; u < n_units; u += n_clusters, ++j) {
-            if (consumer_any(*abort_flag != 0)) break;                   // all 256 threads leave together
+        float2* const wst = wstats + team * (kTeamWarps * 32);
+        float* const cv_team = cvec + team * 32;
+        for (int j = team, u = cid + team * n_clusters; u < n_units; u += kTeams * n_clusters, j += kTeams) {
+            if (barrier_any(*abort_flag != 0, 1 + team, kTeamThreads)) break;   // the whole team leaves together
             const Unit x = unit_of(u);
             const int p = j & 1;
             const uint32_t ph = uint32_t(j >> 1) & 1u;
             const int first_masked_key = x.L - W;
             const uint8_t* modp = a.modality + int64_t(x.b) * a.mod_sb + int64_t(x.h) * a.mod_sh;
-            if (tid == 0 && rank == 0) {
+            if (tw == 0 && lane == 0 && rank == 0) {
                 const int Lraw = a.seq_lens[x.b];
                 if (Lraw < 0 || Lraw > a.max_len) atomicOr(a.status, CSP_DEV_BAD_LEN);
             }
@@ -311,48 +339,61 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     const float oz = __shfl_xor_sync(0xffffffffu, z_run[jj], d);
                     merge_stats(m_run[jj], z_run[jj], om, oz);
                 }
-                if (lr == 0) wstats[warp * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
+                if (lr == 0) wst[tw * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
             }
-            consumer_sync();
-            if (warp == 0) {
-                float m = kNeg, z = 0.f;
+            team_sync(team);
+            if (tw == 0) {
+                float2 v[kTeamWarps];
 #pragma unroll
-                for (int w = 0; w < 8; ++w) {
-                    const float2 s = wstats[w * 32 + lane];
-                    merge_stats(m, z, s.x, s.y);
-                }
-                cstats[p * 32 + lane] = make_float2(m, z);
+                for (int w = 0; w < kTeamWarps; ++w) v[w] = wst[w * 32 + lane];
+#pragma unroll
+                for (int d = 1; d < kTeamWarps; d <<= 1)                  // pairwise tree, fixed order
+#pragma unroll
+                    for (int w = 0; w < kTeamWarps; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
+                cstats[p * 32 + lane] = v[0];
                 __syncwarp();
                 asm volatile("fence.acq_rel.cluster;" ::: "memory");
                 if (lane < int(csize)) mbar_arrive_remote(stats_ready + 8 * p, uint32_t(lane));   // publish to every CTA
             }
             mbar_wait_cluster(stats_ready + 8 * p, ph, abort_flag);
-            if (warp == 0) {
-                float m = kNeg, z = 0.f;
-                for (uint32_t r = 0; r < csize; ++r) {
-                    const float2 s = ld_remote_f2(smem_u32(&cstats[p * 32 + lane]), r);
-                    merge_stats(m, z, s.x, s.y);
-                }
+            if (tw == 0) {
+                float2 v[8];
+#pragma unroll
+                for (uint32_t r = 0; r < 8; ++r)                           // loads first, then one merge chain
+                    v[r] = r < csize ? ld_remote_f2(smem_u32(&cstats[p * 32 + lane]), r) : make_float2(kNeg, 0.f);
+#pragma unroll
+                for (int d = 1; d < 8; d <<= 1)
+#pragma unroll
+                    for (int w = 0; w < 8; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
+                const float m = v[0].x, z = v[0].y;
                 // weight of 2^(x - m) is 1 / (n 2^-m + Z); fold it and -m into one additive constant
                 const float denom = a.n * ex2f(-m) + z;
-                cvec[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
+                cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
             }
-            mbar_wait(q_ready + 8 * p, ph, abort_flag);                  // label table of this unit
-            consumer_sync();
+            const int qs = j % kQSets;
+            mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
+            team_sync(team);
 
             // ---------------------------------- pass 2 ----------------------------------
             float* const out_s = a.score_self + (int64_t(x.b) * a.n_kv_heads + x.h) * a.max_len;
             float* const out_c = a.score_cross + (int64_t(x.b) * a.n_kv_heads + x.h) * a.max_len;
-            const int ndq = n_dq[p];
+            const int ndq = n_dq[qs];
             auto t_of = [&](int i) { return (i * int(csize) + int(rank)) * kTileKeys + quarter * 32 + lane; };
             uint32_t kmod_next = (group < x.my_cand && t_of(group) < x.N) ? modp[t_of(group)] : 0u;
-            for (int i = group; i < x.my_cand; i += 2) {
+            for (int i = group; i < kHalfBufs; i += 2) {
                 const int buf = p * kHalfBufs + i;
+                if (i >= x.my_cand) {                                    // nothing to score: just hand the buffer back
+                    if (i >= x.my_all) mbar_wait(tmem_full + 8 * buf, ph, abort_flag);   // keep phases in step
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
+                    continue;
+                }
                 const int t = t_of(i);
                 const uint32_t kmod = kmod_next;
                 kmod_next = (i + 2 < x.my_cand && t_of(i + 2) < x.N) ? modp[t_of(i + 2)] : 0u;
                 uint32_t same = 0u;                                        // window columns with the key's label
-                for (int q = 0; q < ndq; ++q) same = dq_val[p * 32 + q] == kmod ? dq_mask[p * 32 + q] : same;
+                for (int q = 0; q < ndq; ++q) same = dq_val[qs * 32 + q] == kmod ? dq_mask[qs * 32 + q] : same;
                 const int delta = t - first_masked_key;                    // column w sees the key iff w >= delta
                 const uint32_t vis = delta <= 0 ? wmask : (delta >= 32 ? 0u : (wmask & (0xFFFFFFFFu << delta)));
                 const uint32_t add_s = same & vis, add_c = ~same & vis;
@@ -365,7 +406,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     tc_wait_ld();
                     uint32_t (&cur)[16] = ch ? vb : va;
                     if (ch == 0) tc_ld_row16(vb, row_addr + 16u);
-                    const float4* cv = reinterpret_cast<const float4*>(cvec + ch * 16);
+                    const float4* cv = reinterpret_cast<const float4*>(cv_team + ch * 16);
                     const uint32_t as = add_s >> (ch * 16), ac = add_c >> (ch * 16);
 #pragma unroll
                     for (int j4 = 0; j4 < 4; ++j4) {
@@ -380,14 +421,16 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                         s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);          // the tensor core may refill this buffer
                 if (t < x.N) { out_s[t] = s0 + s1; out_c[t] = c0 + c1; }
             }
-            // this half of tensor memory, the label table and Q of this parity may now be reused
-            tc_fence_before();
+            // the label table and Q of this parity may now be restaged
             __syncwarp();
-            if (lane == 0) mbar_arrive(half_free + 8 * p);
+            if (lane == 0) mbar_arrive(unit_done + 8 * qs);
         }
-        if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
+        if (*abort_flag && tw == 0 && lane == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
     }
 
     // every warp: give tensor memory back, then keep shared memory alive until the peers are done
