@@ -60,7 +60,7 @@ __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
     s.q = off;        off += uint32_t(kQSets) * uint32_t(nh) * 32u * 128u;   // staged ahead of the tensor core
     s.wstats = off;   off += 16u * 32u * 8u;                     // [team][warp][column]
-    s.cstats = off;   off += 2u * 32u * 8u;                       // ping-pong, read by the peers
+    s.cstats = off;   off += 4u * 8u * 32u * 8u;                  // [unit & 3][rank][row], written by the peers
     s.cvec = off;     off += 2u * 32u * 4u;                      // per team
     s.dq_mask = off;  off += uint32_t(kQSets) * 32u * 4u;
     s.dq_val = off;   off += uint32_t(kQSets) * 32u * 4u;
@@ -342,7 +342,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 if (lr == 0) wst[tw * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
             }
             team_sync(team);
+            const int qs = j % kQSets;
             if (tw == 0) {
+                // lane l owns window row l: merge the team's warps, push the result into every peer's
+                // shared memory (slot [p][my rank][l]) and tell the peer; then wait for all peers' pushes
                 float2 v[kTeamWarps];
 #pragma unroll
                 for (int w = 0; w < kTeamWarps; ++w) v[w] = wst[w * 32 + lane];
@@ -350,28 +353,27 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 for (int d = 1; d < kTeamWarps; d <<= 1)                  // pairwise tree, fixed order
 #pragma unroll
                     for (int w = 0; w < kTeamWarps; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
-                cstats[p * 32 + lane] = v[0];
-                __syncwarp();
+                const int slot4 = j & 3;   // a peer can only overwrite a slot four units later, after this CTA's arrive for j + 2
+                const uint32_t mine = smem_u32(&cstats[(slot4 * 8 + int(rank)) * 32 + lane]);
+                for (uint32_t r = 0; r < csize; ++r) st_remote_f2(mine, r, v[0]);
                 asm volatile("fence.acq_rel.cluster;" ::: "memory");
-                if (lane < int(csize)) mbar_arrive_remote(stats_ready + 8 * p, uint32_t(lane));   // publish to every CTA
-            }
-            mbar_wait_cluster(stats_ready + 8 * p, ph, abort_flag);
-            if (tw == 0) {
-                float2 v[8];
+                __syncwarp();
+                if (lane < int(csize)) mbar_arrive_remote(stats_ready + 8 * p, uint32_t(lane));
+                mbar_wait_cluster(stats_ready + 8 * p, ph, abort_flag);
+                float2 c8[8];
 #pragma unroll
-                for (uint32_t r = 0; r < 8; ++r)                           // loads first, then one merge chain
-                    v[r] = r < csize ? ld_remote_f2(smem_u32(&cstats[p * 32 + lane]), r) : make_float2(kNeg, 0.f);
+                for (int r = 0; r < 8; ++r)
+                    c8[r] = r < int(csize) ? cstats[(slot4 * 8 + r) * 32 + lane] : make_float2(kNeg, 0.f);
 #pragma unroll
                 for (int d = 1; d < 8; d <<= 1)
 #pragma unroll
-                    for (int w = 0; w < 8; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
-                const float m = v[0].x, z = v[0].y;
+                    for (int w = 0; w < 8; w += 2 * d) merge_stats(c8[w].x, c8[w].y, c8[w + d].x, c8[w + d].y);
+                const float m = c8[0].x, z = c8[0].y;
                 // weight of 2^(x - m) is 1 / (n 2^-m + Z); fold it and -m into one additive constant
                 const float denom = a.n * ex2f(-m) + z;
                 cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
+                mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
             }
-            const int qs = j % kQSets;
-            mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
             team_sync(team);
 
             // ---------------------------------- pass 2 ----------------------------------

@@ -1,7 +1,7 @@
 // Selection kernel for caches up to 65536 positions: the two top-K masks (Eq. 2), their combination
 // (Eq. 3) and the ascending list of kept positions followed by the recent block (index side of Eq. 4).
 //
-// A cluster of 1-8 CTAs (512 or 1024 threads) owns one (sequence, KV head) unit.  Every thread keeps E (4
+// A cluster of 1-8 CTAs (1024 threads) owns one (sequence, KV head) unit.  Every thread keeps E (4
 // or 8) of the unit's keys in registers for the whole kernel (the order-preserving integer images of
 // both scores plus a label bit); a warp covers 32 E consecutive positions, lane l holding positions
 // base + 32 e + l, so loads are coalesced and "position order" inside a warp is (e, lane) order,
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Sel
                 }
 #pragma unroll
                 for (int iter = 0; iter < 2; ++iter) {
-                    if (todo == 0u) break;
+                    if (__all_sync(kFull, todo == 0u)) break;           // whole warp done
                     uint32_t first = 0u;
                     bool have = false;
 #pragma unroll
@@ -171,7 +171,17 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Sel
 #pragma unroll
                     for (int e = 0; e < E; ++e)
                         if (((todo >> e) & 1u) && slot[e] == first) same |= 1u << e;
-                    atomicAdd(&hb[first], uint32_t(__popc(same)));
+                    // neighbouring positions mostly share the slot: when the whole warp agrees, one lane adds
+                    // the warp's total instead of 32 lanes hitting the same shared-memory word
+                    const uint32_t cnt = uint32_t(__popc(same));
+                    const uint32_t voters = __ballot_sync(kFull, todo != 0u);
+                    const uint32_t f0 = __shfl_sync(kFull, first, voters ? __ffs(voters) - 1 : 0);
+                    if (__all_sync(kFull, todo == 0u || first == f0)) {
+                        const uint32_t total = __reduce_add_sync(kFull, cnt);
+                        if (lane == 0 && total) atomicAdd(&hb[f0], total);
+                    } else if (todo != 0u) {
+                        atomicAdd(&hb[first], cnt);
+                    }
                     todo &= ~same;
                 }
                 if (todo != 0u) {
@@ -348,15 +358,12 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     if (units > 65535) return CSP_ERR_UNSUPPORTED;
-    // A CTA covers 4096 keys (8192 for caches above 32768 positions).  With few units the kernel is
-    // latency-bound: 1024 threads x 4 keys, many warps with little code each.  With many units it is
-    // throughput-bound: 512 threads x 8 keys, two CTAs per SM overlapping each other's barriers.
+    // A CTA of 1024 threads covers 4096 keys (8192 for caches above 32768 positions): many warps with
+    // little code each hide the latencies of the short dependent phases.
     const int per_cta = p.max_len <= 8 * 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
-    if (per_cta == 8192) return launch_e<1024, 8>(p, a, cs, s);
-    if (units * cs >= 2 * 148) return launch_e<512, 8>(p, a, cs, s);
-    return launch_e<1024, 4>(p, a, cs, s);
+    return per_cta == 8192 ? launch_e<1024, 8>(p, a, cs, s) : launch_e<1024, 4>(p, a, cs, s);
 }
 
 }  // namespace csp
