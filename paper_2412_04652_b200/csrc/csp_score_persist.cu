@@ -5,17 +5,18 @@
 // CTAs stays resident and walks over units cluster_id, cluster_id + n_clusters, ...  The roles of a
 // CTA are decoupled by mbarriers so that the K stream never stops between units:
 //   warp 16  TMA producer: runs ahead into the next unit's K tiles as soon as ring stages free up
-//   warp 17  MMA issuer: logits of unit j go to half (j & 1) of tensor memory (8 tiles of 32 columns)
+//   warp 17  MMA issuer: tile i of every unit uses accumulator buffer i of tensor memory (16 buffers of 32
+//            columns); it is refilled as soon as pass 2 of the previous unit has read it
 //   warp 18  stages Q and the query-label table up to two units ahead (ring of three sets)
-//   warps 0-15 two epilogue teams of 8 warps; team p owns half p of tensor memory and every second
-//            unit: pass 1 statistics, cluster-wide merge, pass 2 from tensor memory, scores.  While one
+//   warps 0-15 two epilogue teams of 8 warps; team j & 1 takes unit j: pass 1 statistics, cluster-wide
+//            merge, pass 2 from tensor memory, scores.  While one
 //            team waits for its peers' statistics the other one computes.
-// While the epilogue warps finish unit j (statistics exchange, pass 2), the producer and the tensor
-// core already work on unit j + 1 in the other half.  The cluster-wide merge of the row statistics
+// While one epilogue team finishes unit j (statistics exchange, pass 2), the producer, the tensor core
+// and the other team already work on unit j + 1 in the buffers that pass 2 has released.  The cluster-wide merge of the row statistics
 // uses an mbarrier per CTA that all CTAs of the cluster arrive on remotely, so only the epilogue
 // warps take part and nobody else is held up.  Every wait is bounded.
 //
-// Precondition (checked by the launcher): G = 1, no caller-supplied LSE, and at most 8 tiles per CTA,
+// Precondition (checked by the launcher): G = 1, no caller-supplied LSE, and at most 16 tiles per CTA,
 // so that every tile's logits stay in tensor memory between the passes.
 #include "csp_internal.cuh"
 #include "csp_tc.cuh"
@@ -48,7 +49,7 @@ constexpr int kPsThreads = 32 * (kEpiWarps + 3);        // epilogue warps, produ
 __device__ __forceinline__ void team_sync(int team) {
     asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(kTeamThreads) : "memory");
 }
-constexpr int kHalfBufs = 8;                            // tiles whose logits one half of tensor memory holds
+constexpr int kBufs = 16;                               // tiles whose logits tensor memory holds (32 columns each)
 constexpr int kPsMaxStages = 8;
 constexpr int kQSets = 3;                               // Q tiles and label tables staged ahead (ring)
 
@@ -64,7 +65,7 @@ __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     s.cvec = off;     off += 2u * 32u * 4u;                      // per team
     s.dq_mask = off;  off += uint32_t(kQSets) * 32u * 4u;
     s.dq_val = off;   off += uint32_t(kQSets) * 32u * 4u;
-    s.bars = off;     off += (2u * kPsMaxStages + 4u * kHalfBufs + 3u * kQSets + 2u) * 8u;
+    s.bars = off;     off += (2u * kPsMaxStages + 3u * kBufs + 3u * kQSets + 2u) * 8u;
     s.misc = off;     off += 32u;     // tmem base, abort flag, n distinct query labels [kQSets]
     s.total = off;
     return s;
@@ -91,9 +92,11 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     uint32_t* const dq_val = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_val);
     const uint32_t full_k = base + sp.bars;
     const uint32_t empty_k = full_k + 8 * kPsMaxStages;
-    const uint32_t tmem_full = empty_k + 8 * kPsMaxStages;        // [2][8]
-    const uint32_t tmem_empty = tmem_full + 8 * 2 * kHalfBufs;    // [2][8] pass 2 done with the tile's logits
-    const uint32_t unit_done = tmem_empty + 8 * 2 * kHalfBufs;    // [kQSets] epilogue team done with the unit's label table
+    // logits of tile i ready, one barrier set per epilogue team (= unit parity): a team only ever waits
+    // on its own set, one phase per unit it handles, so a parity bit identifies the phase
+    const uint32_t tmem_full = empty_k + 8 * kPsMaxStages;        // [2][16]
+    const uint32_t tmem_empty = tmem_full + 8 * 2 * kBufs;        // [16] pass 2 done with the tile's logits
+    const uint32_t unit_done = tmem_empty + 8 * kBufs;    // [kQSets] epilogue team done with the unit's label table
     const uint32_t q_ready = unit_done + 8 * kQSets;              // [kQSets] Q and label table staged
     const uint32_t q_free = q_ready + 8 * kQSets;                 // [kQSets] tensor core done reading Q
     const uint32_t stats_ready = q_free + 8 * kQSets;             // [2] every CTA of the cluster published its statistics
@@ -109,7 +112,11 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
-        for (int i = 0; i < 2 * kHalfBufs; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
+        for (int i = 0; i < kBufs; ++i) {
+            mbar_init(tmem_full + 8 * i, 1);
+            mbar_init(tmem_full + 8 * (kBufs + i), 1);
+            mbar_init(tmem_empty + 8 * i, 4);
+        }
         for (int q = 0; q < kQSets; ++q) {
             mbar_init(unit_done + 8 * q, kTeamWarps);
             mbar_init(q_ready + 8 * q, 1);
@@ -145,7 +152,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
         const int tiles_all = (L + kTileKeys - 1) / kTileKeys, tiles_cand = (x.N + kTileKeys - 1) / kTileKeys;
         x.my_all = tiles_all > int(rank) ? (tiles_all - int(rank) + int(csize) - 1) / int(csize) : 0;
         x.my_cand = tiles_cand > int(rank) ? (tiles_cand - int(rank) + int(csize) - 1) / int(csize) : 0;
-        if (x.my_all > kHalfBufs) x.my_all = kHalfBufs;          // never happens (launcher); keeps indices in range
+        if (x.my_all > kBufs) x.my_all = kBufs;          // never happens (launcher); keeps indices in range
         if (x.my_cand > x.my_all) x.my_cand = x.my_all;
         return x;
     };
@@ -185,8 +192,8 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             int it = 0, j = 0;
             for (int u = cid; u < n_units && !*abort_flag; u += n_clusters, ++j) {
                 const Unit x = unit_of(u);
-                const int p = j & 1;
-                const uint32_t ph = uint32_t(j >> 1) & 1u;
+                const uint32_t bph = uint32_t(j) & 1u;                  // every buffer is released once per unit
+                const uint32_t my_full = tmem_full + 8 * kBufs * (j & 1);   // barrier set of the team that takes unit j
                 const int qs = j % kQSets;
                 const uint32_t qph = uint32_t(j / kQSets) & 1u;
                 mbar_wait(q_ready + 8 * qs, qph, abort_flag);           // Q of this unit is in shared memory
@@ -195,7 +202,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     const int slot = it % n_stages;
                     mbar_wait(full_k + 8 * slot, uint32_t(it / n_stages) & 1u, abort_flag);
                     // the tile that used this buffer two units back has been through pass 2
-                    mbar_wait(tmem_empty + 8 * (p * kHalfBufs + i), ph ^ 1u, abort_flag);
+                    mbar_wait(tmem_empty + 8 * i, bph ^ 1u, abort_flag);
                     if (*abort_flag) break;
                     tc_fence_after();
                     const uint32_t stage_addr = base + slot * kStageBytes;
@@ -203,15 +210,15 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     for (int ks = 0; ks < KS; ++ks) {
                         const uint64_t ad = sw128_desc(stage_addr + uint32_t(ks >> 2) * kBlockBytes + uint32_t(ks & 3) * 32u);
                         const uint64_t bd = sw128_desc(q_s + uint32_t(ks >> 2) * (NC * 128u) + uint32_t(ks & 3) * 32u);
-                        tc_mma_bf16(tmem_base + uint32_t((p * kHalfBufs + i) * NC), ad, bd, kIdesc, ks > 0 ? 1u : 0u);
+                        tc_mma_bf16(tmem_base + uint32_t(i * NC), ad, bd, kIdesc, ks > 0 ? 1u : 0u);
                     }
                     tc_commit(empty_k + 8 * slot);
-                    tc_commit(tmem_full + 8 * (p * kHalfBufs + i));
+                    tc_commit(my_full + 8 * i);
                 }
                 // buffers this unit does not use still flip once per unit: one parity rule for all of them
-                for (int i = x.my_all; i < kHalfBufs; ++i) {
-                    mbar_wait(tmem_empty + 8 * (p * kHalfBufs + i), ph ^ 1u, abort_flag);
-                    mbar_arrive(tmem_full + 8 * (p * kHalfBufs + i));
+                for (int i = x.my_all; i < kBufs; ++i) {
+                    mbar_wait(tmem_empty + 8 * i, bph ^ 1u, abort_flag);
+                    mbar_arrive(my_full + 8 * i);
                 }
                 tc_commit(q_free + 8 * qs);
             }
@@ -223,8 +230,6 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
         for (int u = cid; u < n_units; u += n_clusters, ++j) {
             if (__any_sync(0xffffffffu, *abort_flag != 0)) break;        // the whole warp leaves together
             const Unit x = unit_of(u);
-            const int p = j & 1;
-            const uint32_t ph = uint32_t(j >> 1) & 1u;
             const int qs = j % kQSets;
             const uint32_t qph = uint32_t(j / kQSets) & 1u;
             mbar_wait(q_free + 8 * qs, qph ^ 1u, abort_flag);            // tensor core done with the unit 3 back
@@ -279,6 +284,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             const Unit x = unit_of(u);
             const int p = j & 1;
             const uint32_t ph = uint32_t(j >> 1) & 1u;
+            const uint32_t my_full = tmem_full + 8 * kBufs * team;   // this team's barrier set; one phase per unit it takes
             const int first_masked_key = x.L - W;
             const uint8_t* modp = a.modality + int64_t(x.b) * a.mod_sb + int64_t(x.h) * a.mod_sh;
             if (tw == 0 && lane == 0 && rank == 0) {
@@ -291,9 +297,9 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) { m_run[jj] = kNeg; z_run[jj] = 0.f; }
             for (int i = group; i < x.my_all; i += 2) {
-                const int buf = p * kHalfBufs + i;
+                const int buf = i;
                 const int tile = i * int(csize) + int(rank);
-                mbar_wait(tmem_full + 8 * buf, ph, abort_flag);
+                mbar_wait(my_full + 8 * buf, ph, abort_flag);
                 tc_fence_after();
                 const bool masked = (tile + 1) * kTileKeys > first_masked_key;
                 const int t_base = tile * kTileKeys + quarter * 32 + lr;
@@ -382,10 +388,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             const int ndq = n_dq[qs];
             auto t_of = [&](int i) { return (i * int(csize) + int(rank)) * kTileKeys + quarter * 32 + lane; };
             uint32_t kmod_next = (group < x.my_cand && t_of(group) < x.N) ? modp[t_of(group)] : 0u;
-            for (int i = group; i < kHalfBufs; i += 2) {
-                const int buf = p * kHalfBufs + i;
+            for (int i = group; i < kBufs; i += 2) {
+                const int buf = i;
                 if (i >= x.my_cand) {                                    // nothing to score: just hand the buffer back
-                    if (i >= x.my_all) mbar_wait(tmem_full + 8 * buf, ph, abort_flag);   // keep phases in step
+                    if (i >= x.my_all) mbar_wait(my_full + 8 * buf, ph, abort_flag);     // keep phases in step
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
@@ -504,8 +510,8 @@ csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const C
     if (row_bytes != 128 && row_bytes != 256) return CSP_OK;
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
     int c = 1;
-    while (c < 8 && (max_tiles + c - 1) / c > kHalfBufs) c *= 2;
-    if ((max_tiles + c - 1) / c > kHalfBufs) return CSP_OK;
+    while (c < 8 && (max_tiles + c - 1) / c > kBufs) c *= 2;
+    if ((max_tiles + c - 1) / c > kBufs) return CSP_OK;
     return row_bytes == 128 ? launch_nh<1>(p, a, tmap, c, s, taken) : launch_nh<2>(p, a, tmap, c, s, taken);
 }
 
