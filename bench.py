@@ -204,8 +204,11 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"])
     ap.add_argument("--streams", type=int, default=32, help="concurrent layer chains inside the step graph")
-    ap.add_argument("--fold-layers", action="store_true",
-                    help="one call for all layers: the layer axis of a [layers*B, H, L, d] cache is passed as batch")
+    ap.add_argument("--per-layer-calls", dest="fold_layers", action="store_false",
+                    help="one csp_prune_layer call per layer (concurrent chains in a CUDA graph) instead of the "
+                         "default: one call for all layers, the layer axis of a [layers*B, H, L, d] cache "
+                         "passed as the batch axis")
+    ap.set_defaults(fold_layers=True)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-baseline-units", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -246,6 +249,11 @@ def main():
     sum_l = int(cfg.seq_lens.sum())
 
     # One entry per library call of a step: (params, buffers, labels, lengths, budgets, totals, layers covered)
+    kv_bytes = 2 * n_layers * cfg.batch * cfg.n_kv_heads * cfg.max_len * cfg.head_dim * (2 if cfg.dtype == torch.bfloat16 else 4)
+    if args.fold_layers and (args.layers > 0 or kv_bytes > 40e9):
+        args.fold_layers = False                     # a subset of layer buffers only makes sense per layer
+        if args.layers <= 0 and kv_bytes > 40e9:
+            n_buf = 4                                 # cycle four distinct layers when the cache is huge
     if args.fold_layers:
         import copy
         pf = copy.copy(p)
@@ -383,10 +391,22 @@ def main():
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) ----
     e2e = None
-    if args.e2e_steps > 0 and not args.fold_layers:
+    if args.e2e_steps > 0:
         n_host = min(n_buf, 4)
         pin = lambda t: t.cpu().contiguous().pin_memory()
         host = []
+        if args.fold_layers:      # the host-buffer entry point is called per layer: slice the folded cache
+            B0 = cfg.batch
+            fl = calls[0][1]
+
+            class _View:
+                pass
+            layers = []
+            for i in range(n_host):
+                lv = _View()
+                for name in ("q", "k", "v", "k_out", "v_out", "mod_out", "n_out"):
+                    setattr(lv, name, getattr(fl, name)[i * B0:(i + 1) * B0])
+                layers.append(lv)
         for i in range(n_host):
             lb = layers[i]
             host.append(dict(q=pin(lb.q), k=pin(lb.k), v=pin(lb.v), k_out=pin(lb.k_out), v_out=pin(lb.v_out),
