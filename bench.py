@@ -112,7 +112,10 @@ def job_throughput(world: int, tokens_per_layer: int, n_layers: int, ms_step: fl
 # DRAM bytes (read + write) per launch of each kernel on configs[1], one layer per launch, from the ncu
 # captures summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  Scales with the
 # number of layers a launch covers.  None for workloads that were not captured.
-NCU_DRAM_BYTES_PER_LAYER = {1: {"score": 33.88e6, "select": 1.08e6, "compact": 16.97e6}}
+NCU_DRAM_BYTES_PER_LAYER = {
+    ("all_layers_one_call", 1): {"score": 1.1145e9 / 32, "select": 33.46e6 / 32, "compact": 1.0238e9 / 32},
+    ("one_layer_per_call", 1): {"score": 33.88e6, "select": 1.08e6, "compact": 16.97e6},
+}
 
 
 def algorithmic_bytes(cfg, n_out_total: int):
@@ -378,7 +381,8 @@ def main():
     ab_launch = {k_: v_ * layers_per_launch for k_, v_ in ab.items()}
     dominant = max(per, key=per.get)
     achieved = ab_launch[dominant] / (per[dominant] * 1e-3) / 1e9
-    traffic = NCU_DRAM_BYTES_PER_LAYER.get(args.config, {}).get(dominant)
+    traffic = NCU_DRAM_BYTES_PER_LAYER.get(("all_layers_one_call" if args.fold_layers else "one_layer_per_call",
+                                            args.config), {}).get(dominant)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": None if traffic is None else traffic * layers_per_launch,
                 "peak_kind": f"of {peak_kind}",
