@@ -77,7 +77,13 @@ def lib() -> C.CDLL:
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2412_04652_b200.build`")
+            # not built yet (fresh checkout): compile in-tree now; there is no other implementation to fall
+            # back to, so a failed build is an import error
+            try:
+                from . import build as _build
+                _build.build()
+            except Exception as exc:  # noqa: BLE001
+                raise ImportError(f"{LIB_PATH} is missing and could not be built with nvcc: {exc}") from exc
         l = C.CDLL(LIB_PATH)
         P = C.POINTER(CParams)
         vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
