@@ -244,6 +244,12 @@ def test_select_long_sequence(csp, oracle):
     _select_case(csp, oracle, 1, 1, (32768,), 32, [[1626, 3, 9, 4301]], quantise=64, seed=8)
 
 
+def test_select_cache_longer_than_cluster_limit(csp, oracle):
+    """Above 65536 positions the one-CTA-per-unit kernel takes over (keys partly staged in shared memory)."""
+    _select_case(csp, oracle, 1, 2, (70001,), 32, [[3000, 11, 0, 9000]], seed=10)
+    _select_case(csp, oracle, 1, 1, (66000,), 32, [[500, 500, 500, 500]], quantise=32, seed=11)
+
+
 def test_select_negative_and_signed_zero_scores(csp, oracle):
     rng = np.random.RandomState(9)
     s = rng.randn(1, 1, 700).astype(np.float32)
@@ -472,3 +478,59 @@ def test_reprune_round_with_per_head_labels(csp, oracle):
     assert_scores_close(run2.sc.cpu().numpy(), ref2["score_cross"], [L2], 32)
     assert_index_sets_match(run2.idx.cpu().numpy(), run2.n_out.cpu().numpy(), ref2, mod2.cpu().numpy(), [L2], 32)
     assert_compaction_exact(run2, mod2.cpu().numpy())
+
+
+@pytest.mark.parametrize("budget_pct", [5, 40])
+def test_config4_reprune_rounds(csp, oracle, budget_pct):
+    """Batched serving shape: prune the prompt cache (round 0), then four times append 64 decode tokens to
+    every head's compacted cache and prune back to the same budget (labels now differ per head).
+    Sampled units are checked against the oracle in every round; structure is checked for all units."""
+    cfg = synth.config(4, budget_pct=budget_pct)
+    R, W, d, H = cfg.recent, cfg.window, cfg.head_dim, cfg.n_kv_heads
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    mod = cfg.modality()
+    run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod, cfg.seq_lens, cfg.budgets,
+                 total_budget=cfg.total_budget).prune()
+    assert run.status() & ~csp.DEV_K_CLAMPED == 0
+    rng = np.random.RandomState(budget_pct)
+    gen = torch.Generator(device="cuda").manual_seed(100 + budget_pct)
+    totals = cfg.total_budget.astype(np.int64)
+    budgets = np.array([synth.budgets_from_total(int(t), R) for t in totals], np.int32)
+    for rnd in range(1, 5):
+        n_prev = run.n_out.cpu().numpy()                      # [B, H] rows each head kept
+        assert (n_prev > 0).all()
+        lens2 = (n_prev.max(axis=1) + 64).astype(np.int32)     # heads of a sequence may differ: pad to the longest
+        Lm = int(lens2.max())
+        B = cfg.batch
+        k2 = torch.zeros(B, H, Lm, d, dtype=torch.bfloat16, device="cuda")
+        v2 = torch.zeros_like(k2)
+        mod2 = torch.zeros(B, H, Lm, dtype=torch.uint8, device="cuda")
+        new_k = torch.randn(B, H, 64, d, device="cuda", generator=gen).to(torch.bfloat16)
+        new_v = torch.randn(B, H, 64, d, device="cuda", generator=gen).to(torch.bfloat16)
+        same_len = (n_prev == n_prev[:, :1]).all()
+        assert same_len, "segmented budgets with disjoint supports keep the same number of rows in every head"
+        for b in range(B):
+            n = int(n_prev[b, 0])
+            k2[b, :, :n] = run.k_out[b, :, :n]
+            v2[b, :, :n] = run.v_out[b, :, :n]
+            mod2[b, :, :n] = run.mod_out[b, :, :n]
+            k2[b, :, n:n + 64] = new_k[b]
+            v2[b, :, n:n + 64] = new_v[b]                    # appended decode tokens are text (label 0)
+        q2 = torch.randn(B, cfg.n_q_heads, W, d, device="cuda", generator=gen).to(torch.bfloat16)
+        cap = int((budgets.sum(axis=1) + R).max())
+        p2 = csp.Params(B, cfg.n_q_heads, H, d, W, R, Lm, cap)
+        run = GpuRun(csp, p2, q2, k2, v2, mod2.cpu().numpy(), lens2, budgets, total_budget=totals.astype(np.int32))
+        run.prune()
+        assert run.status() & ~csp.DEV_K_CLAMPED == 0
+        assert_compaction_exact(run, mod2.cpu().numpy())
+        for _ in range(3):
+            b, h = int(rng.randint(B)), int(rng.randint(H))
+            L = int(lens2[b])
+            op = oracle.Params(1, 1, 1, d, W, R, L, cap)
+            ref = oracle.prune_layer(op, q2[b:b + 1, h:h + 1].cpu(), k2[b:b + 1, h:h + 1, :L].cpu(),
+                                     v2[b:b + 1, h:h + 1, :L].cpu(), mod2[b:b + 1, h:h + 1, :L].cpu().numpy(),
+                                     np.array([L], np.int32), budgets[b:b + 1], totals[b:b + 1].astype(np.int32))
+            assert_scores_close(run.ss[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_self"], [L], R)
+            assert_scores_close(run.sc[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], R)
+            assert_index_sets_match(run.idx[b:b + 1, h:h + 1].cpu().numpy(), run.n_out[b:b + 1, h:h + 1].cpu().numpy(),
+                                    ref, mod2[b:b + 1, h:h + 1, :L].cpu().numpy(), [L], R)
