@@ -370,13 +370,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
             uint32_t va[16], vb[16];
             tc_ld_row16(va, row_addr);
-#pragma unroll
-            for (int ch = 0; ch < 2 * G; ++ch) {
-                tc_wait_ld();
-                uint32_t (&cur)[16] = (ch & 1) ? vb : va;
-                if (ch + 1 < 2 * G) tc_ld_row16((ch & 1) ? va : vb, row_addr + uint32_t((ch + 1) * 16));
-                const float4* cv = reinterpret_cast<const float4*>(cvec + ch * 16);
-                const uint32_t as = add_s >> ((ch & 1) * 16), ac = add_c >> ((ch & 1) * 16);
+            // weights of 16 columns: cur = logits, cv = their additive constants, as/ac = which columns count
+            auto chunk = [&](const uint32_t (&cur)[16], const float* cvp, uint32_t as, uint32_t ac) {
+                const float4* cv = reinterpret_cast<const float4*>(cvp);
 #pragma unroll
                 for (int j4 = 0; j4 < 4; ++j4) {
                     const float4 cc = cv[j4];
@@ -389,6 +385,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                     s0 += (as >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c0 += (ac >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
                     s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                 }
+            };
+            // one query head per iteration, kept as a real loop for G > 2 so that the code stays small
+#pragma unroll(G <= 2 ? G : 1)
+            for (int g = 0; g < G; ++g) {
+                tc_wait_ld();
+                tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
+                chunk(va, cvec + g * 32, add_s, add_c);
+                tc_wait_ld();
+                if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
+                chunk(vb, cvec + g * 32 + 16, add_s >> 16, add_c >> 16);
             }
             const float s = s0 + s1, c = c0 + c1;
             if (i >= kept) {
