@@ -34,7 +34,7 @@ __device__ __forceinline__ void cluster_sync_all(uint32_t csize) {
 }
 
 template <int kCsThreads, int E>
-__global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const SelectArgs a) {
+__global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_cluster_kernel(const SelectArgs a) {
     constexpr int kCsWarps = kCsThreads / 32;
     __shared__ __align__(16) uint32_t hist[2][4][256];   // ping-pong: a round never zeroes what peers still read
     __shared__ uint32_t chosen[4];                       // digit of the K-th value decided in the last round
@@ -363,7 +363,11 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int per_cta = p.max_len <= 8 * 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
-    return per_cta == 8192 ? launch_e<1024, 8>(p, a, cs, s) : launch_e<1024, 4>(p, a, cs, s);
+    if (per_cta == 8192) return launch_e<1024, 8>(p, a, cs, s);
+    // many units: half the threads with twice the keys each, two CTAs per SM, so that one CTA's barrier
+    // phases overlap the other's work
+    if (units * cs >= 2 * 148) return launch_e<512, 8>(p, a, cs, s);
+    return launch_e<1024, 4>(p, a, cs, s);
 }
 
 }  // namespace csp
