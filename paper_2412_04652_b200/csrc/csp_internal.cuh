@@ -71,11 +71,16 @@ struct CompactArgs {
 // Cluster size (CTAs per unit, a power of two <= 8).  At least enough CTAs to occupy the 148 SMs when
 // there are few units; more when that lets every CTA keep all of its tiles' logits on chip
 // (`tiles_kept` tiles per CTA; 0 if the kernel keeps none), which removes the second pass over K.
+// Clusters of 4 and 8 fit on 132 and 120 of the 148 SMs only, so when even 8 CTAs cannot keep the
+// logits the cluster stays small: pairs, which also halves the longest CTA of a ragged batch.
 inline int pick_cluster(int units, int max_tiles, int tiles_kept) {
     int c = 1;
     while (c < 8 && units * (c * 2) <= 148 && c * 2 <= max_tiles) c *= 2;
-    if (tiles_kept > 0)
+    if (tiles_kept > 0 && (max_tiles + 7) / 8 <= tiles_kept) {
         while (c < 8 && (max_tiles + c - 1) / c > tiles_kept) c *= 2;
+    } else if (tiles_kept > 0 && c < 2 && max_tiles >= 32) {
+        c = 2;
+    }
     return c;
 }
 

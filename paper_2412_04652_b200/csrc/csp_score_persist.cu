@@ -307,34 +307,8 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC));
                 tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + uint32_t(buf * NC));
                 tc_wait_ld();
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int jj = nt * 2 + e;
-                        float xv[4] = {__uint_as_float(v0[nt * 4 + e]) * scale2, __uint_as_float(v0[nt * 4 + 2 + e]) * scale2,
-                                       __uint_as_float(v1[nt * 4 + e]) * scale2, __uint_as_float(v1[nt * 4 + 2 + e]) * scale2};
-                        if (!masked) {
-                            const float mx = fmaxf(fmaxf(xv[0], xv[1]), fmaxf(xv[2], xv[3]));
-                            if (mx > m_run[jj] + kLazy) { z_run[jj] *= ex2f(m_run[jj] - mx); m_run[jj] = mx; }
-                            const float mm = m_run[jj];
-                            z_run[jj] += (ex2f(xv[0] - mm) + ex2f(xv[1] - mm)) + (ex2f(xv[2] - mm) + ex2f(xv[3] - mm));
-                        } else {
-                            const int colw = nt * 8 + lq * 2 + e;
-                            bool vis[4];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const int t = t_base + (r & 1) * 8 + (r >> 1) * 16;
-                                vis[r] = colw < W && t <= first_masked_key + colw;   // key <= query position
-                                xv[r] = vis[r] ? xv[r] : kNeg;
-                            }
-                            const float mx = fmaxf(fmaxf(xv[0], xv[1]), fmaxf(xv[2], xv[3]));
-                            if (mx > m_run[jj] + kLazy) { z_run[jj] *= ex2f(m_run[jj] - mx); m_run[jj] = mx; }
-                            const float mm = m_run[jj];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) z_run[jj] += vis[r] ? ex2f(xv[r] - mm) : 0.f;
-                        }
-                    }
+                if (!masked) stats_block(v0, v1, m_run, z_run, scale2);
+                else stats_block_masked(v0, v1, m_run, z_run, scale2, t_base, first_masked_key, W, lq);
             }
             // merge: lanes holding the same columns, then warps, then the CTAs of the cluster
 #pragma unroll

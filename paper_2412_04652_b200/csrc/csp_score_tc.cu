@@ -260,34 +260,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                 tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
                 tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
                 tc_wait_ld();
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int jj = nt * 2 + e;
-                        float x[4] = {__uint_as_float(v0[nt * 4 + e]) * scale2, __uint_as_float(v0[nt * 4 + 2 + e]) * scale2,
-                                      __uint_as_float(v1[nt * 4 + e]) * scale2, __uint_as_float(v1[nt * 4 + 2 + e]) * scale2};
-                        if (!masked) {
-                            const float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-                            if (mx > m_run[g][jj] + kLazy) { z_run[g][jj] *= ex2f(m_run[g][jj] - mx); m_run[g][jj] = mx; }
-                            const float mm = m_run[g][jj];
-                            z_run[g][jj] += (ex2f(x[0] - mm) + ex2f(x[1] - mm)) + (ex2f(x[2] - mm) + ex2f(x[3] - mm));
-                        } else {
-                            const int colw = nt * 8 + lq * 2 + e;
-                            bool vis[4];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const int t = t_base + (r & 1) * 8 + (r >> 1) * 16;
-                                vis[r] = colw < W && t <= first_masked_key + colw;   // key <= query position
-                                x[r] = vis[r] ? x[r] : kNeg;
-                            }
-                            const float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-                            if (mx > m_run[g][jj] + kLazy) { z_run[g][jj] *= ex2f(m_run[g][jj] - mx); m_run[g][jj] = mx; }
-                            const float mm = m_run[g][jj];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) z_run[g][jj] += vis[r] ? ex2f(x[r] - mm) : 0.f;
-                        }
-                    }
+                if (!masked) stats_block(v0, v1, m_run[g], z_run[g], scale2);
+                else stats_block_masked(v0, v1, m_run[g], z_run[g], scale2, t_base, first_masked_key, W, lq);
             }
             if (i >= kept) {                      // streaming buffer: hand it back to the MMA issuer
                 tc_fence_before();

@@ -109,5 +109,61 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     }
 }
 
+// ---- pass-1 row statistics of one 32-row x 32-column accumulator block ---------------------------------
+// v0 / v1: the two 16-row halves as loaded by tc_ld_16x32.  Statistic slot jj = 2 nt + e belongs to window
+// column 8 nt + 2 (lane % 4) + e; (m, z) is a running (reference, sum of 2^(x scale2 - reference)) over the
+// keys this thread has seen.  The reference is only raised when a value exceeds it by more than kLazy, which
+// is rare after the first tiles: the test is taken once for the whole block, so that the 32 exponentials
+// that follow are straight-line code.  scale2 > 0.
+__device__ __forceinline__ void stats_block(const uint32_t (&v0)[16], const uint32_t (&v1)[16], float (&m)[8],
+                                            float (&z)[8], float scale2) {
+    float mx[8];
+    bool raise = false;
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+        const int i = (jj >> 1) * 4 + (jj & 1);
+        mx[jj] = fmaxf(fmaxf(__uint_as_float(v0[i]), __uint_as_float(v0[i + 2])),
+                       fmaxf(__uint_as_float(v1[i]), __uint_as_float(v1[i + 2]))) * scale2;
+        raise |= mx[jj] > m[jj] + kLazy;
+    }
+    if (raise) {
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj)
+            if (mx[jj] > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - mx[jj]); m[jj] = mx[jj]; }
+    }
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+        const int i = (jj >> 1) * 4 + (jj & 1);
+        const float nm = -m[jj];
+        z[jj] += (ex2f(fmaf(__uint_as_float(v0[i]), scale2, nm)) + ex2f(fmaf(__uint_as_float(v0[i + 2]), scale2, nm))) +
+                 (ex2f(fmaf(__uint_as_float(v1[i]), scale2, nm)) + ex2f(fmaf(__uint_as_float(v1[i + 2]), scale2, nm)));
+    }
+}
+// The same for a tile that reaches into the window: key t is visible to window column w iff w < W and
+// t <= first_masked_key + w.  t_base = key of this thread's first row; lq = lane % 4.
+__device__ __forceinline__ void stats_block_masked(const uint32_t (&v0)[16], const uint32_t (&v1)[16], float (&m)[8],
+                                                   float (&z)[8], float scale2, int t_base, int first_masked_key,
+                                                   int W, int lq) {
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+        const int i = (jj >> 1) * 4 + (jj & 1);
+        const int colw = (jj >> 1) * 8 + lq * 2 + (jj & 1);
+        float x[4] = {__uint_as_float(v0[i]) * scale2, __uint_as_float(v0[i + 2]) * scale2,
+                      __uint_as_float(v1[i]) * scale2, __uint_as_float(v1[i + 2]) * scale2};
+        bool vis[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int t = t_base + (r & 1) * 8 + (r >> 1) * 16;
+            vis[r] = colw < W && t <= first_masked_key + colw;
+            x[r] = vis[r] ? x[r] : kNeg;
+        }
+        const float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+        if (mx > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - mx); m[jj] = mx; }
+        const float mm = m[jj];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) z[jj] += vis[r] ? ex2f(x[r] - mm) : 0.f;
+    }
+}
+
 }  // namespace dev
 }  // namespace csp
