@@ -383,12 +383,27 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
                 uint32_t va[16], vb[16];
                 tc_ld_row16(va, row_addr);
+                // Common case: every window query carries the same label and no column of this tile is
+                // hidden.  Then a key's weights all go to one of the two sums, chosen once per key, and the
+                // columns beyond W add exact zeros (their constant is -inf): plain sums, no selection.
+                const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     tc_wait_ld();
                     uint32_t (&cur)[16] = ch ? vb : va;
                     if (ch == 0) tc_ld_row16(vb, row_addr + 16u);
                     const float4* cv = reinterpret_cast<const float4*>(cv_team + ch * 16);
+                    if (plain) {
+#pragma unroll
+                        for (int j4 = 0; j4 < 4; ++j4) {
+                            const float4 cc = cv[j4];
+                            s0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                            s1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                            c0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                            c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                        }
+                        continue;
+                    }
                     const uint32_t as = add_s >> (ch * 16), ac = add_c >> (ch * 16);
 #pragma unroll
                     for (int j4 = 0; j4 < 4; ++j4) {
@@ -402,6 +417,11 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                         s0 += (as >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c0 += (ac >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;
                         s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                     }
+                }
+                if (plain) {
+                    const float total = (s0 + s1) + (c0 + c1);
+                    s0 = same ? total : 0.f; s1 = 0.f;
+                    c0 = same ? 0.f : total; c1 = 0.f;
                 }
                 tc_fence_before();
                 __syncwarp();

@@ -360,15 +360,45 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                     s1 += (as >> (j4 * 4 + 3)) & 1u ? p3 : 0.f; c1 += (ac >> (j4 * 4 + 3)) & 1u ? p3 : 0.f;
                 }
             };
+            // Common case: every window query carries the same label and no column of this tile is hidden.
+            // Then a key's weights all go to one of the two sums, chosen once per key, and the columns
+            // beyond W add exact zeros (their constant is -inf): plain sums, no per-column selection.
+            const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
+            auto chunk_plain = [&](const uint32_t (&cur)[16], const float* cvp) {
+                const float4* cv = reinterpret_cast<const float4*>(cvp);
+#pragma unroll
+                for (int j4 = 0; j4 < 4; ++j4) {
+                    const float4 cc = cv[j4];
+                    s0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                    s1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                    c0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                    c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                }
+            };
             // one query head per iteration, kept as a real loop for G > 2 so that the code stays small
+            if (plain) {
 #pragma unroll(G <= 2 ? G : 1)
-            for (int g = 0; g < G; ++g) {
-                tc_wait_ld();
-                tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
-                chunk(va, cvec + g * 32, add_s, add_c);
-                tc_wait_ld();
-                if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
-                chunk(vb, cvec + g * 32 + 16, add_s >> 16, add_c >> 16);
+                for (int g = 0; g < G; ++g) {
+                    tc_wait_ld();
+                    tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
+                    chunk_plain(va, cvec + g * 32);
+                    tc_wait_ld();
+                    if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
+                    chunk_plain(vb, cvec + g * 32 + 16);
+                }
+                const float total = (s0 + s1) + (c0 + c1);
+                s0 = same ? total : 0.f; s1 = 0.f;
+                c0 = same ? 0.f : total; c1 = 0.f;
+            } else {
+#pragma unroll(G <= 2 ? G : 1)
+                for (int g = 0; g < G; ++g) {
+                    tc_wait_ld();
+                    tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
+                    chunk(va, cvec + g * 32, add_s, add_c);
+                    tc_wait_ld();
+                    if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
+                    chunk(vb, cvec + g * 32 + 16, add_s >> 16, add_c >> 16);
+                }
             }
             const float s = s0 + s1, c = c0 + c1;
             if (i >= kept) {
