@@ -7,7 +7,10 @@
 //   warp 8      TMA producer: K tiles -> ring of 128B-swizzled shared-memory stages
 //   warp 9      one thread issues tcgen05.mma: D[128 keys x 32G queries] = K_tile . Q^T, fp32
 //               accumulators in tensor memory, several tiles in flight (ring of TMEM buffers)
-//   warps 0-7   epilogue, two groups of four warps taking alternate tiles, reading TMEM
+//   warps 0-7   epilogue, two groups of four warps taking alternate tiles, reading TMEM.  For G >= 3
+//               a second set of eight warps works on the same tiles: each set takes half of the
+//               query heads (columns), which halves the per-thread statistics and doubles the warps
+//               that hide the latency of tensor-memory loads and exponentials
 // The same tile stream runs twice:
 //   pass 1  all tiles of the unit: per window row a running (max, sum of 2^(x-max)); merged over
 //           lanes, warps and - through distributed shared memory - the CTAs of the cluster
@@ -24,9 +27,17 @@ namespace csp {
 namespace {
 using namespace dev;
 
-constexpr int kTcThreads = 320;
-constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
+// epilogue organisation for a group of G query heads per KV head
+template <int G> struct EpiPlan {
+    static constexpr bool kSplit = G >= 3;              // two warp sets, each with half of the heads
+    static constexpr int kSets = kSplit ? 2 : 1;
+    static constexpr int kWarps = 8 * kSets;
+    static constexpr int kEpiThreads = 32 * kWarps;
+    static constexpr int kHeads0 = kSplit ? (G + 1) / 2 : G;   // heads of set 0; set 1 takes the rest
+    static constexpr int kProducerWarp = kWarps;
+    static constexpr int kMmaWarp = kWarps + 1;
+    static constexpr int kThreads = 32 * (kWarps + 2);
+};
 constexpr int kMaxStages = 8;
 constexpr int kMaxTmemBufs = 16;
 
@@ -44,15 +55,16 @@ template <int G> struct TmemPlan {
 };
 
 struct TcSmemPlan {   // byte offsets from the 1024-aligned base
-    uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
+    uint32_t q, wstats, cstats, cvec, xchg, dq_mask, dq_val, bars, misc, total;
 };
 __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
     TcSmemPlan s;
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
     s.q = off;        off += uint32_t(nh) * uint32_t(g) * 32u * 128u;
-    s.wstats = off;   off += 8u * uint32_t(g) * 32u * 8u;
+    s.wstats = off;   off += (g >= 3 ? 16u * uint32_t((g + 1) / 2) : 8u * uint32_t(g)) * 32u * 8u;   // [warp][head of its set][column]
     s.cstats = off;   off += uint32_t(g) * 32u * 8u;
     s.cvec = off;     off += uint32_t(g) * 32u * 4u;
+    s.xchg = off;     off += 2u * 2u * 128u * 8u;       // [parity][group][key row]: set 1's partial sums
     s.dq_mask = off;  off += 32u * 4u;
     s.dq_val = off;   off += 32u * 4u;
     s.bars = off;     off += (2u * kMaxStages + 2u * kMaxTmemBufs + 1u) * 8u;
@@ -62,9 +74,11 @@ __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
 }
 
 template <int NH, int G>
-__global__ void __launch_bounds__(kTcThreads, (G == 1 && NH <= 2) ? 2 : 1)
+__global__ void __launch_bounds__(EpiPlan<G>::kThreads, (G == 1 && NH <= 2) ? 2 : 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages,
                 const int tmem_cols) {
+    using EP = EpiPlan<G>;
+    constexpr int kProducerWarp = EP::kProducerWarp, kMmaWarp = EP::kMmaWarp;
     constexpr int KS = NH * 4;                          // MMAs (K = 16 elements = 32 bytes) per tile
     constexpr int NC = TmemPlan<G>::kCols;
     const int TB = tmem_cols / NC;                      // accumulator buffers this CTA owns
@@ -81,6 +95,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     float2* const wstats = reinterpret_cast<float2*>(base_ptr + sp.wstats);
     float2* const cstats = reinterpret_cast<float2*>(base_ptr + sp.cstats);
     float* const cvec = reinterpret_cast<float*>(base_ptr + sp.cvec);
+    float2* const xchg = reinterpret_cast<float2*>(base_ptr + sp.xchg);
     uint32_t* const dq_mask = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_mask);
     uint32_t* const dq_val = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_val);
     const uint32_t full_k = base + sp.bars;
@@ -121,8 +136,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_k + 8 * s, 1); mbar_init(empty_k + 8 * s, 1); }
-        for (int i = 0; i < TB; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4); }
-        mbar_init(q_ready, 8);
+        for (int i = 0; i < TB; ++i) { mbar_init(tmem_full + 8 * i, 1); mbar_init(tmem_empty + 8 * i, 4 * EP::kSets); }
+        mbar_init(q_ready, EP::kWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -193,15 +208,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         cluster_wait();
     } else {
         // =============================== epilogue warps ===============================
-        const int quarter = warp & 3, group = warp >> 2;
+        const int set = warp >> 3;                          // which half of the query heads
+        const int quarter = warp & 3, group = (warp >> 2) & 1;
         const int lq = lane & 3, lr = lane >> 2;
+        const int g_lo = set * EP::kHeads0;                 // this warp's heads: [g_lo, g_lo + g_n)
+        const int g_n = set ? G - EP::kHeads0 : EP::kHeads0;
+        auto epi_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(EP::kEpiThreads) : "memory"); };
         const uint8_t* modp = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
 
         // stage Q of this KV group: row (g*32 + w), 128-byte column blocks, 16-byte chunks XOR-swizzled
         if (!skip) {
             const uint8_t* qb = static_cast<const uint8_t*>(a.q);
             constexpr int kChunksPerRow = NH * 8;
-            for (int i = tid; i < G * 32 * kChunksPerRow; i += kConsumerThreads) {
+            for (int i = tid; i < G * 32 * kChunksPerRow; i += EP::kEpiThreads) {
                 const int r = i / kChunksPerRow, c = i % kChunksPerRow;
                 const int g = r >> 5, w = r & 31;
                 uint4 v = make_uint4(0, 0, 0, 0);
@@ -213,7 +232,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                 *reinterpret_cast<uint4*>(base_ptr + sp.q + off) = v;
             }
         } else {
-            for (int i = tid; i < NH * NC * 8; i += kConsumerThreads)
+            for (int i = tid; i < NH * NC * 8; i += EP::kEpiThreads)
                 *reinterpret_cast<uint4*>(base_ptr + sp.q + i * 16) = make_uint4(0, 0, 0, 0);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make Q visible to the tensor core
@@ -240,11 +259,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         const int first_masked_key = L - W;       // keys beyond this may be hidden from some window row
 
         // ---------------------------------- pass 1 ----------------------------------
-        float m_run[G][8], z_run[G][8];
+        float m_run[EP::kHeads0][8], z_run[EP::kHeads0][8];
 #pragma unroll
-        for (int g = 0; g < G; ++g)
+        for (int gl = 0; gl < EP::kHeads0; ++gl)
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj) { m_run[g][jj] = kNeg; z_run[g][jj] = 0.f; }
+            for (int jj = 0; jj < 8; ++jj) { m_run[gl][jj] = kNeg; z_run[gl][jj] = 0.f; }
 
         for (int i = group; i < my_all; i += 2) {
             const int buf = buf_of(i, 0);
@@ -254,14 +273,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             const bool masked = (tile + 1) * kTileKeys > first_masked_key;
             const int t_base = tile * kTileKeys + quarter * 32 + lr;
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                uint32_t v0[16], v1[16];
-                const uint32_t col = uint32_t(buf * NC + g * 32);
-                tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
-                tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
-                tc_wait_ld();
-                if (!masked) stats_block(v0, v1, m_run[g], z_run[g], scale2);
-                else stats_block_masked(v0, v1, m_run[g], z_run[g], scale2, t_base, first_masked_key, W, lq);
+            for (int gl = 0; gl < EP::kHeads0; ++gl) {
+                if (gl < g_n) {
+                    uint32_t v0[16], v1[16];
+                    const uint32_t col = uint32_t(buf * NC + (g_lo + gl) * 32);
+                    tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
+                    tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
+                    tc_wait_ld();
+                    if (!masked) stats_block(v0, v1, m_run[gl], z_run[gl], scale2);
+                    else stats_block_masked(v0, v1, m_run[gl], z_run[gl], scale2, t_base, first_masked_key, W, lq);
+                }
             }
             if (i >= kept) {                      // streaming buffer: hand it back to the MMA issuer
                 tc_fence_before();
@@ -272,23 +293,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
 
         // merge the running statistics: lanes holding the same columns, then warps, then CTAs
 #pragma unroll
-        for (int g = 0; g < G; ++g)
+        for (int gl = 0; gl < EP::kHeads0; ++gl)
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
 #pragma unroll
                 for (int d = 4; d <= 16; d <<= 1) {
-                    const float om = __shfl_xor_sync(0xffffffffu, m_run[g][jj], d);
-                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[g][jj], d);
-                    merge_stats(m_run[g][jj], z_run[g][jj], om, oz);
+                    const float om = __shfl_xor_sync(0xffffffffu, m_run[gl][jj], d);
+                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[gl][jj], d);
+                    merge_stats(m_run[gl][jj], z_run[gl][jj], om, oz);
                 }
-                if (lr == 0) wstats[(warp * G + g) * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[g][jj], z_run[g][jj]);
+                if (lr == 0) wstats[(warp * EP::kHeads0 + gl) * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[gl][jj], z_run[gl][jj]);
             }
-        consumer_sync();
+        epi_sync();
         if (tid < G * 32) {
+            const int g = tid >> 5, gs = g >= EP::kHeads0 ? 1 : 0;       // head, and the warp set that holds it
+            const int gl = g - gs * EP::kHeads0;
             float m = kNeg, z = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) {
-                const float2 s = wstats[w * (G * 32) + tid];
+                const float2 s = wstats[((gs * 8 + w) * EP::kHeads0 + gl) * 32 + (tid & 31)];
                 merge_stats(m, z, s.x, s.y);
             }
             cstats[tid] = make_float2(m, z);
@@ -315,7 +338,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             const float denom = a.n * ex2f(-m) + z;
             cvec[tid] = col < W ? lg2f(a.weight / denom) - m : -INFINITY;
         }
-        consumer_sync();
+        epi_sync();
 
         // ---------------------------------- pass 2 ----------------------------------
         float* const out_s = a.score_self + (int64_t(b) * a.n_kv_heads + h) * a.max_len;
@@ -341,7 +364,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // the row of 32 G logits is read in chunks of 16 columns; the load of the next chunk is in
             // flight while the current one is turned into weights (two accumulators per score)
             float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
-            const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
+            const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + g_lo * 32);
+            const float* const cv_mine = cvec + g_lo * 32;
             uint32_t va[16], vb[16];
             tc_ld_row16(va, row_addr);
             // weights of 16 columns: cur = logits, cv = their additive constants, as/ac = which columns count
@@ -378,35 +402,44 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // one query head per iteration, kept as a real loop for G > 2 so that the code stays small
             if (plain) {
 #pragma unroll(G <= 2 ? G : 1)
-                for (int g = 0; g < G; ++g) {
+                for (int gl = 0; gl < g_n; ++gl) {
                     tc_wait_ld();
-                    tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
-                    chunk_plain(va, cvec + g * 32);
+                    tc_ld_row16(vb, row_addr + uint32_t(gl * 32 + 16));
+                    chunk_plain(va, cv_mine + gl * 32);
                     tc_wait_ld();
-                    if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
-                    chunk_plain(vb, cvec + g * 32 + 16);
+                    if (gl + 1 < g_n) tc_ld_row16(va, row_addr + uint32_t(gl * 32 + 32));
+                    chunk_plain(vb, cv_mine + gl * 32 + 16);
                 }
                 const float total = (s0 + s1) + (c0 + c1);
                 s0 = same ? total : 0.f; s1 = 0.f;
                 c0 = same ? 0.f : total; c1 = 0.f;
             } else {
 #pragma unroll(G <= 2 ? G : 1)
-                for (int g = 0; g < G; ++g) {
+                for (int gl = 0; gl < g_n; ++gl) {
                     tc_wait_ld();
-                    tc_ld_row16(vb, row_addr + uint32_t(g * 32 + 16));
-                    chunk(va, cvec + g * 32, add_s, add_c);
+                    tc_ld_row16(vb, row_addr + uint32_t(gl * 32 + 16));
+                    chunk(va, cv_mine + gl * 32, add_s, add_c);
                     tc_wait_ld();
-                    if (g + 1 < G) tc_ld_row16(va, row_addr + uint32_t(g * 32 + 32));
-                    chunk(vb, cvec + g * 32 + 16, add_s >> 16, add_c >> 16);
+                    if (gl + 1 < g_n) tc_ld_row16(va, row_addr + uint32_t(gl * 32 + 32));
+                    chunk(vb, cv_mine + gl * 32 + 16, add_s >> 16, add_c >> 16);
                 }
             }
-            const float s = s0 + s1, c = c0 + c1;
+            float s = s0 + s1, c = c0 + c1;
             if (i >= kept) {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);
             }
-            if (t < N) { out_s[t] = s; out_c[t] = c; }
+            if (EP::kSplit) {
+                // set 1 hands its partial sums to the set-0 warp that holds the same keys (a 64-thread
+                // barrier per warp pair); the slot alternates with the iteration, so set 1 can only
+                // overwrite it after set 0 has passed the next barrier, i.e. after it has read it
+                float2* const slot = xchg + (((i >> 1) & 1) * 2 + group) * 128 + quarter * 32 + lane;
+                if (set == 1) *slot = make_float2(s, c);
+                asm volatile("bar.sync %0, 64;" ::"r"(2 + group * 4 + quarter) : "memory");
+                if (set == 0) { const float2 o = *slot; s += o.x; c += o.y; }
+            }
+            if (set == 0 && t < N) { out_s[t] = s; out_c[t] = c; }
         }
         if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
     }
@@ -449,7 +482,7 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
-    cfg.blockDim = dim3(kTcThreads);
+    cfg.blockDim = dim3(EpiPlan<G>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
