@@ -196,6 +196,13 @@ def run_reference(args, rank, world):
 
 # ------------------------------------------------------------------------------------ CUDA arm
 
+def kernels_per_call(p) -> int:
+    """Kernels one csp_prune_layer call launches: score, select, compact, and, for a bf16 cache with more
+    (sequence, head) units than SMs and several sequences, the kernel that orders them by length."""
+    ordered = p.dtype == 1 and 2 <= p.batch <= 4096 and p.batch * p.n_kv_heads > 148
+    return 4 if ordered else 3
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -487,7 +494,7 @@ def main():
                            "l2": "inputs larger than L2: every layer has its own K/V buffers"
                                  if n_buf * ab["score"] > 2 * 126e6 else "inputs smaller than L2",
                            "replicas": "one independent replica per GPU, no collective"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(calls) * 3,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * sum(kernels_per_call(c[0]) for c in calls),
                 "roofline": roofline, "path": path, "cpu_baseline": cpu_baseline, "device_status": status}
         print(json.dumps(line), flush=True)
     if dist is not None:

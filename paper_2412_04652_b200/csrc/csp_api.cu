@@ -63,6 +63,8 @@ csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& 
     a.score_self = mean_all ? reinterpret_cast<float*>(static_cast<char*>(ws) + wl.part_self) : score_self;
     a.score_cross = mean_all ? reinterpret_cast<float*>(static_cast<char*>(ws) + wl.part_cross) : score_cross;
     a.status = static_cast<int32_t*>(ws);
+    a.order_buf = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + wl.order);
+    a.order = nullptr;
     a.n_kv_heads = p.n_kv_heads; a.group = p.n_q_heads / p.n_kv_heads;
     a.window = p.window; a.recent = p.recent; a.max_len = p.max_len;
     a.n = p.n;

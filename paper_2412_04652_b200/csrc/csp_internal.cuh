@@ -17,10 +17,11 @@ namespace csp {
 //   part_self   fp32 [B, Hkv, max_len]     (MEAN_ALL: per-KV-head partial sums)
 //   part_cross  fp32 [B, Hkv, max_len]
 //   keep_idx    int32 [B, Hkv, out_capacity]
+//   order       int32 [B]                  (sequences by descending length, for load balance)
 constexpr size_t kStatusBytes = 256;
 
 struct WorkspaceLayout {
-    size_t score_self, score_cross, part_self, part_cross, keep_idx, total;
+    size_t score_self, score_cross, part_self, part_cross, keep_idx, order, total;
 };
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -34,7 +35,8 @@ inline WorkspaceLayout workspace_layout(const csp_params& p) {
     w.part_self = w.score_cross + sc;
     w.part_cross = w.part_self + sc;
     w.keep_idx = w.part_cross + sc;
-    w.total = w.keep_idx + round256(units * size_t(p.out_capacity) * 4);
+    w.order = w.keep_idx + round256(units * size_t(p.out_capacity) * 4);
+    w.total = w.order + round256(size_t(p.batch) * 4);
     return w;
 }
 
@@ -46,6 +48,8 @@ struct ScoreArgs {
     const float* lse;                                // may be null
     float* score_self; float* score_cross;           // [B, Hkv, max_len]
     int32_t* status;
+    int32_t* order_buf;                              // scratch for `order`, int32 [B]
+    const int32_t* order;                            // null, or the sequences by descending length
     int32_t n_kv_heads, group, window, recent, max_len;
     float n, scale_log2, weight;                     // weight = 1/G or 1/Hq
 };

@@ -507,9 +507,27 @@ csp_status launch_t(const csp_params& p, const ScoreArgs& a, const CUtensorMap& 
     }
 }
 
+// order[r] = the sequence with the r-th longest valid length (ties: lower index first).  The scoring
+// kernels take sequences in this order, longest first, so that a ragged batch does not end with one
+// long unit running alone.
+__global__ void length_order_kernel(const int32_t* __restrict__ seq_lens, int batch, int max_len,
+                                    int32_t* __restrict__ order) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= batch) return;
+    auto len = [&](int i) { const int L = seq_lens[i]; return (L < 0 || L > max_len) ? 0 : L; };
+    const int Lt = len(t);
+    int r = 0;
+    for (int j = 0; j < batch; ++j) {
+        const int Lj = len(j);
+        r += (Lj > Lt || (Lj == Lt && j < t)) ? 1 : 0;
+    }
+    order[r] = t;
+}
+
 }  // namespace
 
-csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s) {
+csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_tensor& k, cudaStream_t s) {
+    ScoreArgs a = a_in;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return CSP_ERR_CUDA;
     const uint64_t es = p.dtype == CSP_F32 ? 4 : 2;
@@ -533,6 +551,12 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tenso
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return CSP_ERR_UNSUPPORTED;
     if (p.dtype == CSP_F32) return launch_t<float>(p, a, tmap, s);
+    // more units than SMs and several sequences: take them longest first
+    if (p.batch >= 2 && p.batch <= 4096 && p.batch * p.n_kv_heads > 148) {
+        length_order_kernel<<<(p.batch + 255) / 256, 256, 0, s>>>(a.seq_lens, p.batch, p.max_len, a.order_buf);
+        if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
+        a.order = a.order_buf;
+    }
     // many MHA units: resident clusters that stream unit after unit; otherwise one cluster per unit
     bool taken = false;
     const csp_status ps = launch_score_persist(p, a, tmap, s, &taken);

@@ -143,6 +143,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     auto unit_of = [&](int u) {
         Unit x;
         x.b = u / a.n_kv_heads; x.h = u % a.n_kv_heads;
+        if (a.order) x.b = a.order[x.b];
         int L = a.seq_lens[x.b];
         const bool bad = L < 0 || L > a.max_len;
         x.skip = bad || L < a.window || L < a.recent;
@@ -157,12 +158,24 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
         return x;
     };
 
+    // The j-th unit of this cluster, or -1 when it has none left.  Units are dealt to the clusters in
+    // rounds of n_clusters; with the sequences sorted by length the direction alternates from round to
+    // round, so that every cluster gets a similar share of long and short ones.  Only the last round can
+    // be short: a cluster's list never has a hole.
+    auto unit_at = [&](int j) {
+        const int pos = (a.order && (j & 1)) ? n_clusters - 1 - cid : cid;
+        const int u = j * n_clusters + pos;
+        return u < n_units ? u : -1;
+    };
+
     if (warp == kPsProducerWarp) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
             int it = 0;
-            for (int u = cid; u < n_units && !*abort_flag; u += n_clusters) {
+            for (int j = 0; !*abort_flag; ++j) {
+                const int u = unit_at(j);
+                if (u < 0) break;
                 const Unit x = unit_of(u);
                 for (int i = 0; i < x.my_all; ++i, ++it) {
                     const int slot = it % n_stages;
@@ -189,8 +202,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     } else if (warp == kPsMmaWarp) {
         // =============================== MMA issuer ===============================
         if (lane == 0) {
-            int it = 0, j = 0;
-            for (int u = cid; u < n_units && !*abort_flag; u += n_clusters, ++j) {
+            int it = 0;
+            for (int j = 0; !*abort_flag; ++j) {
+                const int u = unit_at(j);
+                if (u < 0) break;
                 const Unit x = unit_of(u);
                 const uint32_t bph = uint32_t(j) & 1u;                  // every buffer is released once per unit
                 const uint32_t my_full = tmem_full + 8 * kBufs * (j & 1);   // barrier set of the team that takes unit j
@@ -226,9 +241,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
         __syncwarp();
     } else if (warp == kPsStageWarp) {
         // =============================== Q / label-table stager ===============================
-        int j = 0;
-        for (int u = cid; u < n_units; u += n_clusters, ++j) {
+        for (int j = 0;; ++j) {
             if (__any_sync(0xffffffffu, *abort_flag != 0)) break;        // the whole warp leaves together
+            const int u = unit_at(j);
+            if (u < 0) break;
             const Unit x = unit_of(u);
             const int qs = j % kQSets;
             const uint32_t qph = uint32_t(j / kQSets) & 1u;
@@ -279,7 +295,9 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
         const uint32_t wmask = W >= 32 ? 0xFFFFFFFFu : ((1u << W) - 1u);
         float2* const wst = wstats + team * (kTeamWarps * 32);
         float* const cv_team = cvec + team * 32;
-        for (int j = team, u = cid + team * n_clusters; u < n_units; u += kTeams * n_clusters, j += kTeams) {
+        for (int j = team;; j += kTeams) {
+            const int u = unit_at(j);
+            if (u < 0) break;
             if (barrier_any(*abort_flag != 0, 1 + team, kTeamThreads)) break;   // the whole team leaves together
             const Unit x = unit_of(u);
             const int p = j & 1;

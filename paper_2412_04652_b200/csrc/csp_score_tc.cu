@@ -108,7 +108,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     volatile int* const n_dq = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 8);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int h = blockIdx.y, b = blockIdx.z;
+    const int h = blockIdx.y, b = a.order ? a.order[blockIdx.z] : int(blockIdx.z);
     const uint32_t rank = cluster_rank(), csize = cluster_size();
 
     int L = a.seq_lens[b];

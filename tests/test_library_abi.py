@@ -40,7 +40,8 @@ def test_workspace_size_formula(csp):
     p = csp.Params(2, 8, 4, 128, 32, 32, 1000, 300)
     scores = ((2 * 4 * 1000 * 4 + 255) // 256) * 256
     idx = ((2 * 4 * 300 * 4 + 255) // 256) * 256
-    assert csp.workspace_bytes(p) == 256 + 4 * scores + idx
+    order = 256                  # one int32 per sequence, rounded up
+    assert csp.workspace_bytes(p) == 256 + 4 * scores + idx + order
     assert csp.host_staging_bytes(p) > csp.workspace_bytes(p)
 
 
