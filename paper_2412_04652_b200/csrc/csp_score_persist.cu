@@ -325,8 +325,8 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC));
                 tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + uint32_t(buf * NC));
                 tc_wait_ld();
-                if (!masked) stats_block(v0, v1, m_run, z_run, scale2);
-                else stats_block_masked(v0, v1, m_run, z_run, scale2, t_base, first_masked_key, W, lq);
+                if (!masked) stats_block<4>(v0, v1, m_run, z_run, scale2);
+                else stats_block_masked<4>(v0, v1, m_run, z_run, scale2, t_base, first_masked_key, W, lq * 2);
             }
             // merge: lanes holding the same columns, then warps, then the CTAs of the cluster
 #pragma unroll

@@ -8,9 +8,9 @@
 //   warp 9      one thread issues tcgen05.mma: D[128 keys x 32G queries] = K_tile . Q^T, fp32
 //               accumulators in tensor memory, several tiles in flight (ring of TMEM buffers)
 //   warps 0-7   epilogue, two groups of four warps taking alternate tiles, reading TMEM.  For G >= 3
-//               a second set of eight warps works on the same tiles: each set takes half of the
-//               query heads (columns), which halves the per-thread statistics and doubles the warps
-//               that hide the latency of tensor-memory loads and exponentials
+//               a second set of eight warps works on the same tiles: each set takes 16 of the 32
+//               window columns of every query head, which halves the per-thread statistics and
+//               doubles the warps that hide the latency of tensor-memory loads and exponentials
 // The same tile stream runs twice:
 //   pass 1  all tiles of the unit: per window row a running (max, sum of 2^(x-max)); merged over
 //           lanes, warps and - through distributed shared memory - the CTAs of the cluster
@@ -29,11 +29,12 @@ using namespace dev;
 
 // epilogue organisation for a group of G query heads per KV head
 template <int G> struct EpiPlan {
-    static constexpr bool kSplit = G >= 3;              // two warp sets, each with half of the heads
+    static constexpr bool kSplit = G >= 3;              // two warp sets, each with half of the window columns
     static constexpr int kSets = kSplit ? 2 : 1;
     static constexpr int kWarps = 8 * kSets;
     static constexpr int kEpiThreads = 32 * kWarps;
-    static constexpr int kHeads0 = kSplit ? (G + 1) / 2 : G;   // heads of set 0; set 1 takes the rest
+    static constexpr int kBlocks = kSplit ? 2 : 4;      // 8-column blocks per head and thread in pass 1
+    static constexpr int kCols = 8 * kBlocks;           // window columns of a head that one set handles
     static constexpr int kProducerWarp = kWarps;
     static constexpr int kMmaWarp = kWarps + 1;
     static constexpr int kThreads = 32 * (kWarps + 2);
@@ -61,7 +62,7 @@ __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
     TcSmemPlan s;
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
     s.q = off;        off += uint32_t(nh) * uint32_t(g) * 32u * 128u;
-    s.wstats = off;   off += (g >= 3 ? 16u * uint32_t((g + 1) / 2) : 8u * uint32_t(g)) * 32u * 8u;   // [warp][head of its set][column]
+    s.wstats = off;   off += 8u * uint32_t(g) * 32u * 8u;   // [warp][head][column of its set]
     s.cstats = off;   off += uint32_t(g) * 32u * 8u;
     s.cvec = off;     off += uint32_t(g) * 32u * 4u;
     s.xchg = off;     off += 2u * 2u * 128u * 8u;       // [parity][group][key row]: set 1's partial sums
@@ -208,11 +209,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         cluster_wait();
     } else {
         // =============================== epilogue warps ===============================
-        const int set = warp >> 3;                          // which half of the query heads
+        const int set = warp >> 3;                          // which half of the window columns
         const int quarter = warp & 3, group = (warp >> 2) & 1;
         const int lq = lane & 3, lr = lane >> 2;
-        const int g_lo = set * EP::kHeads0;                 // this warp's heads: [g_lo, g_lo + g_n)
-        const int g_n = set ? G - EP::kHeads0 : EP::kHeads0;
+        const int cofs = set * EP::kCols;                   // this warp's columns of every head: [cofs, cofs + kCols)
         auto epi_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(EP::kEpiThreads) : "memory"); };
         const uint8_t* modp = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
 
@@ -259,11 +259,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         const int first_masked_key = L - W;       // keys beyond this may be hidden from some window row
 
         // ---------------------------------- pass 1 ----------------------------------
-        float m_run[EP::kHeads0][8], z_run[EP::kHeads0][8];
+        constexpr int NB = EP::kBlocks;
+        float m_run[G][2 * NB], z_run[G][2 * NB];
 #pragma unroll
-        for (int gl = 0; gl < EP::kHeads0; ++gl)
+        for (int g = 0; g < G; ++g)
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj) { m_run[gl][jj] = kNeg; z_run[gl][jj] = 0.f; }
+            for (int jj = 0; jj < 2 * NB; ++jj) { m_run[g][jj] = kNeg; z_run[g][jj] = 0.f; }
 
         for (int i = group; i < my_all; i += 2) {
             const int buf = buf_of(i, 0);
@@ -273,16 +274,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             const bool masked = (tile + 1) * kTileKeys > first_masked_key;
             const int t_base = tile * kTileKeys + quarter * 32 + lr;
 #pragma unroll
-            for (int gl = 0; gl < EP::kHeads0; ++gl) {
-                if (gl < g_n) {
-                    uint32_t v0[16], v1[16];
-                    const uint32_t col = uint32_t(buf * NC + (g_lo + gl) * 32);
-                    tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
-                    tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
-                    tc_wait_ld();
-                    if (!masked) stats_block(v0, v1, m_run[gl], z_run[gl], scale2);
-                    else stats_block_masked(v0, v1, m_run[gl], z_run[gl], scale2, t_base, first_masked_key, W, lq);
-                }
+            for (int g = 0; g < G; ++g) {
+                uint32_t v0[4 * NB], v1[4 * NB];
+                const uint32_t col = uint32_t(buf * NC + g * 32 + cofs);
+                tc_ld_frag(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
+                tc_ld_frag(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
+                tc_wait_ld();
+                if (!masked) stats_block<NB>(v0, v1, m_run[g], z_run[g], scale2);
+                else stats_block_masked<NB>(v0, v1, m_run[g], z_run[g], scale2, t_base, first_masked_key, W, cofs + lq * 2);
             }
             if (i >= kept) {                      // streaming buffer: hand it back to the MMA issuer
                 tc_fence_before();
@@ -293,25 +292,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
 
         // merge the running statistics: lanes holding the same columns, then warps, then CTAs
 #pragma unroll
-        for (int gl = 0; gl < EP::kHeads0; ++gl)
+        for (int g = 0; g < G; ++g)
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
+            for (int jj = 0; jj < 2 * NB; ++jj) {
 #pragma unroll
                 for (int d = 4; d <= 16; d <<= 1) {
-                    const float om = __shfl_xor_sync(0xffffffffu, m_run[gl][jj], d);
-                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[gl][jj], d);
-                    merge_stats(m_run[gl][jj], z_run[gl][jj], om, oz);
+                    const float om = __shfl_xor_sync(0xffffffffu, m_run[g][jj], d);
+                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[g][jj], d);
+                    merge_stats(m_run[g][jj], z_run[g][jj], om, oz);
                 }
-                if (lr == 0) wstats[(warp * EP::kHeads0 + gl) * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[gl][jj], z_run[gl][jj]);
+                if (lr == 0) wstats[(warp * G + g) * EP::kCols + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[g][jj], z_run[g][jj]);
             }
         epi_sync();
         if (tid < G * 32) {
-            const int g = tid >> 5, gs = g >= EP::kHeads0 ? 1 : 0;       // head, and the warp set that holds it
-            const int gl = g - gs * EP::kHeads0;
+            const int g = tid >> 5, col = tid & 31;
+            const int cs = col / EP::kCols, cl = col % EP::kCols;        // the warp set that holds the column
             float m = kNeg, z = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) {
-                const float2 s = wstats[((gs * 8 + w) * EP::kHeads0 + gl) * 32 + (tid & 31)];
+                const float2 s = wstats[((cs * 8 + w) * G + g) * EP::kCols + cl];
                 merge_stats(m, z, s.x, s.y);
             }
             cstats[tid] = make_float2(m, z);
@@ -364,8 +363,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // the row of 32 G logits is read in chunks of 16 columns; the load of the next chunk is in
             // flight while the current one is turned into weights (two accumulators per score)
             float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
-            const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + g_lo * 32);
-            const float* const cv_mine = cvec + g_lo * 32;
+            const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + cofs);
             uint32_t va[16], vb[16];
             tc_ld_row16(va, row_addr);
             // weights of 16 columns: cur = logits, cv = their additive constants, as/ac = which columns count
@@ -399,29 +397,40 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                     c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
                 }
             };
-            // one query head per iteration, kept as a real loop for G > 2 so that the code stays small
+            // The thread's columns come in chunks of 16: chunk k sits kStep columns after chunk k - 1 (both
+            // halves of every head, or this set's half of every head) and uses bits kShift(k) of the masks.
+            // Two chunks per iteration, the load of the next one in flight while one is turned into weights;
+            // kept as a real loop for G > 2 so that the code stays small.
+            constexpr int kChunks = EP::kSplit ? G : 2 * G;
+            constexpr int kStep = EP::kSplit ? 32 : 16;
+            const float* const cv_mine = cvec + cofs;
+            auto shift_of = [&](int k) { return EP::kSplit ? cofs : (k & 1) * 16; };
             if (plain) {
 #pragma unroll(G <= 2 ? G : 1)
-                for (int gl = 0; gl < g_n; ++gl) {
+                for (int k = 0; k < kChunks; k += 2) {
                     tc_wait_ld();
-                    tc_ld_row16(vb, row_addr + uint32_t(gl * 32 + 16));
-                    chunk_plain(va, cv_mine + gl * 32);
-                    tc_wait_ld();
-                    if (gl + 1 < g_n) tc_ld_row16(va, row_addr + uint32_t(gl * 32 + 32));
-                    chunk_plain(vb, cv_mine + gl * 32 + 16);
+                    if (k + 1 < kChunks) tc_ld_row16(vb, row_addr + uint32_t((k + 1) * kStep));
+                    chunk_plain(va, cv_mine + k * kStep);
+                    if (k + 1 < kChunks) {
+                        tc_wait_ld();
+                        if (k + 2 < kChunks) tc_ld_row16(va, row_addr + uint32_t((k + 2) * kStep));
+                        chunk_plain(vb, cv_mine + (k + 1) * kStep);
+                    }
                 }
                 const float total = (s0 + s1) + (c0 + c1);
                 s0 = same ? total : 0.f; s1 = 0.f;
                 c0 = same ? 0.f : total; c1 = 0.f;
             } else {
 #pragma unroll(G <= 2 ? G : 1)
-                for (int gl = 0; gl < g_n; ++gl) {
+                for (int k = 0; k < kChunks; k += 2) {
                     tc_wait_ld();
-                    tc_ld_row16(vb, row_addr + uint32_t(gl * 32 + 16));
-                    chunk(va, cv_mine + gl * 32, add_s, add_c);
-                    tc_wait_ld();
-                    if (gl + 1 < g_n) tc_ld_row16(va, row_addr + uint32_t(gl * 32 + 32));
-                    chunk(vb, cv_mine + gl * 32 + 16, add_s >> 16, add_c >> 16);
+                    if (k + 1 < kChunks) tc_ld_row16(vb, row_addr + uint32_t((k + 1) * kStep));
+                    chunk(va, cv_mine + k * kStep, add_s >> shift_of(k), add_c >> shift_of(k));
+                    if (k + 1 < kChunks) {
+                        tc_wait_ld();
+                        if (k + 2 < kChunks) tc_ld_row16(va, row_addr + uint32_t((k + 2) * kStep));
+                        chunk(vb, cv_mine + (k + 1) * kStep, add_s >> shift_of(k + 1), add_c >> shift_of(k + 1));
+                    }
                 }
             }
             float s = s0 + s1, c = c0 + c1;

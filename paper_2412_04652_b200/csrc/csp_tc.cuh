@@ -67,6 +67,15 @@ __device__ __forceinline__ void tc_ld_16x32(uint32_t (&v)[16], uint32_t taddr) {
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr) : "memory");
 }
+// the same for 16 columns: regs 4i..4i+3 of 8-column block i = 0, 1
+__device__ __forceinline__ void tc_ld_16x16(uint32_t (&v)[8], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_frag(uint32_t (&v)[16], uint32_t taddr) { tc_ld_16x32(v, taddr); }
+__device__ __forceinline__ void tc_ld_frag(uint32_t (&v)[8], uint32_t taddr) { tc_ld_16x16(v, taddr); }
 // shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
 __device__ __forceinline__ uint64_t sw128_desc(uint32_t smem_addr) {
     uint64_t d = uint64_t((smem_addr & 0x3FFFFu) >> 4);
@@ -109,18 +118,19 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     }
 }
 
-// ---- pass-1 row statistics of one 32-row x 32-column accumulator block ---------------------------------
-// v0 / v1: the two 16-row halves as loaded by tc_ld_16x32.  Statistic slot jj = 2 nt + e belongs to window
-// column 8 nt + 2 (lane % 4) + e; (m, z) is a running (reference, sum of 2^(x scale2 - reference)) over the
-// keys this thread has seen.  The reference is only raised when a value exceeds it by more than kLazy, which
-// is rare after the first tiles: the test is taken once for the whole block, so that the 32 exponentials
+// ---- pass-1 row statistics of one accumulator block of 32 rows x 8 NB columns ----------------------------
+// v0 / v1: the two 16-row halves as loaded by tc_ld_frag.  Statistic slot jj = 2 nt + e belongs to column
+// 8 nt + 2 (lane % 4) + e of the block; (m, z) is a running (reference, sum of 2^(x scale2 - reference)) over
+// the keys this thread has seen.  The reference is only raised when a value exceeds it by more than kLazy,
+// which is rare after the first tiles: the test is taken once for the whole block, so that the exponentials
 // that follow are straight-line code.  scale2 > 0.
-__device__ __forceinline__ void stats_block(const uint32_t (&v0)[16], const uint32_t (&v1)[16], float (&m)[8],
-                                            float (&z)[8], float scale2) {
-    float mx[8];
+template <int NB>
+__device__ __forceinline__ void stats_block(const uint32_t (&v0)[4 * NB], const uint32_t (&v1)[4 * NB],
+                                            float (&m)[2 * NB], float (&z)[2 * NB], float scale2) {
+    float mx[2 * NB];
     bool raise = false;
 #pragma unroll
-    for (int jj = 0; jj < 8; ++jj) {
+    for (int jj = 0; jj < 2 * NB; ++jj) {
         const int i = (jj >> 1) * 4 + (jj & 1);
         mx[jj] = fmaxf(fmaxf(__uint_as_float(v0[i]), __uint_as_float(v0[i + 2])),
                        fmaxf(__uint_as_float(v1[i]), __uint_as_float(v1[i + 2]))) * scale2;
@@ -128,11 +138,11 @@ __device__ __forceinline__ void stats_block(const uint32_t (&v0)[16], const uint
     }
     if (raise) {
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
+        for (int jj = 0; jj < 2 * NB; ++jj)
             if (mx[jj] > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - mx[jj]); m[jj] = mx[jj]; }
     }
 #pragma unroll
-    for (int jj = 0; jj < 8; ++jj) {
+    for (int jj = 0; jj < 2 * NB; ++jj) {
         const int i = (jj >> 1) * 4 + (jj & 1);
         const float nm = -m[jj];
         z[jj] += (ex2f(fmaf(__uint_as_float(v0[i]), scale2, nm)) + ex2f(fmaf(__uint_as_float(v0[i + 2]), scale2, nm))) +
@@ -140,14 +150,16 @@ __device__ __forceinline__ void stats_block(const uint32_t (&v0)[16], const uint
     }
 }
 // The same for a tile that reaches into the window: key t is visible to window column w iff w < W and
-// t <= first_masked_key + w.  t_base = key of this thread's first row; lq = lane % 4.
-__device__ __forceinline__ void stats_block_masked(const uint32_t (&v0)[16], const uint32_t (&v1)[16], float (&m)[8],
-                                                   float (&z)[8], float scale2, int t_base, int first_masked_key,
-                                                   int W, int lq) {
+// t <= first_masked_key + w.  t_base = key of this thread's first row; col0 = window column of the block's
+// first column plus 2 (lane % 4).
+template <int NB>
+__device__ __forceinline__ void stats_block_masked(const uint32_t (&v0)[4 * NB], const uint32_t (&v1)[4 * NB],
+                                                   float (&m)[2 * NB], float (&z)[2 * NB], float scale2, int t_base,
+                                                   int first_masked_key, int W, int col0) {
 #pragma unroll
-    for (int jj = 0; jj < 8; ++jj) {
+    for (int jj = 0; jj < 2 * NB; ++jj) {
         const int i = (jj >> 1) * 4 + (jj & 1);
-        const int colw = (jj >> 1) * 8 + lq * 2 + (jj & 1);
+        const int colw = col0 + (jj >> 1) * 8 + (jj & 1);
         float x[4] = {__uint_as_float(v0[i]) * scale2, __uint_as_float(v0[i + 2]) * scale2,
                       __uint_as_float(v1[i]) * scale2, __uint_as_float(v1[i + 2]) * scale2};
         bool vis[4];
