@@ -13,6 +13,7 @@ workload; there is no exchange step on this path, so the job throughput is the s
 from __future__ import annotations
 
 import argparse
+import concurrent.futures
 import json
 import os
 import sys
@@ -219,6 +220,7 @@ def main():
                          "default: one call for all layers, the layer axis of a [layers*B, H, L, d] cache "
                          "passed as the batch axis")
     ap.set_defaults(fold_layers=True)
+    ap.add_argument("--e2e-lanes", type=int, default=2, help="host threads (each with a stream and a staging area) of the end-to-end measurement")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-baseline-units", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -424,13 +426,26 @@ def main():
                              mod_out=pin(lb.mod_out), n_out=pin(lb.n_out)))
         h_mod, h_lens, h_bud = pin(mod), pin(lens), pin(bud)
         h_tot = None if tot is None else pin(tot)
-        staging = torch.empty(csp.host_staging_bytes(p), dtype=torch.uint8, device=dev)
+        # Two host threads, each with its own stream and staging area, take alternate layers: the call is
+        # synchronous, so this is what lets one layer's device-to-host copy run beside the next one's
+        # host-to-device copy (PCIe is full duplex) and beside its kernels.
+        n_lanes = max(1, args.e2e_lanes)
+        stagings = [torch.empty(csp.host_staging_bytes(p), dtype=torch.uint8, device=dev) for _ in range(n_lanes)]
+        lane_streams = [torch.cuda.Stream(device=dev) for _ in range(n_lanes)]
+
+        def lane_work(lane):
+            torch.cuda.set_device(dev)
+            with torch.cuda.stream(lane_streams[lane]):
+                for i in range(lane, n_layers, n_lanes):
+                    hb = host[i % n_host]
+                    csp.prune_layer_host(p, hb["q"], hb["k"], hb["v"], h_mod, h_lens, h_bud, hb["k_out"],
+                                         hb["v_out"], hb["mod_out"], hb["n_out"], stagings[lane], total_budget=h_tot)
+
+        pool = concurrent.futures.ThreadPoolExecutor(max_workers=n_lanes)
 
         def host_step():
-            for i in range(n_layers):
-                hb = host[i % n_host]
-                csp.prune_layer_host(p, hb["q"], hb["k"], hb["v"], h_mod, h_lens, h_bud, hb["k_out"], hb["v_out"],
-                                     hb["mod_out"], hb["n_out"], staging, total_budget=h_tot)
+            for f in [pool.submit(lane_work, lane) for lane in range(n_lanes)]:
+                f.result()                      # every call has synchronised its stream before returning
 
         with torch.cuda.stream(stream):
             host_step()
@@ -441,16 +456,18 @@ def main():
             e0.record(stream)
             for _ in range(args.e2e_steps):
                 host_step()
-            e1.record(stream)
+            e1.record(stream)                   # all lanes are idle again: the interval covers every copy and kernel
             stream.synchronize()
             ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
+        pool.shutdown()
         ms_e2e = max_over_ranks(ms_e2e, dist, dev)
         hb = host[0]
         h2d = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("q", "k", "v")) + \
             n_layers * (h_mod.numel() + 4 * h_lens.numel() + 4 * h_bud.numel())
         d2h = n_layers * sum(hb[x].numel() * hb[x].element_size() for x in ("k_out", "v_out", "mod_out", "n_out"))
         e2e = {"value": job_throughput(world, sum_l, n_layers, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "api": "csp_prune_layer_host"}
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "api": "csp_prune_layer_host",
+               "host_threads": n_lanes}
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N=1 only ----
     cpu_baseline = None
