@@ -325,3 +325,39 @@ int orc_prune_layer(const orc_params* p, const void* q, const void* k, const voi
     if (rc) return rc;
     return orc_compact(p, k, v, modality, mod_per_head, keep_idx, n_out, k_out, v_out, mod_out);
 }
+
+/* Section 3.3 / Eq. 7 applied to one decode query per head: logits over the rows of the pruned cache,
+ * n-softmax weights (orc_nsoftmax), weighted sum of the value rows. */
+int orc_decode_attn(const orc_params* p, const void* q, const void* k, const void* v,
+                    const int32_t* n_rows, double* out) {
+    const int64_t d = p->head_dim, cap = p->out_capacity;
+    const int G = p->n_q_heads / p->n_kv_heads;
+    const double scale = p->scale > 0.0 ? p->scale : 1.0 / sqrt((double)d);
+    int bad = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < p->batch; ++b) {
+        for (int hq = 0; hq < p->n_q_heads; ++hq) {
+            const int hkv = hq / G;
+            const int64_t rows = n_rows[(int64_t)b * p->n_kv_heads + hkv];
+            double* o_vec = out + ((int64_t)b * p->n_q_heads + hq) * d;
+            for (int64_t c = 0; c < d; ++c) o_vec[c] = 0.0;
+            if (rows < 0 || rows > cap) { bad = 1; continue; }
+            if (rows == 0) continue;
+            const int64_t qbase = ((int64_t)b * p->n_q_heads + hq) * d;
+            const int64_t kbase = ((int64_t)b * p->n_kv_heads + hkv) * cap * d;
+            double* o = (double*)malloc(sizeof(double) * (size_t)rows);
+            double* a = (double*)malloc(sizeof(double) * (size_t)rows);
+            for (int64_t t = 0; t < rows; ++t) {
+                double acc = 0.0;
+                for (int64_t c = 0; c < d; ++c)
+                    acc += load_elem(q, qbase + c, p->dtype) * load_elem(k, kbase + t * d + c, p->dtype);
+                o[t] = acc * scale;
+            }
+            orc_nsoftmax(o, rows, p->n, a);
+            for (int64_t t = 0; t < rows; ++t)
+                for (int64_t c = 0; c < d; ++c) o_vec[c] += a[t] * load_elem(v, kbase + t * d + c, p->dtype);
+            free(o); free(a);
+        }
+    }
+    return bad ? -1 : 0;
+}

@@ -3,7 +3,8 @@
  *
  * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, double-precision
  * restatement of what the paper defines (Eq. 1-4, Eq. 5, Eq. 7, Algorithm 1).
- * It exists to check the CUDA library and to be timed as a CPU baseline.  It
+ * It also holds the plain definition of decode attention with the n-softmax
+ * normaliser (Section 3.3).  It exists to check the CUDA library and to be timed as a CPU baseline.  It
  * shares no code with the CUDA library and must never be called from it.
  *
  * Every function has at least one independent pin in the CPU test-suite
@@ -90,6 +91,16 @@ int orc_prune_layer(const orc_params* p, const void* q, const void* k, const voi
                     float* score_self, float* score_cross,
                     int32_t* keep_idx, int32_t* n_out, int32_t* flags, float* margins,
                     void* k_out, void* v_out, uint8_t* mod_out);
+
+/* Attention of one new query per head over a pruned cache, with the n-softmax of Eq. 7 as the
+ * normaliser (Section 3.3: the denominator keeps the constant n for the mass that pruning removed):
+ *   o_t = scale <q[b,hq,:], k[b,hkv,t,:]>,  t < n_rows[b,hkv]   (hkv = hq / (Hq / Hkv))
+ *   out[b,hq,:] = sum_t  e^{o_t} / (n + sum_j e^{o_j})  v[b,hkv,t,:]
+ * q: [B, Hq, d]; k, v: [B, Hkv, out_capacity, d]; n_rows: [B, Hkv] (rows beyond it are ignored);
+ * out: [B, Hq, d] doubles.  A head with no rows gives a zero vector.  Returns 0, or -1 on a bad
+ * argument (n_rows outside [0, out_capacity]). */
+int orc_decode_attn(const orc_params* p, const void* q, const void* k, const void* v,
+                    const int32_t* n_rows, double* out);
 
 /* number of OpenMP threads the unit loops will use */
 int orc_num_threads(void);

@@ -204,3 +204,15 @@ def prune_layer(p: Params, q, k, v, modality, seq_lens, budgets, total_budget=No
     if rc:
         raise ValueError("orc_prune_layer: bad argument")
     return out
+
+
+def decode_attn(p: Params, q, k, v, n_rows):
+    """Section 3.3: one query per head over the pruned cache with the n-softmax normaliser.
+    q [B, Hq, d]; k, v [B, Hkv, out_capacity, d]; n_rows [B, Hkv] -> float64 [B, Hq, d]."""
+    q, k, v = _np(q, _elem(p)), _np(k, _elem(p)), _np(v, _elem(p))
+    n_rows = _np(n_rows, np.int32)
+    out = np.zeros((p.batch, p.n_q_heads, p.head_dim), np.float64)
+    cp = p.c()
+    if lib().orc_decode_attn(C.byref(cp), _ptr(q), _ptr(k), _ptr(v), _ptr(n_rows), _ptr(out)):
+        raise ValueError("orc_decode_attn: bad argument")
+    return out

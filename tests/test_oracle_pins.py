@@ -393,6 +393,109 @@ def test_short_sequence_is_identity(oracle):
 
 # ---------------------------------------------------------------- input generator sanity
 
+# ---------------------------------------------------------------- Section 3.3: n-softmax decode attention
+
+def _decode_case(oracle, seed, B=2, Hq=6, Hkv=2, d=16, cap=37, dtype=torch.float32, gain=1.0, **pk):
+    rng = np.random.RandomState(seed)
+    q = (torch.from_numpy(rng.randn(B, Hq, d).astype(np.float32)) * gain).to(dtype)
+    k = torch.from_numpy(rng.randn(B, Hkv, cap, d).astype(np.float32)).to(dtype)
+    v = torch.from_numpy(rng.randn(B, Hkv, cap, d).astype(np.float32)).to(dtype)
+    rows = rng.randint(1, cap + 1, size=(B, Hkv)).astype(np.int32)
+    p = oracle.Params(B, Hq, Hkv, d, 1, 0, cap, cap, dtype=oracle.F32 if dtype == torch.float32 else oracle.BF16, **pk)
+    return p, q, k, v, rows
+
+
+def test_decode_n0_is_library_attention(oracle):
+    """With n = 0 the normaliser is the plain softmax: torch's scaled_dot_product_attention per head."""
+    p, q, k, v, rows = _decode_case(oracle, 40, n=0.0)
+    out = oracle.decode_attn(p, q, k, v, rows)
+    G = p.n_q_heads // p.n_kv_heads
+    for b in range(p.batch):
+        for hq in range(p.n_q_heads):
+            r = int(rows[b, hq // G])
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                q[b, hq][None, None].double(), k[b, hq // G, :r][None].double(), v[b, hq // G, :r][None].double())
+            np.testing.assert_allclose(out[b, hq], ref[0, 0].numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_decode_n1_is_attention_with_one_extra_zero_key(oracle):
+    """n = 1 equals ordinary softmax attention over the cache plus one key with logit 0 and a zero value row
+    (the slot that holds the mass of what pruning removed)."""
+    p, q, k, v, rows = _decode_case(oracle, 41, n=1.0, gain=2.0)
+    out = oracle.decode_attn(p, q, k, v, rows)
+    G = p.n_q_heads // p.n_kv_heads
+    for b in range(p.batch):
+        for hq in range(p.n_q_heads):
+            r = int(rows[b, hq // G])
+            kk = torch.cat([k[b, hq // G, :r], torch.zeros(1, p.head_dim)]).double()     # q . 0 = logit 0
+            vv = torch.cat([v[b, hq // G, :r], torch.zeros(1, p.head_dim)]).double()
+            w = scipy_softmax((kk @ q[b, hq].double()).numpy() / np.sqrt(p.head_dim))
+            np.testing.assert_allclose(out[b, hq], w @ vv.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_decode_zero_query_closed_form(oracle):
+    """q = 0: every logit is 0, every weight 1 / (n + rows), the output is the column sum of V over n + rows."""
+    p, q, k, v, rows = _decode_case(oracle, 42, n=3.0)
+    out = oracle.decode_attn(p, torch.zeros_like(q), k, v, rows)
+    G = p.n_q_heads // p.n_kv_heads
+    for b in range(p.batch):
+        for hq in range(p.n_q_heads):
+            r = int(rows[b, hq // G])
+            want = [float(sum(Fraction(float(x)) for x in v[b, hq // G, :r, c]) / (3 + r)) for c in range(p.head_dim)]
+            np.testing.assert_allclose(out[b, hq], want, rtol=1e-13, atol=1e-15)
+
+
+def test_decode_restores_pre_pruning_weights(oracle):
+    """Eq. 6 -> Eq. 7: if n equals the exponential mass of the rows that were removed, attention over the kept
+    rows gives exactly the kept rows' share of full softmax attention over all rows."""
+    p, q, k, v, rows = _decode_case(oracle, 43, B=1, Hq=2, Hkv=2, cap=29, n=0.0)
+    rows[:] = 29
+    keep = 11
+    for h in range(2):
+        o = (k[0, h].double() @ q[0, h].double()).numpy() / np.sqrt(p.head_dim)
+        w_full = scipy_softmax(o)
+        want = w_full[:keep] @ v[0, h, :keep].double().numpy()
+        removed_mass = float(np.exp(o[keep:]).sum())
+        ph = oracle.Params(1, 1, 1, p.head_dim, 1, 0, 29, 29, dtype=oracle.F32, n=removed_mass)
+        got = oracle.decode_attn(ph, q[:, h:h + 1], k[:, h:h + 1], v[:, h:h + 1], np.array([[keep]], np.int32))
+        np.testing.assert_allclose(got[0, 0], want, rtol=1e-10, atol=1e-12)
+
+
+def test_decode_rows_beyond_n_rows_and_head_mapping(oracle):
+    """Rows past n_rows never matter; query head hq reads KV head hq // G; empty heads give zeros."""
+    p, q, k, v, rows = _decode_case(oracle, 44)
+    out = oracle.decode_attn(p, q, k, v, rows)
+    k2, v2 = k.clone(), v.clone()
+    for b in range(p.batch):
+        for h in range(p.n_kv_heads):
+            k2[b, h, rows[b, h]:] = 1e6
+            v2[b, h, rows[b, h]:] = -1e6
+    np.testing.assert_array_equal(oracle.decode_attn(p, q, k2, v2, rows), out)
+    # swapping the two KV heads together with the two groups of query heads swaps the outputs
+    G = p.n_q_heads // p.n_kv_heads
+    perm = list(range(G, 2 * G)) + list(range(G))
+    out_sw = oracle.decode_attn(p, q[:, perm], k.flip(1), v.flip(1), rows[:, ::-1].copy())
+    np.testing.assert_array_equal(out_sw, out[:, perm])
+    rows0 = rows.copy(); rows0[0, 0] = 0
+    assert (oracle.decode_attn(p, q, k, v, rows0)[0, :G] == 0).all()
+    # a transposed operand (q.k over the wrong axis) or a missing 1/sqrt(d) would break this closed form:
+    # one row only -> out = v_0 * e^o / (n + e^o)
+    one = np.ones_like(rows)
+    got = oracle.decode_attn(p, q, k, v, one)
+    for b in range(p.batch):
+        for hq in range(p.n_q_heads):
+            o = float(q[b, hq].double() @ k[b, hq // G, 0].double()) / np.sqrt(p.head_dim)
+            np.testing.assert_allclose(got[b, hq], v[b, hq // G, 0].double().numpy() * np.exp(o) / (1.0 + np.exp(o)),
+                                       rtol=1e-12, atol=1e-15)
+
+
+def test_decode_bf16_inputs_are_widened_exactly(oracle):
+    p, q, k, v, rows = _decode_case(oracle, 45, dtype=torch.bfloat16)
+    p32 = oracle.Params(**{**p.__dict__, "dtype": oracle.F32})
+    np.testing.assert_array_equal(oracle.decode_attn(p, q, k, v, rows),
+                                  oracle.decode_attn(p32, q.float(), k.float(), v.float(), rows))
+
+
 def test_benchmark_shapes_match_their_description():
     c1 = synth.config(1)
     assert c1.seq_lens.tolist() == [4096] and c1.budgets.tolist() == [[304, 0, 0, 691]]
