@@ -167,6 +167,28 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
                            int32_t* keep_idx_or_null,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Bytes of scratch that csp_decode_attn needs (status word + per-split partial results).  The first
+ * 256 bytes must be zero before first use (csp_workspace_reset). */
+size_t csp_decode_workspace_bytes(const csp_params* p);
+
+/*
+ * Section 3.3, Eq. 6-7: attention of ONE new query per head over a pruned cache, normalised with the
+ * n-softmax, whose constant n stands for the exponential mass of the rows that pruning removed:
+ *   out[b,hq,:] = sum_{t < n_rows[b,hkv]} e^{o_t} / (n + sum_j e^{o_j}) v[b,hkv,t,:],
+ *   o_t = scale <q[b,hq,:], k[b,hkv,t,:]>,  hkv = hq / (H_q / H_kv).
+ *   q       [B, H_q, d] (stride_b, stride_h; stride_t is not used), bf16
+ *   k, v    [B, H_kv, out_capacity, d] bf16: the k_out / v_out of csp_prune_layer (or any cache of that
+ *           layout); p->out_capacity is the row capacity, p->max_len / window / recent are not used
+ *   n_rows  [B, H_kv] int32 device: valid rows per head (the n_out of the prune); values outside
+ *           [0, out_capacity] are clamped and flagged CSP_DEV_BAD_LEN; 0 rows give a zero vector
+ *   out     [B, H_q, d] fp32, dense
+ * bf16 caches with head_dim 64 or 128 only (CSP_ERR_UNSUPPORTED otherwise).  Nothing is allocated; the
+ * caller owns the workspace; the work is enqueued on the stream.
+ */
+csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_tensor v,
+                           const int32_t* n_rows, float* out,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Bytes of device staging that csp_prune_layer_host needs for these parameters. */
 size_t csp_host_staging_bytes(const csp_params* p);
 

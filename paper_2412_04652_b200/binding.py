@@ -25,7 +25,8 @@ DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
 
 EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_select", "csp_compact",
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
-           "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit")
+           "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
+           "csp_decode_workspace_bytes", "csp_decode_attn")
 
 
 class CspError(RuntimeError):
@@ -110,6 +111,10 @@ def lib() -> C.CDLL:
                                              CTensor, CTensor, vp, vp, vp, vp]
         l.csp_static_workspace_limit.restype = sz
         l.csp_static_workspace_limit.argtypes = []
+        l.csp_decode_workspace_bytes.restype = sz
+        l.csp_decode_workspace_bytes.argtypes = [P]
+        l.csp_decode_attn.restype = C.c_int
+        l.csp_decode_attn.argtypes = [P, CTensor, CTensor, CTensor, vp, vp, vp, sz, vp]
         l.csp_device_status.restype = C.c_int
         l.csp_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         l.csp_status_string.restype = C.c_char_p
@@ -164,6 +169,28 @@ def new_workspace(p: Params, device="cuda") -> torch.Tensor:
 
 def workspace_reset(ws: torch.Tensor):
     _check(lib().csp_workspace_reset(_ptr(ws), _stream()), "csp_workspace_reset")
+
+
+def decode_workspace_bytes(p: Params) -> int:
+    cp = p.c()
+    return int(lib().csp_decode_workspace_bytes(C.byref(cp)))
+
+
+def new_decode_workspace(p: Params, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and zeroes a workspace for csp_decode_attn."""
+    n = decode_workspace_bytes(p)
+    if n == 0:
+        raise CspError(ERR_UNSUPPORTED, "csp_decode_workspace_bytes")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def decode_attn(p: Params, q, k, v, n_rows, out, ws):
+    """q [B, Hq, d]; k, v [B, Hkv, out_capacity, d]; n_rows int32 [B, Hkv]; out fp32 [B, Hq, d] (dense)."""
+    cp = p.c()
+    assert q.dim() == 3 and q.stride(2) == 1 and out.is_contiguous() and out.dtype == torch.float32
+    qt = CTensor(q.data_ptr(), q.stride(0), q.stride(1), q.shape[2])
+    _check(lib().csp_decode_attn(C.byref(cp), qt, tensor4(k), tensor4(v), _ptr(n_rows), _ptr(out), _ptr(ws),
+                                 ws.numel(), _stream()), "csp_decode_attn")
 
 
 def score(p: Params, q_win, k, modality, seq_lens, score_self, score_cross, ws, lse=None):

@@ -298,6 +298,24 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
     return CSP_OK;
 }
 
+size_t csp_decode_workspace_bytes(const csp_params* p) {
+    if (check_params(p) != CSP_OK) return 0;
+    return decode_workspace_bytes(*p);
+}
+
+csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_tensor v, const int32_t* n_rows,
+                           float* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!q.ptr || !k.ptr || !v.ptr || !n_rows || !out) return CSP_ERR_INVALID_ARG;
+    if (p->dtype != CSP_BF16 || (p->head_dim != 64 && p->head_dim != 128)) return CSP_ERR_UNSUPPORTED;
+    if (!tensor_ok(*p, q) || !tensor_ok(*p, k) || !tensor_ok(*p, v)) return CSP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < decode_workspace_bytes(*p) || (uintptr_t(workspace) % 256))
+        return CSP_ERR_WORKSPACE;
+    if ((st = check_arch()) != CSP_OK) return st;
+    return launch_decode_attn(*p, q, k, v, n_rows, out, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
 csp_status csp_device_status(void* workspace, void* cuda_stream, int32_t* host_out) {
     if (!workspace) return CSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

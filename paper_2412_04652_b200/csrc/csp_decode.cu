@@ -1,0 +1,340 @@
+// Decode attention over a pruned cache with the n-softmax normaliser (Section 3.3, Eq. 6-7): one new query
+// per head attends to the n_rows[b, h_kv] rows that a prune left,
+//   out[b, h_q, :] = sum_t  e^{o_t} / (n + sum_j e^{o_j})  v[b, h_kv, t, :],   o_t = scale <q, k_t>.
+//
+// The work is one pass over K and V: HBM-bound (512 bytes per cached row and KV head at d = 128).  The rows of a
+// (sequence, KV head) unit are split over several CTAs so that a small batch still fills the GPU; every CTA
+// leaves an un-normalised partial result (reference exponent m, sum l, weighted value sum) and a second small
+// kernel merges the partials and divides by n 2^-m + l.
+//
+// Inside a CTA
+//   warp 4      one thread streams 64-row tiles of K and V with TMA (128-byte swizzle, no multicast) through a
+//               ring of shared-memory stages, bounded waits on full/empty mbarriers
+//   warps 0-3   each owns 16 rows of every tile.  The G query heads that share the KV head are the M rows of a
+//               bf16 m16n8k16 mma (padded to 16): S = Q K^T from ldmatrix fragments, streaming softmax in the
+//               base-2 domain with a lazily raised reference, then P V with P split into a bf16 head and a bf16
+//               remainder (two mma per fragment) so that the weights keep fp32-like accuracy.
+// This is a skinny contraction (at most 8 query rows per key): the legacy warp-level mma is ample for an
+// HBM-bound stream, and tensor memory would add nothing.
+#include <mutex>
+
+#include "csp_device.cuh"
+#include "csp_internal.cuh"
+
+namespace csp {
+namespace {
+using namespace dev;
+
+constexpr int kDecTile = 64;                       // rows per stage
+constexpr int kDecWarps = 4;                       // consumer warps, 16 rows of every tile each
+constexpr int kDecThreads = 32 * (kDecWarps + 1);
+constexpr int kDecStages = 3;
+constexpr int kDecBlock = kDecTile * 128;          // bytes of one 64-column block of a tile
+
+struct DecodeArgs {
+    const void* q; int64_t q_sb, q_sh;             // element strides of [B, Hq, d]
+    const int32_t* n_rows;                         // [B, Hkv]
+    float* partial;                                // [units, splits, G, d + 2]
+    float* out;                                    // [B, Hq, d]
+    int32_t* status;
+    int32_t n_kv_heads, group, head_dim, capacity, splits, tiles_per_split;
+    float n, scale_log2;
+};
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D += A B with A = (a0, 0, a2, 0): rows 8-15 of the 16-row operand are padding
+__device__ __forceinline__ void mma_rows8(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+// two floats -> packed bf16 pair (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <int NH>   // head_dim = 64 NH
+__global__ void __launch_bounds__(kDecThreads, 2)
+decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                   const DecodeArgs a) {
+    constexpr int D = 64 * NH;
+    constexpr int KS = D / 16;                     // k-steps of S = Q K^T
+    constexpr int NT = D / 8;                      // 8-column tiles of the output
+    constexpr uint32_t kTileBytes = NH * kDecBlock;           // K (or V) of one stage
+    constexpr uint32_t kStageBytes = 2 * kTileBytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    float* const merge = reinterpret_cast<float*>(base_ptr + kDecStages * kStageBytes);     // [warp][8][D + 2]
+    const uint32_t full_bar = base + kDecStages * kStageBytes + kDecWarps * 8 * (D + 2) * 4;
+    const uint32_t empty_bar = full_bar + 8 * kDecStages;
+    volatile int* const abort_flag = reinterpret_cast<volatile int*>(base_ptr + kDecStages * kStageBytes +
+                                                                     kDecWarps * 8 * (D + 2) * 4 + 16 * kDecStages);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sp = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int u = b * a.n_kv_heads + h;
+    int rows = a.n_rows[u];
+    if (rows < 0 || rows > a.capacity) {
+        if (tid == 0 && sp == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
+        rows = rows < 0 ? 0 : a.capacity;
+    }
+    const int tiles = (rows + kDecTile - 1) / kDecTile;
+    const int tile0 = sp * a.tiles_per_split;
+    const int tile1 = min(tiles, tile0 + a.tiles_per_split);
+    if (tile0 >= tile1) return;                    // nothing for this split: the merge kernel skips it too
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < kDecStages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, kDecWarps); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kDecWarps) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            for (int it = 0; it < tile1 - tile0; ++it) {
+                const int s = it % kDecStages;
+                mbar_wait(empty_bar + 8 * s, (uint32_t(it / kDecStages) & 1u) ^ 1u, abort_flag);
+                if (*abort_flag) break;
+                mbar_expect_tx(full_bar + 8 * s, kStageBytes);
+                const int row = (tile0 + it) * kDecTile;
+#pragma unroll
+                for (int hb = 0; hb < NH; ++hb) {
+                    tma_load_4d(base + s * kStageBytes + hb * kDecBlock, &tmap_k, full_bar + 8 * s, hb * 64, row, h, b);
+                    tma_load_4d(base + s * kStageBytes + kTileBytes + hb * kDecBlock, &tmap_v, full_bar + 8 * s, hb * 64, row, h, b);
+                }
+            }
+            if (*abort_flag) {
+                // let copies that were issued land before the CTA's shared memory is given up
+                for (int s = 0; s < kDecStages; ++s) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_bar + 8 * s, 0) && !mbar_try_wait(full_bar + 8 * s, 1) &&
+                           global_ns() - t0 < kWaitLimitNs / 8) {}
+                }
+            }
+        }
+    } else {
+        // =============================== consumer warps ===============================
+        const int g = lane >> 2, qd = lane & 3;    // this thread's query row and column pair
+        const int G = a.group;
+        // Q fragments: row g, columns 16 ks + 2 qd + {0,1} and + 8
+        uint32_t qa0[KS], qa2[KS];
+        {
+            const uint16_t* qrow = static_cast<const uint16_t*>(a.q) + int64_t(b) * a.q_sb + int64_t(h * G + g) * a.q_sh;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                qa0[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * qd) : 0u;
+                qa2[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * qd) : 0u;
+            }
+        }
+        float acc[NT][4];
+#pragma unroll
+        for (int t = 0; t < NT; ++t) { acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f; }
+        float m_run = kNeg, l_run = 0.f;           // reference exponent of row g, this thread's share of its sum
+
+        // ldmatrix row addresses: lane l supplies row (l % 8) of matrix (l / 8)
+        const int kr = warp * 16 + ((lane >> 4) << 3) + (lane & 7);      // K: matrices 2,3 are the second 8 rows
+        const int kc = (lane >> 3) & 1;                                  //    matrices 1,3 the second 8 columns
+        const int vr = warp * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);  // V: matrices 1,3 are the second 8 rows
+        const int vc = lane >> 4;                                        //    matrices 2,3 the next 8 columns
+
+        for (int it = 0; it < tile1 - tile0; ++it) {
+            const int s = it % kDecStages;
+            mbar_wait(full_bar + 8 * s, uint32_t(it / kDecStages) & 1u, abort_flag);
+            const uint32_t k_s = base + s * kStageBytes, v_s = k_s + kTileBytes;
+            const int row_w = (tile0 + it) * kDecTile + warp * 16;       // first row of this warp's slice
+            if (row_w + 16 > rows) {
+                // Rows past the end hold whatever the cache holds: their weights are zero, but zero times a
+                // non-finite value is not, so clear this warp's value rows beyond the end.
+                for (int i = lane; i < 16 * NH * 8; i += 32) {
+                    const int r = warp * 16 + i / (NH * 8), c = i % (NH * 8);
+                    if ((tile0 + it) * kDecTile + r >= rows)
+                        *reinterpret_cast<uint4*>(base_ptr + (v_s - base) + (c >> 3) * kDecBlock + r * 128 +
+                                                  (((c & 7) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                }
+                __syncwarp();
+            }
+            // ---- S = Q K^T for 16 rows: two 8-row tiles
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const int chunk = ks * 2 + kc;
+                uint32_t kb[4];
+                ldsm_x4(kb, k_s + (chunk >> 3) * kDecBlock + kr * 128 + (((chunk & 7) ^ (kr & 7)) << 4));
+                mma_rows8(s0, qa0[ks], qa2[ks], kb[0], kb[1]);
+                mma_rows8(s1, qa0[ks], qa2[ks], kb[2], kb[3]);
+            }
+            // ---- streaming softmax of row g over rows row_w + {2 qd, 2 qd + 1, 8 + 2 qd, 9 + 2 qd}
+            const int r0 = row_w + 2 * qd;
+            float x[4] = {r0 < rows ? s0[0] * a.scale_log2 : kNeg, r0 + 1 < rows ? s0[1] * a.scale_log2 : kNeg,
+                          r0 + 8 < rows ? s1[0] * a.scale_log2 : kNeg, r0 + 9 < rows ? s1[1] * a.scale_log2 : kNeg};
+            float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            if (mx > m_run + kLazy) {              // same decision in the four lanes of a row
+                const float alpha = ex2f(m_run - mx);
+                l_run *= alpha;
+#pragma unroll
+                for (int t = 0; t < NT; ++t) { acc[t][0] *= alpha; acc[t][1] *= alpha; }
+                m_run = mx;
+            }
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = x[i] > 0.5f * kNeg ? ex2f(x[i] - m_run) : 0.f;
+            l_run += (p[0] + p[1]) + (p[2] + p[3]);
+            // weights as bf16 head + bf16 remainder
+            const uint32_t ph0 = pack_bf16(p[0], p[1]), ph2 = pack_bf16(p[2], p[3]);
+            const uint32_t pl0 = pack_bf16(p[0] - __uint_as_float(ph0 << 16), p[1] - __uint_as_float(ph0 & 0xffff0000u));
+            const uint32_t pl2 = pack_bf16(p[2] - __uint_as_float(ph2 << 16), p[3] - __uint_as_float(ph2 & 0xffff0000u));
+            // ---- acc += P V
+#pragma unroll
+            for (int t = 0; t < NT; t += 2) {
+                const int chunk = t + vc;
+                uint32_t vb[4];
+                ldsm_x4_t(vb, v_s + (chunk >> 3) * kDecBlock + vr * 128 + (((chunk & 7) ^ (vr & 7)) << 4));
+                mma_rows8(acc[t], ph0, ph2, vb[0], vb[1]);
+                mma_rows8(acc[t], pl0, pl2, vb[0], vb[1]);
+                mma_rows8(acc[t + 1], ph0, ph2, vb[2], vb[3]);
+                mma_rows8(acc[t + 1], pl0, pl2, vb[2], vb[3]);
+            }
+            if (row_w + 16 > rows) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar + 8 * s);
+        }
+        // row sum over the four lanes of a row; then this warp's (m, l, acc) to shared memory
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        float* const mine = merge + (warp * 8 + g) * (D + 2);
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            mine[t * 8 + 2 * qd] = acc[t][0];
+            mine[t * 8 + 2 * qd + 1] = acc[t][1];
+        }
+        if (qd == 0) { mine[D] = m_run; mine[D + 1] = l_run; }
+    }
+    __syncthreads();
+    if (*abort_flag) {
+        if (tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
+        return;
+    }
+    // merge the four warps (fixed order) and write this split's partial result
+    float* const part = a.partial + (int64_t(u) * a.splits + sp) * a.group * (D + 2);
+    for (int i = tid; i < a.group * (D + 2); i += kDecThreads) {
+        const int g = i / (D + 2), c = i % (D + 2);
+        float m = kNeg;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) m = fmaxf(m, merge[(w * 8 + g) * (D + 2) + D]);
+        float v = 0.f;
+        if (c == D) {
+            v = m;
+        } else {
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) {
+                const float* wm = merge + (w * 8 + g) * (D + 2);
+                v += wm[c] * ex2f(wm[D] - m);      // c == D + 1 sums the l's the same way
+            }
+        }
+        part[i] = v;
+    }
+}
+
+// out[b, hq, :] = sum_s acc_s 2^(m_s - m) / (n 2^-m + sum_s l_s 2^(m_s - m)) over the splits that had rows
+__global__ void decode_merge_kernel(const DecodeArgs a) {
+    const int u = blockIdx.x / a.group, g = blockIdx.x % a.group;
+    const int b = u / a.n_kv_heads, h = u % a.n_kv_heads;
+    const int D = a.head_dim;
+    int rows = a.n_rows[u];
+    rows = rows < 0 ? 0 : (rows > a.capacity ? a.capacity : rows);
+    const int tiles = (rows + kDecTile - 1) / kDecTile;
+    const int used = (tiles + a.tiles_per_split - 1) / a.tiles_per_split;
+    float* const o = a.out + (int64_t(b) * a.n_kv_heads * a.group + h * a.group + g) * D;
+    const float* const part = a.partial + (int64_t(u) * a.splits * a.group + g) * (D + 2);
+    const int64_t stride = int64_t(a.group) * (D + 2);
+    float m = kNeg;
+    for (int s = 0; s < used; ++s) m = fmaxf(m, part[s * stride + D]);
+    float l = 0.f;
+    for (int s = 0; s < used; ++s) l += part[s * stride + D + 1] * ex2f(part[s * stride + D] - m);
+    const float denom = a.n * ex2f(-m) + l;
+    for (int c = threadIdx.x; c < D; c += blockDim.x) {
+        float v = 0.f;
+        for (int s = 0; s < used; ++s) v += part[s * stride + c] * ex2f(part[s * stride + D] - m);
+        o[c] = (used > 0 && denom > 0.f) ? v / denom : 0.f;
+    }
+}
+
+}  // namespace
+
+int decode_splits(const csp_params& p) {
+    const int units = p.batch * p.n_kv_heads;
+    const int tiles = (p.out_capacity + kDecTile - 1) / kDecTile;
+    if (units <= 0 || tiles <= 0) return 1;
+    int splits = (2 * 2 * 148 + units - 1) / units;          // about two waves of two CTAs per SM
+    if (splits > tiles) splits = tiles;
+    return splits < 1 ? 1 : splits;
+}
+
+size_t decode_workspace_bytes(const csp_params& p) {
+    const size_t units = size_t(p.batch) * size_t(p.n_kv_heads);
+    const size_t G = size_t(p.n_q_heads / p.n_kv_heads);
+    return kStatusBytes + round256(units * size_t(decode_splits(p)) * G * size_t(p.head_dim + 2) * 4);
+}
+
+csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
+                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s) {
+    if (p.dtype != CSP_BF16 || (p.head_dim != 64 && p.head_dim != 128)) return CSP_ERR_UNSUPPORTED;
+    const int units = p.batch * p.n_kv_heads;
+    if (units == 0) return CSP_OK;
+    DecodeArgs a;
+    a.q = q.ptr; a.q_sb = q.stride_b; a.q_sh = q.stride_h;
+    a.n_rows = n_rows;
+    a.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
+    a.out = out;
+    a.status = static_cast<int32_t*>(ws);
+    a.n_kv_heads = p.n_kv_heads; a.group = p.n_q_heads / p.n_kv_heads; a.head_dim = p.head_dim;
+    a.capacity = p.out_capacity;
+    a.splits = decode_splits(p);
+    const int tiles = (p.out_capacity + kDecTile - 1) / kDecTile;
+    a.tiles_per_split = (tiles + a.splits - 1) / a.splits;
+    a.n = p.n;
+    a.scale_log2 = (p.scale > 0.f ? p.scale : 1.0f / sqrtf(float(p.head_dim))) * 1.4426950408889634f;
+    if (p.out_capacity > 0) {
+        CUtensorMap tk, tv;
+        if (!make_cache_tensor_map(&tk, k, p.dtype, p.head_dim, p.out_capacity, p.n_kv_heads, p.batch, kDecTile) ||
+            !make_cache_tensor_map(&tv, v, p.dtype, p.head_dim, p.out_capacity, p.n_kv_heads, p.batch, kDecTile))
+            return CSP_ERR_UNSUPPORTED;
+        const int NH = p.head_dim / 64;
+        const size_t smem = 1024 + size_t(kDecStages) * 2 * NH * kDecBlock + size_t(kDecWarps) * 8 * (p.head_dim + 2) * 4 +
+                            16 * kDecStages + 16;
+        auto kern = NH == 1 ? decode_attn_kernel<1> : decode_attn_kernel<2>;
+        static bool configured[2][64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
+        if (dev < 0 || dev >= 64 || !configured[NH - 1][dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
+                cudaGetLastError();
+                return CSP_ERR_CUDA;
+            }
+            if (dev >= 0 && dev < 64) configured[NH - 1][dev] = true;
+        }
+        kern<<<dim3(a.splits, p.n_kv_heads, p.batch), kDecThreads, smem, s>>>(tk, tv, a);
+        if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
+    }
+    decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
+}
+
+}  // namespace csp

@@ -101,4 +101,15 @@ constexpr int kSelectClusterMaxLen = 8 * 1024 * 8;   // longest cache the regist
 csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaStream_t s);
 csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_t s);
 
+// 4-D tensor map over a cache [batch, heads, rows, head_dim] with 128-byte swizzle and boxes of 128 bytes x
+// box_rows rows; false if the driver entry point is missing or the strides / alignment do not qualify.
+bool make_cache_tensor_map(CUtensorMap* map, const csp_tensor& t, int dtype, int head_dim, int rows, int heads,
+                           int batch, int box_rows);
+
+// decode attention over the pruned cache (csp_decode.cu)
+int decode_splits(const csp_params& p);
+size_t decode_workspace_bytes(const csp_params& p);
+csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
+                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s);
+
 }  // namespace csp

@@ -526,6 +526,25 @@ __global__ void length_order_kernel(const int32_t* __restrict__ seq_lens, int ba
 
 }  // namespace
 
+bool make_cache_tensor_map(CUtensorMap* map, const csp_tensor& t, int dtype, int head_dim, int rows, int heads,
+                           int batch, int box_rows) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return false;
+    const uint64_t es = dtype == CSP_F32 ? 4 : 2;
+    // sizes of 1 carry no usable stride: give them a legal one
+    const uint64_t st = uint64_t(t.stride_t) * es;
+    const uint64_t sh = heads > 1 ? uint64_t(t.stride_h) * es : st * uint64_t(rows);
+    const uint64_t sb = batch > 1 ? uint64_t(t.stride_b) * es : sh * uint64_t(heads);
+    if (t.stride_t < head_dim || (st % 16) || (sh % 16) || (sb % 16) || (uintptr_t(t.ptr) % 16)) return false;
+    const cuuint64_t dims[4] = {cuuint64_t(head_dim), cuuint64_t(rows), cuuint64_t(heads), cuuint64_t(batch)};
+    const cuuint64_t strides[3] = {st, sh, sb};
+    const cuuint32_t box[4] = {cuuint32_t(128 / es), cuuint32_t(box_rows), 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return encode(map, dtype == CSP_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, t.ptr,
+                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_tensor& k, cudaStream_t s) {
     ScoreArgs a = a_in;
     EncodeTiledFn encode = encode_tiled_fn();
