@@ -205,6 +205,102 @@ def kernels_per_call(p) -> int:
     return 4 if ordered else 3
 
 
+def run_decode(args, rank, world, local_rank):
+    """`--decode`: the step after the pruning pass (Section 3.3): one new query per head attends, with the
+    n-softmax normaliser, to the compacted caches that csp_prune_layer left.  All layers of the workload in one
+    csp_decode_attn call (layer axis folded into the batch axis).  Prints its own JSON line; not the default."""
+    from paper_2412_04652_b200 import binding as csp
+    csp.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = synth.config(args.config, budget_pct=args.budget_pct) if args.config == 4 else synth.config(args.config)
+    n_layers, cap = cfg.n_layers, cfg.out_capacity()
+    import copy
+    pf = csp.Params(cfg.batch * n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.recent,
+                    cfg.max_len, cap)
+    lb = LayerBuffers(csp, cfg, pf, 0, dev, n_fold=n_layers)
+    mod = torch.from_numpy(cfg.modality()).to(dev).repeat(n_layers, 1)
+    lens = torch.from_numpy(cfg.seq_lens).to(dev).repeat(n_layers)
+    bud = torch.from_numpy(cfg.budgets).to(dev).repeat(n_layers, 1)
+    tot = None if cfg.total_budget is None else torch.from_numpy(cfg.total_budget).to(dev).repeat(n_layers)
+    ws = csp.new_workspace(pf, dev)
+    csp.prune_layer(pf, lb.q, lb.k, lb.v, mod, lens, bud, lb.k_out, lb.v_out, lb.mod_out, lb.n_out, ws, total_budget=tot)
+    status = csp.device_status(ws)
+    k_c, v_c, n_rows = lb.k_out, lb.v_out, lb.n_out
+    del lb.k, lb.v
+    pd = csp.Params(pf.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, 1, 0, cap, cap)
+    g = torch.Generator(device=dev).manual_seed(1234)
+    q1 = torch.randn(pf.batch, cfg.n_q_heads, cfg.head_dim, generator=g, device=dev).to(torch.bfloat16)
+    out = torch.zeros(pf.batch, cfg.n_q_heads, cfg.head_dim, device=dev)
+    wd = csp.new_decode_workspace(pd, dev)
+    rows_total = int(n_rows.clamp(min=0).sum().item())
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            csp.decode_attn(pd, q1, k_c, v_c, n_rows, out, wd)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            csp.decode_attn(pd, q1, k_c, v_c, n_rows, out, wd)
+        graph.replay()
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        clocks = sampler.stop()
+    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    status |= csp.device_status(wd)
+    es = 2
+    ab = rows_total * 2 * cfg.head_dim * es + q1.numel() * es + out.numel() * 4 + n_rows.numel() * 4
+    peak, peak_kind = measured_peaks()
+    achieved = ab / (ms_step * 1e-3) / 1e9
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import csp_oracle as orc
+        orc.build()
+        po = orc.Params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, 1, 0, cap, cap, dtype=orc.BF16)
+        B0 = cfg.batch
+        qs, ks, vs, rs = q1[:B0].cpu(), k_c[:B0].cpu(), v_c[:B0].cpu(), n_rows[:B0].clamp(min=0).cpu().numpy()
+        t0 = time.perf_counter()
+        reps = 0
+        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 5000):
+            orc.decode_attn(po, qs, ks, vs, rs)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        cpu_baseline = {"value": float(rs.sum()) / dt, "unit": "kv_rows/s", "cores": orc.num_threads(),
+                        "kind": "oracle", "sample": f"all heads of one layer, {reps} repetitions, {dt:.4f} s each"}
+    if rank == 0:
+        line = {"metric": "decode_attn_kv_rows_per_sec", "value": world * rows_total / (ms_step * 1e-3), "unit": "kv_rows/s",
+                "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"decode over the pruned caches of configs[{args.config}] {cfg.name}",
+                           "layers": n_layers, "kv_heads": cfg.n_kv_heads, "q_heads": cfg.n_q_heads,
+                           "head_dim": cfg.head_dim, "row_capacity": cap, "kv_rows_per_step": rows_total,
+                           "launch": "one csp_decode_attn call for all layers (layer axis folded into the batch axis)",
+                           "l2": "inputs larger than L2" if ab > 2 * 126e6 else "inputs smaller than L2",
+                           "replicas": "one independent replica per GPU, no collective"},
+                "clocks": clocks, "e2e": None, "gpu_launches": args.steps * 2,
+                "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                             "algorithmic_bytes_per_launch": ab, "us_per_launch": ms_step * 1e3},
+                "cpu_baseline": cpu_baseline, "device_status": status}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -225,6 +321,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-baseline-units", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode", action="store_true",
+                    help="time the step after the pruning pass instead: n-softmax decode attention over the pruned caches")
     ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
     args = ap.parse_args()
 
@@ -240,6 +338,9 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    if args.decode:
+        run_decode(args, rank, world, local_rank)
+        return
     from paper_2412_04652_b200 import binding as csp
     csp.lib()
     torch.cuda.set_device(local_rank)

@@ -3,13 +3,14 @@
 //   out[b, h_q, :] = sum_t  e^{o_t} / (n + sum_j e^{o_j})  v[b, h_kv, t, :],   o_t = scale <q, k_t>.
 //
 // The work is one pass over K and V: HBM-bound (512 bytes per cached row and KV head at d = 128).  The rows of a
-// (sequence, KV head) unit are split over several CTAs so that a small batch still fills the GPU; every CTA
-// leaves an un-normalised partial result (reference exponent m, sum l, weighted value sum) and a second small
-// kernel merges the partials and divides by n 2^-m + l.
+// (sequence, KV head) unit are split into work items so that a small batch still fills the GPU; one CTA per SM
+// stays resident and walks over items; every item leaves an un-normalised partial result (reference exponent
+// m, sum l, weighted value sum) and a second small kernel merges the partials and divides by n 2^-m + l.
 //
 // Inside a CTA
 //   warp 4      one thread streams 64-row tiles of K and V with TMA (128-byte swizzle, no multicast) through a
-//               ring of shared-memory stages, bounded waits on full/empty mbarriers
+//               ring of six shared-memory stages, bounded waits on full/empty mbarriers; it runs ahead into the
+//               next item, so the stream does not drain between items
 //   warps 0-3   each owns 16 rows of every tile.  The G query heads that share the KV head are the M rows of a
 //               bf16 m16n8k16 mma (padded to 16): S = Q K^T from ldmatrix fragments, streaming softmax in the
 //               base-2 domain with a lazily raised reference, then P V with P split into a bf16 head and a bf16
@@ -28,7 +29,7 @@ using namespace dev;
 constexpr int kDecTile = 64;                       // rows per stage
 constexpr int kDecWarps = 4;                       // consumer warps, 16 rows of every tile each
 constexpr int kDecThreads = 32 * (kDecWarps + 1);
-constexpr int kDecStages = 3;
+constexpr int kDecStages = 6;                      // 32 KB each at d = 128: one resident CTA per SM
 constexpr int kDecBlock = kDecTile * 128;          // bytes of one 64-column block of a tile
 
 struct DecodeArgs {
@@ -37,6 +38,7 @@ struct DecodeArgs {
     float* partial;                                // [units, splits, G, d + 2]
     float* out;                                    // [B, Hq, d]
     int32_t* status;
+    int32_t* next_item;                            // work counter in the status area: zero between calls
     int32_t n_kv_heads, group, head_dim, capacity, splits, tiles_per_split;
     float n, scale_log2;
 };
@@ -63,10 +65,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+// barrier over the consumer threads (barrier 1) that also tells everyone whether any of them saw `pred`
+__device__ __forceinline__ bool consumers_any(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "barrier.cta.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(uint32_t(pred)), "n"(32 * kDecWarps) : "memory");
+    return r != 0;
+}
+
 template <int NH>   // head_dim = 64 NH
-__global__ void __launch_bounds__(kDecThreads, 2)
+__global__ void __launch_bounds__(kDecThreads, 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                   const DecodeArgs a) {
+                   const DecodeArgs a, const int n_items) {
     constexpr int D = 64 * NH;
     constexpr int KS = D / 16;                     // k-steps of S = Q K^T
     constexpr int NT = D / 8;                      // 8-column tiles of the output
@@ -77,23 +91,33 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
     float* const merge = reinterpret_cast<float*>(base_ptr + kDecStages * kStageBytes);     // [warp][8][D + 2]
-    const uint32_t full_bar = base + kDecStages * kStageBytes + kDecWarps * 8 * (D + 2) * 4;
+    const uint32_t full_bar = base + kDecStages * kStageBytes + kDecWarps * 8 * (D + 2) * 4;   // then: abort flag, item queue
     const uint32_t empty_bar = full_bar + 8 * kDecStages;
     volatile int* const abort_flag = reinterpret_cast<volatile int*>(base_ptr + kDecStages * kStageBytes +
                                                                      kDecWarps * 8 * (D + 2) * 4 + 16 * kDecStages);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sp = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int u = b * a.n_kv_heads + h;
-    int rows = a.n_rows[u];
-    if (rows < 0 || rows > a.capacity) {
-        if (tid == 0 && sp == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
-        rows = rows < 0 ? 0 : a.capacity;
-    }
-    const int tiles = (rows + kDecTile - 1) / kDecTile;
-    const int tile0 = sp * a.tiles_per_split;
-    const int tile1 = min(tiles, tile0 + a.tiles_per_split);
-    if (tile0 >= tile1) return;                    // nothing for this split: the merge kernel skips it too
+
+    // Work item = (unit, split): a contiguous range of 64-row tiles of one (sequence, KV head).  The CTA is
+    // resident; its producer thread draws items from a global counter (so ragged row counts balance by
+    // themselves), tells the consumers which item the next tiles belong to through a small queue in shared
+    // memory, and runs ahead into the next item while the consumers finish the current one.
+    constexpr int kQueue = 8;                      // > stages: the producer is at most kDecStages items ahead
+    volatile int* const item_q = abort_flag + 1;
+    struct Item { int u, b, h, sp, rows, tile0, n_tiles; };
+    auto item_of = [&](int w) {
+        Item x;
+        x.u = w / a.splits; x.sp = w % a.splits;
+        x.b = x.u / a.n_kv_heads; x.h = x.u % a.n_kv_heads;
+        int rows = a.n_rows[x.u];
+        rows = rows < 0 ? 0 : (rows > a.capacity ? a.capacity : rows);
+        x.rows = rows;
+        const int tiles = (rows + kDecTile - 1) / kDecTile;
+        x.tile0 = x.sp * a.tiles_per_split;
+        const int t1 = min(tiles, x.tile0 + a.tiles_per_split);
+        x.n_tiles = t1 > x.tile0 ? t1 - x.tile0 : 0;       // 0: nothing for this split, the merge kernel skips it too
+        return x;
+    };
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -106,17 +130,33 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (warp == kDecWarps) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
-            for (int it = 0; it < tile1 - tile0; ++it) {
+            int it = 0, j = 0;
+            while (!*abort_flag) {
+                const int w = atomicAdd(a.next_item, 1);
+                if (w >= n_items) break;
+                const Item x = item_of(w);
+                if (x.n_tiles == 0) continue;
+                for (int i = 0; i < x.n_tiles; ++i, ++it) {
+                    const int s = it % kDecStages;
+                    mbar_wait(empty_bar + 8 * s, (uint32_t(it / kDecStages) & 1u) ^ 1u, abort_flag);
+                    if (*abort_flag) break;
+                    if (i == 0) item_q[j % kQueue] = w;     // published by the arrive below (release)
+                    mbar_expect_tx(full_bar + 8 * s, kStageBytes);
+                    const int row = (x.tile0 + i) * kDecTile;
+#pragma unroll
+                    for (int hb = 0; hb < NH; ++hb) {
+                        tma_load_4d(base + s * kStageBytes + hb * kDecBlock, &tmap_k, full_bar + 8 * s, hb * 64, row, x.h, x.b);
+                        tma_load_4d(base + s * kStageBytes + kTileBytes + hb * kDecBlock, &tmap_v, full_bar + 8 * s, hb * 64, row, x.h, x.b);
+                    }
+                }
+                ++j;
+            }
+            if (!*abort_flag) {
+                // end marker: one more phase of the next stage's barrier, without data
                 const int s = it % kDecStages;
                 mbar_wait(empty_bar + 8 * s, (uint32_t(it / kDecStages) & 1u) ^ 1u, abort_flag);
-                if (*abort_flag) break;
-                mbar_expect_tx(full_bar + 8 * s, kStageBytes);
-                const int row = (tile0 + it) * kDecTile;
-#pragma unroll
-                for (int hb = 0; hb < NH; ++hb) {
-                    tma_load_4d(base + s * kStageBytes + hb * kDecBlock, &tmap_k, full_bar + 8 * s, hb * 64, row, h, b);
-                    tma_load_4d(base + s * kStageBytes + kTileBytes + hb * kDecBlock, &tmap_v, full_bar + 8 * s, hb * 64, row, h, b);
-                }
+                item_q[j % kQueue] = -1;
+                mbar_arrive(full_bar + 8 * s);
             }
             if (*abort_flag) {
                 // let copies that were issued land before the CTA's shared memory is given up
@@ -131,124 +171,135 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // =============================== consumer warps ===============================
         const int g = lane >> 2, qd = lane & 3;    // this thread's query row and column pair
         const int G = a.group;
-        // Q fragments: row g, columns 16 ks + 2 qd + {0,1} and + 8
-        uint32_t qa0[KS], qa2[KS];
-        {
-            const uint16_t* qrow = static_cast<const uint16_t*>(a.q) + int64_t(b) * a.q_sb + int64_t(h * G + g) * a.q_sh;
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                qa0[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * qd) : 0u;
-                qa2[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * qd) : 0u;
-            }
-        }
-        float acc[NT][4];
-#pragma unroll
-        for (int t = 0; t < NT; ++t) { acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f; }
-        float m_run = kNeg, l_run = 0.f;           // reference exponent of row g, this thread's share of its sum
-
         // ldmatrix row addresses: lane l supplies row (l % 8) of matrix (l / 8)
         const int kr = warp * 16 + ((lane >> 4) << 3) + (lane & 7);      // K: matrices 2,3 are the second 8 rows
         const int kc = (lane >> 3) & 1;                                  //    matrices 1,3 the second 8 columns
         const int vr = warp * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);  // V: matrices 1,3 are the second 8 rows
         const int vc = lane >> 4;                                        //    matrices 2,3 the next 8 columns
-
-        for (int it = 0; it < tile1 - tile0; ++it) {
-            const int s = it % kDecStages;
-            mbar_wait(full_bar + 8 * s, uint32_t(it / kDecStages) & 1u, abort_flag);
-            const uint32_t k_s = base + s * kStageBytes, v_s = k_s + kTileBytes;
-            const int row_w = (tile0 + it) * kDecTile + warp * 16;       // first row of this warp's slice
-            if (row_w + 16 > rows) {
-                // Rows past the end hold whatever the cache holds: their weights are zero, but zero times a
-                // non-finite value is not, so clear this warp's value rows beyond the end.
-                for (int i = lane; i < 16 * NH * 8; i += 32) {
-                    const int r = warp * 16 + i / (NH * 8), c = i % (NH * 8);
-                    if ((tile0 + it) * kDecTile + r >= rows)
-                        *reinterpret_cast<uint4*>(base_ptr + (v_s - base) + (c >> 3) * kDecBlock + r * 128 +
-                                                  (((c & 7) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+        auto consumers_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(32 * kDecWarps) : "memory"); };
+        int it = 0;
+        for (int j = 0;; ++j) {
+            // the first tile of the next item (or the end marker) tells which item it is
+            const bool ok = mbar_wait(full_bar + 8 * (it % kDecStages), uint32_t(it / kDecStages) & 1u, abort_flag);
+            const int w = ok ? item_q[j % kQueue] : -1;
+            if (consumers_any(w < 0)) break;       // end of work, or a wait gave up: all consumers leave together
+            const Item x = item_of(w);
+            const int rows = x.rows;
+            // Q fragments: row g, columns 16 ks + 2 qd + {0,1} and + 8
+            uint32_t qa0[KS], qa2[KS];
+            {
+                const uint16_t* qrow = static_cast<const uint16_t*>(a.q) + int64_t(x.b) * a.q_sb + int64_t(x.h * G + g) * a.q_sh;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    qa0[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * qd) : 0u;
+                    qa2[ks] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * qd) : 0u;
                 }
+            }
+            float acc[NT][4];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) { acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f; }
+            float m_run = kNeg, l_run = 0.f;       // reference exponent of row g, this thread's share of its sum
+
+            for (int i = 0; i < x.n_tiles; ++i, ++it) {
+                const int s = it % kDecStages;
+                mbar_wait(full_bar + 8 * s, uint32_t(it / kDecStages) & 1u, abort_flag);
+                const uint32_t k_s = base + s * kStageBytes, v_s = k_s + kTileBytes;
+                const int row_t = (x.tile0 + i) * kDecTile;              // first row of the tile
+                const int row_w = row_t + warp * 16;                     // first row of this warp's slice
+                if (row_w + 16 > rows) {
+                    // Rows past the end hold whatever the cache holds: their weights are zero, but zero times a
+                    // non-finite value is not, so clear this warp's value rows beyond the end.
+                    for (int j = lane; j < 16 * NH * 8; j += 32) {
+                        const int r = warp * 16 + j / (NH * 8), c = j % (NH * 8);
+                        if (row_t + r >= rows)
+                            *reinterpret_cast<uint4*>(base_ptr + (v_s - base) + (c >> 3) * kDecBlock + r * 128 +
+                                                      (((c & 7) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                    }
+                    __syncwarp();
+                }
+                // ---- S = Q K^T for 16 rows: two 8-row tiles
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int chunk = ks * 2 + kc;
+                    uint32_t kb[4];
+                    ldsm_x4(kb, k_s + (chunk >> 3) * kDecBlock + kr * 128 + (((chunk & 7) ^ (kr & 7)) << 4));
+                    mma_rows8(s0, qa0[ks], qa2[ks], kb[0], kb[1]);
+                    mma_rows8(s1, qa0[ks], qa2[ks], kb[2], kb[3]);
+                }
+                // ---- streaming softmax of row g over rows row_w + {2 qd, 2 qd + 1, 8 + 2 qd, 9 + 2 qd}
+                const int r0 = row_w + 2 * qd;
+                float xs[4] = {r0 < rows ? s0[0] * a.scale_log2 : kNeg, r0 + 1 < rows ? s0[1] * a.scale_log2 : kNeg,
+                               r0 + 8 < rows ? s1[0] * a.scale_log2 : kNeg, r0 + 9 < rows ? s1[1] * a.scale_log2 : kNeg};
+                float mx = fmaxf(fmaxf(xs[0], xs[1]), fmaxf(xs[2], xs[3]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                if (mx > m_run + kLazy) {          // same decision in the four lanes of a row
+                    const float alpha = ex2f(m_run - mx);
+                    l_run *= alpha;
+#pragma unroll
+                    for (int t = 0; t < NT; ++t) { acc[t][0] *= alpha; acc[t][1] *= alpha; }
+                    m_run = mx;
+                }
+                float p[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) p[j] = xs[j] > 0.5f * kNeg ? ex2f(xs[j] - m_run) : 0.f;
+                l_run += (p[0] + p[1]) + (p[2] + p[3]);
+                // weights as bf16 head + bf16 remainder
+                const uint32_t ph0 = pack_bf16(p[0], p[1]), ph2 = pack_bf16(p[2], p[3]);
+                const uint32_t pl0 = pack_bf16(p[0] - __uint_as_float(ph0 << 16), p[1] - __uint_as_float(ph0 & 0xffff0000u));
+                const uint32_t pl2 = pack_bf16(p[2] - __uint_as_float(ph2 << 16), p[3] - __uint_as_float(ph2 & 0xffff0000u));
+                // ---- acc += P V
+#pragma unroll
+                for (int t = 0; t < NT; t += 2) {
+                    const int chunk = t + vc;
+                    uint32_t vb[4];
+                    ldsm_x4_t(vb, v_s + (chunk >> 3) * kDecBlock + vr * 128 + (((chunk & 7) ^ (vr & 7)) << 4));
+                    mma_rows8(acc[t], ph0, ph2, vb[0], vb[1]);
+                    mma_rows8(acc[t], pl0, pl2, vb[0], vb[1]);
+                    mma_rows8(acc[t + 1], ph0, ph2, vb[2], vb[3]);
+                    mma_rows8(acc[t + 1], pl0, pl2, vb[2], vb[3]);
+                }
+                if (row_w + 16 > rows) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar + 8 * s);
             }
-            // ---- S = Q K^T for 16 rows: two 8-row tiles
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            // row sum over the four lanes of a row; then this warp's (m, l, acc) to shared memory
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+            float* const mine = merge + (warp * 8 + g) * (D + 2);
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                const int chunk = ks * 2 + kc;
-                uint32_t kb[4];
-                ldsm_x4(kb, k_s + (chunk >> 3) * kDecBlock + kr * 128 + (((chunk & 7) ^ (kr & 7)) << 4));
-                mma_rows8(s0, qa0[ks], qa2[ks], kb[0], kb[1]);
-                mma_rows8(s1, qa0[ks], qa2[ks], kb[2], kb[3]);
+            for (int t = 0; t < NT; ++t) {
+                mine[t * 8 + 2 * qd] = acc[t][0];
+                mine[t * 8 + 2 * qd + 1] = acc[t][1];
             }
-            // ---- streaming softmax of row g over rows row_w + {2 qd, 2 qd + 1, 8 + 2 qd, 9 + 2 qd}
-            const int r0 = row_w + 2 * qd;
-            float x[4] = {r0 < rows ? s0[0] * a.scale_log2 : kNeg, r0 + 1 < rows ? s0[1] * a.scale_log2 : kNeg,
-                          r0 + 8 < rows ? s1[0] * a.scale_log2 : kNeg, r0 + 9 < rows ? s1[1] * a.scale_log2 : kNeg};
-            float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            if (mx > m_run + kLazy) {              // same decision in the four lanes of a row
-                const float alpha = ex2f(m_run - mx);
-                l_run *= alpha;
+            if (qd == 0) { mine[D] = m_run; mine[D + 1] = l_run; }
+            consumers_sync();
+            const bool aborted = *abort_flag != 0;
+            // merge the four warps (fixed order) and write this split's partial result
+            if (!aborted) {
+                float* const part = a.partial + (int64_t(x.u) * a.splits + x.sp) * a.group * (D + 2);
+                for (int j = tid; j < a.group * (D + 2); j += 32 * kDecWarps) {
+                    const int gg = j / (D + 2), c = j % (D + 2);
+                    float m = kNeg;
 #pragma unroll
-                for (int t = 0; t < NT; ++t) { acc[t][0] *= alpha; acc[t][1] *= alpha; }
-                m_run = mx;
+                    for (int ww = 0; ww < kDecWarps; ++ww) m = fmaxf(m, merge[(ww * 8 + gg) * (D + 2) + D]);
+                    float v = 0.f;
+                    if (c == D) {
+                        v = m;
+                    } else {
+#pragma unroll
+                        for (int ww = 0; ww < kDecWarps; ++ww) {
+                            const float* wm = merge + (ww * 8 + gg) * (D + 2);
+                            v += wm[c] * ex2f(wm[D] - m);      // c == D + 1 sums the l's the same way
+                        }
+                    }
+                    part[j] = v;
+                }
             }
-            float p[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) p[i] = x[i] > 0.5f * kNeg ? ex2f(x[i] - m_run) : 0.f;
-            l_run += (p[0] + p[1]) + (p[2] + p[3]);
-            // weights as bf16 head + bf16 remainder
-            const uint32_t ph0 = pack_bf16(p[0], p[1]), ph2 = pack_bf16(p[2], p[3]);
-            const uint32_t pl0 = pack_bf16(p[0] - __uint_as_float(ph0 << 16), p[1] - __uint_as_float(ph0 & 0xffff0000u));
-            const uint32_t pl2 = pack_bf16(p[2] - __uint_as_float(ph2 << 16), p[3] - __uint_as_float(ph2 & 0xffff0000u));
-            // ---- acc += P V
-#pragma unroll
-            for (int t = 0; t < NT; t += 2) {
-                const int chunk = t + vc;
-                uint32_t vb[4];
-                ldsm_x4_t(vb, v_s + (chunk >> 3) * kDecBlock + vr * 128 + (((chunk & 7) ^ (vr & 7)) << 4));
-                mma_rows8(acc[t], ph0, ph2, vb[0], vb[1]);
-                mma_rows8(acc[t], pl0, pl2, vb[0], vb[1]);
-                mma_rows8(acc[t + 1], ph0, ph2, vb[2], vb[3]);
-                mma_rows8(acc[t + 1], pl0, pl2, vb[2], vb[3]);
-            }
-            if (row_w + 16 > rows) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar + 8 * s);
+            // the barrier at the top of the next item also frees the merge area
         }
-        // row sum over the four lanes of a row; then this warp's (m, l, acc) to shared memory
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        float* const mine = merge + (warp * 8 + g) * (D + 2);
-#pragma unroll
-        for (int t = 0; t < NT; ++t) {
-            mine[t * 8 + 2 * qd] = acc[t][0];
-            mine[t * 8 + 2 * qd + 1] = acc[t][1];
-        }
-        if (qd == 0) { mine[D] = m_run; mine[D + 1] = l_run; }
-    }
-    __syncthreads();
-    if (*abort_flag) {
-        if (tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
-        return;
-    }
-    // merge the four warps (fixed order) and write this split's partial result
-    float* const part = a.partial + (int64_t(u) * a.splits + sp) * a.group * (D + 2);
-    for (int i = tid; i < a.group * (D + 2); i += kDecThreads) {
-        const int g = i / (D + 2), c = i % (D + 2);
-        float m = kNeg;
-#pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) m = fmaxf(m, merge[(w * 8 + g) * (D + 2) + D]);
-        float v = 0.f;
-        if (c == D) {
-            v = m;
-        } else {
-#pragma unroll
-            for (int w = 0; w < kDecWarps; ++w) {
-                const float* wm = merge + (w * 8 + g) * (D + 2);
-                v += wm[c] * ex2f(wm[D] - m);      // c == D + 1 sums the l's the same way
-            }
-        }
-        part[i] = v;
+        if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
     }
 }
 
@@ -257,7 +308,9 @@ __global__ void decode_merge_kernel(const DecodeArgs a) {
     const int u = blockIdx.x / a.group, g = blockIdx.x % a.group;
     const int b = u / a.n_kv_heads, h = u % a.n_kv_heads;
     const int D = a.head_dim;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.next_item = 0;     // the work counter is zero again for the next call
     int rows = a.n_rows[u];
+    if ((rows < 0 || rows > a.capacity) && g == 0 && threadIdx.x == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
     rows = rows < 0 ? 0 : (rows > a.capacity ? a.capacity : rows);
     const int tiles = (rows + kDecTile - 1) / kDecTile;
     const int used = (tiles + a.tiles_per_split - 1) / a.tiles_per_split;
@@ -282,8 +335,9 @@ int decode_splits(const csp_params& p) {
     const int units = p.batch * p.n_kv_heads;
     const int tiles = (p.out_capacity + kDecTile - 1) / kDecTile;
     if (units <= 0 || tiles <= 0) return 1;
-    int splits = (2 * 2 * 148 + units - 1) / units;          // about two waves of two CTAs per SM
-    if (splits > tiles) splits = tiles;
+    // at least about four work items per resident CTA (148), but no item shorter than four tiles
+    int splits = (4 * 148 + units - 1) / units;
+    if (splits > (tiles + 3) / 4) splits = (tiles + 3) / 4;
     return splits < 1 ? 1 : splits;
 }
 
@@ -304,6 +358,7 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
     a.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
     a.out = out;
     a.status = static_cast<int32_t*>(ws);
+    a.next_item = a.status + 8;
     a.n_kv_heads = p.n_kv_heads; a.group = p.n_q_heads / p.n_kv_heads; a.head_dim = p.head_dim;
     a.capacity = p.out_capacity;
     a.splits = decode_splits(p);
@@ -318,7 +373,7 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
             return CSP_ERR_UNSUPPORTED;
         const int NH = p.head_dim / 64;
         const size_t smem = 1024 + size_t(kDecStages) * 2 * NH * kDecBlock + size_t(kDecWarps) * 8 * (p.head_dim + 2) * 4 +
-                            16 * kDecStages + 16;
+                            16 * kDecStages + 64;
         auto kern = NH == 1 ? decode_attn_kernel<1> : decode_attn_kernel<2>;
         static bool configured[2][64] = {};
         int dev = 0;
@@ -330,7 +385,8 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
             }
             if (dev >= 0 && dev < 64) configured[NH - 1][dev] = true;
         }
-        kern<<<dim3(a.splits, p.n_kv_heads, p.batch), kDecThreads, smem, s>>>(tk, tv, a);
+        const int n_items = units * a.splits;
+        kern<<<n_items < 148 ? n_items : 148, kDecThreads, smem, s>>>(tk, tv, a, n_items);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
     }
     decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);
