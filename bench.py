@@ -120,6 +120,10 @@ NCU_DRAM_BYTES_PER_LAYER = {
 }
 
 
+# the same for one launch of the decode kernel (bench.py --decode), all layers in one call
+NCU_DECODE_DRAM_BYTES = {1: 543.55e6}
+
+
 def algorithmic_bytes(cfg, n_out_total: int):
     """Per-layer algorithmic bytes of each kernel (every tensor touched exactly once)."""
     es = 2 if cfg.dtype == torch.bfloat16 else 4
@@ -293,7 +297,8 @@ def run_decode(args, rank, world, local_rank):
                            "replicas": "one independent replica per GPU, no collective"},
                 "clocks": clocks, "e2e": None, "gpu_launches": args.steps * 2,
                 "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                             "frac": achieved / peak, "traffic": NCU_DECODE_DRAM_BYTES.get(args.config),
+                             "peak_kind": f"of {peak_kind}",
                              "algorithmic_bytes_per_launch": ab, "us_per_launch": ms_step * 1e3},
                 "cpu_baseline": cpu_baseline, "device_status": status}
         print(json.dumps(line), flush=True)
