@@ -358,9 +358,9 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     if (units > 65535) return CSP_ERR_UNSUPPORTED;
-    // A CTA covers 4096 keys, or 8192 (1024 threads x 8) for caches above 8192 positions: smaller clusters
+    // A CTA covers 4096 keys, or 8192 (1024 threads x 8) for caches above 4096 positions: smaller clusters
     // mean fewer cluster barriers per round and, in a ragged batch, fewer CTAs that hold no keys.
-    const int per_cta = p.max_len <= 2 * 4096 ? 4096 : 8192;
+    const int per_cta = p.max_len <= 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
     if (per_cta == 8192) return launch_e<1024, 8>(p, a, cs, s);
