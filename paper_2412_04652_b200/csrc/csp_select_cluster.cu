@@ -358,14 +358,13 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     if (units > 65535) return CSP_ERR_UNSUPPORTED;
-    // A CTA covers 4096 keys, or 8192 (1024 threads x 8) for caches above 4096 positions: smaller clusters
-    // mean fewer cluster barriers per round and, in a ragged batch, fewer CTAs that hold no keys.
+    // A CTA covers 4096 keys, or 8192 for caches above 4096 positions: smaller clusters mean fewer cluster
+    // barriers per round and, in a ragged batch, fewer CTAs that hold no keys.  With many units the CTAs have
+    // 512 threads (8 or 16 keys per thread), two per SM, so that one CTA's barrier phases overlap the other's work.
     const int per_cta = p.max_len <= 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
-    if (per_cta == 8192) return launch_e<1024, 8>(p, a, cs, s);
-    // many units: half the threads with twice the keys each, two CTAs per SM, so that one CTA's barrier
-    // phases overlap the other's work
+    if (per_cta == 8192) return units * cs >= 2 * 148 ? launch_e<512, 16>(p, a, cs, s) : launch_e<1024, 8>(p, a, cs, s);
     if (units * cs >= 2 * 148) return launch_e<512, 8>(p, a, cs, s);
     return launch_e<1024, 4>(p, a, cs, s);
 }
