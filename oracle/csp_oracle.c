@@ -244,6 +244,17 @@ int orc_select(const orc_params* p, const float* score_self, const float* score_
                 orc_topk(cross ? c : s, cand, N, kb[prob], cross ? mc : ms,
                          mg ? mg + prob * 2 : NULL, mg ? mg + prob * 2 + 1 : NULL);
             }
+        } else if (p->select_mode == ORC_SELECT_OVERALL) {
+            /* the ablation's comparison arm ("Influence of n-softmax"): one top-k straight on the overall
+             * selection function, i.e. on the column sums of A over the whole window = s + c (Eq. 1 without
+             * the split); budgets [B, 1].  The sum is taken in fp32, the precision the scores are carried in. */
+            const int32_t kb = budgets[b];
+            float* mix = (float*)malloc(sizeof(float) * (size_t)(N > 0 ? N : 1));
+            for (int64_t t = 0; t < N; ++t) { cand[t] = 1; mix[t] = s[t] + c[t]; }
+            if (kb > N || kb < 0) fl |= ORC_FLAG_K_CLAMPED;
+            orc_topk(mix, cand, N, kb, ms, mg ? mg : NULL, mg ? mg + 1 : NULL);
+            memcpy(mc, ms, (size_t)(N > 0 ? N : 1));
+            free(mix);
         } else {
             const int32_t* kb = budgets + (int64_t)b * 2;
             for (int64_t t = 0; t < N; ++t) cand[t] = 1;

@@ -30,7 +30,7 @@ extern "C" {
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
 enum { ORC_COMBINE_OR = 0, ORC_COMBINE_AND = 1 };
-enum { ORC_SELECT_SEGMENTED = 0, ORC_SELECT_GLOBAL = 1 };
+enum { ORC_SELECT_SEGMENTED = 0, ORC_SELECT_GLOBAL = 1, ORC_SELECT_OVERALL = 2 };
 enum { ORC_HEADS_PER_KV = 0, ORC_HEADS_MEAN_ALL = 1 };
 
 /* per-unit flag bits written by orc_select / orc_prune_layer */

@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "libcsp_oracle.so")
 
 F32, BF16 = 0, 1
 COMBINE_OR, COMBINE_AND = 0, 1
-SELECT_SEGMENTED, SELECT_GLOBAL = 0, 1
+SELECT_SEGMENTED, SELECT_GLOBAL, SELECT_OVERALL = 0, 1, 2
 HEADS_PER_KV, HEADS_MEAN_ALL = 0, 1
 FLAG_K_CLAMPED, FLAG_CAPACITY, FLAG_IDENTITY = 1, 2, 4
 

@@ -393,6 +393,35 @@ def test_short_sequence_is_identity(oracle):
 
 # ---------------------------------------------------------------- input generator sanity
 
+def test_overall_topk_mode_is_one_stable_topk_on_the_summed_scores(oracle):
+    """The ablation's comparison arm: one top-k on s + c over all candidates, no split.  Checked against a
+    stable descending argsort of the fp32 sum; a window of a single label makes s + c the plain column sum of A."""
+    p, q, k, v, mod, L = _rand_case(oracle, 31, L=(40, 33), R=5, select_mode=oracle.SELECT_OVERALL)
+    s, c = oracle.score(p, q, k, mod, L)
+    s32, c32 = s.astype(np.float32), c.astype(np.float32)
+    bud = np.array([[7], [50]], np.int32)            # the second budget exceeds its candidates: clamped
+    idx, n_out, flags, _ = oracle.select(p, s32, c32, mod, L, bud)
+    for b in range(p.batch):
+        N = int(L[b]) - p.recent
+        kk = min(int(bud[b, 0]), N)
+        for h in range(p.n_kv_heads):
+            mix = s32[b, h, :N] + c32[b, h, :N]
+            want = np.sort(np.argsort(-mix.astype(np.float64), kind="stable")[:kk])
+            got = idx[b, h, :n_out[b, h]]
+            np.testing.assert_array_equal(got[:kk], want)
+            np.testing.assert_array_equal(got[kk:], np.arange(N, int(L[b])))
+            assert bool(flags[b, h] & oracle.FLAG_K_CLAMPED) == (int(bud[b, 0]) > N)
+    # with every query and key carrying one label the inter score is zero and s is the whole column sum
+    one = np.zeros_like(mod)
+    s1, c1 = oracle.score(p, q, k, one, L)
+    assert (c1 == 0).all()
+    i_over, n_over, _, _ = oracle.select(p, s1.astype(np.float32), c1.astype(np.float32), one, L, np.array([[6], [6]], np.int32))
+    pg = oracle.Params(**{**p.__dict__, "select_mode": oracle.SELECT_GLOBAL})
+    i_glob, n_glob, _, _ = oracle.select(pg, s1.astype(np.float32), c1.astype(np.float32), one, L, np.array([[6, 0], [6, 0]], np.int32))
+    np.testing.assert_array_equal(n_over, n_glob)
+    np.testing.assert_array_equal(i_over, i_glob)
+
+
 # ---------------------------------------------------------------- Section 3.3: n-softmax decode attention
 
 def _decode_case(oracle, seed, B=2, Hq=6, Hkv=2, d=16, cap=37, dtype=torch.float32, gain=1.0, **pk):
