@@ -62,8 +62,10 @@ typedef enum { CSP_F32 = 0, CSP_BF16 = 1 } csp_dtype;
 typedef enum { CSP_COMBINE_OR = 0, CSP_COMBINE_AND = 1 } csp_combine;
 
 /* SEGMENTED: four budgets per sequence, a top-K of the intra score and of the inter score among
- * the text keys and among the visual keys.  GLOBAL: the paper's literal K^s and K^c over all keys. */
-typedef enum { CSP_SELECT_SEGMENTED = 0, CSP_SELECT_GLOBAL = 1 } csp_select_mode;
+ * the text keys and among the visual keys.  GLOBAL: the paper's literal K^s and K^c over all keys.
+ * OVERALL: the comparison arm of the paper's ablation ("Influence of n-softmax"): one budget per
+ * sequence, a single top-K on the overall selection function s + c (fp32 sum), no split. */
+typedef enum { CSP_SELECT_SEGMENTED = 0, CSP_SELECT_GLOBAL = 1, CSP_SELECT_OVERALL = 2 } csp_select_mode;
 
 /* PER_KV: one selection per KV head from the mean over its query-head group.
  * MEAN_ALL: one selection per sequence from the mean over every head (Section 3.2). */
@@ -128,7 +130,8 @@ csp_status csp_score(const csp_params* p, csp_tensor q_win, csp_tensor k,
 /*
  * Eq. 2, Eq. 3 and the index list of Eq. 4.
  *   budgets    int32. SEGMENTED: [B,4] = k_self_text, k_self_visual, k_cross_text, k_cross_visual.
- *              GLOBAL: [B,2] = k_self, k_cross.  Each is clamped to [0, candidates] (flagged).
+ *              GLOBAL: [B,2] = k_self, k_cross.  OVERALL: [B,1] = k.  Each is clamped to
+ *              [0, candidates] (flagged).
  *   total_budget_or_null [B] int32 = T of Algorithm 1: a sequence with L_b < T keeps everything.
  *   keep_idx   [B, H_kv, out_capacity] int32: kept positions ascending, then L_b-R .. L_b-1
  *   n_out      [B, H_kv] int32: length of that list; -1 if it would exceed out_capacity (flagged,

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libcsp.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
 F32, BF16 = 0, 1
 COMBINE_OR, COMBINE_AND = 0, 1
-SELECT_SEGMENTED, SELECT_GLOBAL = 0, 1
+SELECT_SEGMENTED, SELECT_GLOBAL, SELECT_OVERALL = 0, 1, 2
 HEADS_PER_KV, HEADS_MEAN_ALL = 0, 1
 DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
 

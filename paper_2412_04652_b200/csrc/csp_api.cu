@@ -25,7 +25,9 @@ csp_status check_params(const csp_params* p) {
         return CSP_ERR_INVALID_ARG;
     if (p->dtype != CSP_F32 && p->dtype != CSP_BF16) return CSP_ERR_UNSUPPORTED;
     if (p->combine != CSP_COMBINE_OR && p->combine != CSP_COMBINE_AND) return CSP_ERR_INVALID_ARG;
-    if (p->select_mode != CSP_SELECT_SEGMENTED && p->select_mode != CSP_SELECT_GLOBAL) return CSP_ERR_INVALID_ARG;
+    if (p->select_mode != CSP_SELECT_SEGMENTED && p->select_mode != CSP_SELECT_GLOBAL &&
+        p->select_mode != CSP_SELECT_OVERALL)
+        return CSP_ERR_INVALID_ARG;
     if (p->head_reduce != CSP_HEADS_PER_KV && p->head_reduce != CSP_HEADS_MEAN_ALL) return CSP_ERR_INVALID_ARG;
     if (p->n_q_heads % p->n_kv_heads) return CSP_ERR_INVALID_ARG;
     if (!(p->n >= 0.f) || !(p->scale >= 0.f)) return CSP_ERR_INVALID_ARG;
@@ -88,7 +90,10 @@ csp_status do_select(const csp_params& p, const float* score_self, const float* 
     a.keep_idx = keep_idx; a.n_out = n_out; a.status = static_cast<int32_t*>(ws);
     a.n_kv_heads = p.n_kv_heads; a.window = p.window; a.recent = p.recent; a.max_len = p.max_len;
     a.out_capacity = p.out_capacity;
-    a.combine_and = p.combine == CSP_COMBINE_AND; a.global_mode = p.select_mode == CSP_SELECT_GLOBAL;
+    a.combine_and = p.combine == CSP_COMBINE_AND;
+    // OVERALL runs as GLOBAL with both problems on the summed score and the same budget: their union is the one top-K
+    a.overall = p.select_mode == CSP_SELECT_OVERALL;
+    a.global_mode = p.select_mode == CSP_SELECT_GLOBAL || a.overall;
     return launch_select(p, a, stream);
 }
 
@@ -256,7 +261,7 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
     const size_t kv_bytes = units * p->max_len * p->head_dim * es;
     const size_t mod_bytes = (mod_per_head ? units : size_t(p->batch)) * p->max_len;
     const size_t out_bytes = units * p->out_capacity * p->head_dim * es;
-    const int nbud = p->select_mode == CSP_SELECT_GLOBAL ? 2 : 4;
+    const int nbud = p->select_mode == CSP_SELECT_GLOBAL ? 2 : (p->select_mode == CSP_SELECT_OVERALL ? 1 : 4);
     bool ok = true;
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
         if (bytes) ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;

@@ -61,6 +61,7 @@ struct SelectArgs {
     int32_t* keep_idx; int32_t* n_out; int32_t* status;
     int32_t n_kv_heads, window, recent, max_len, out_capacity;
     int32_t combine_and, global_mode;
+    int32_t overall;                                 // global_mode with both problems on s + c and budgets [B, 1]
 };
 
 struct CompactArgs {

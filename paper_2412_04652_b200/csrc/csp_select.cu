@@ -96,22 +96,22 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
     const float* const sc = a.score_cross + int64_t(u) * a.max_len;
     const uint8_t* const mod = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
     const int nprob = a.global_mode ? 2 : 4;
-    const int32_t* const bud = a.budgets + int64_t(b) * nprob;
+    const int32_t* const bud = a.budgets + int64_t(b) * (a.overall ? 1 : nprob);
 
     // stage the order-preserving keys and labels on chip once; every later pass reads them from there
     const int n_cached = min(N, n_cached_max);
     for (int t = tid; t < n_cached; t += kSelThreads) {
-        cache_s[t] = order_key(ss[t]);
-        cache_c[t] = order_key(sc[t]);
+        cache_s[t] = order_key(a.overall ? ss[t] + sc[t] : ss[t]);
+        cache_c[t] = order_key(a.overall ? ss[t] + sc[t] : sc[t]);
         cache_m[t] = mod[t];
     }
-    auto key_s = [&](int t) { return t < n_cached ? cache_s[t] : order_key(ss[t]); };
-    auto key_c = [&](int t) { return t < n_cached ? cache_c[t] : order_key(sc[t]); };
+    auto key_s = [&](int t) { return t < n_cached ? cache_s[t] : order_key(a.overall ? ss[t] + sc[t] : ss[t]); };
+    auto key_c = [&](int t) { return t < n_cached ? cache_c[t] : order_key(a.overall ? ss[t] + sc[t] : sc[t]); };
     auto label = [&](int t) { return t < n_cached ? cache_m[t] : mod[t]; };
 
     if (tid < 4) {
         prefix[tid] = 0;
-        const int32_t k = tid < nprob ? bud[tid] : 0;
+        const int32_t k = tid < nprob ? bud[a.overall ? 0 : tid] : 0;
         krem[tid] = k;
         act[tid] = k > 0;
         if (k < 0) atomicOr(a.status, CSP_DEV_K_CLAMPED);

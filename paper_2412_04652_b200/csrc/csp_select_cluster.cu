@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_
     const float* const sc = a.score_cross + int64_t(u) * a.max_len;
     const uint8_t* const mod = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
     const int nprob = a.global_mode ? 2 : 4;
-    const int32_t* const bud = a.budgets + int64_t(b) * nprob;
+    const int32_t* const bud = a.budgets + int64_t(b) * (a.overall ? 1 : nprob);
     const int pc_base = a.global_mode ? 1 : 2;           // first inter-score problem
     const int pc1 = pc_base + 1 < 4 ? pc_base + 1 : 3;
 
@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             const bool ok = warp_base + e * 32 + lane < N;
+            if (a.overall) fs[e] = fc[e] = fs[e] + fc[e];        // one top-K on the summed score, run twice
             ks[e] = ok ? order_key(fs[e]) : 0u;
             kc[e] = ok ? order_key(fc[e]) : 0u;
             if (ok) valid |= 1u << e;
@@ -104,7 +105,7 @@ __global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_
     }
     if (tid < 4) {
         chosen[tid] = 256u;
-        const int32_t k = tid < nprob ? bud[tid] : 0;
+        const int32_t k = tid < nprob ? bud[a.overall ? 0 : tid] : 0;
         krem[tid] = k;
         act[tid] = k > 0;
         eqcnt[tid] = 0;

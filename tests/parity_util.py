@@ -49,7 +49,7 @@ def assert_scores_close(got: np.ndarray, want: np.ndarray, seq_lens, recent, wha
             assert (g[zero] == 0.0).all(), f"{what} unit ({b},{h}): structural zeros must be exactly 0"
 
 
-def assert_index_sets_match(gpu_idx, gpu_n, ref, modality, seq_lens, recent, global_mode=False):
+def assert_index_sets_match(gpu_idx, gpu_n, ref, modality, seq_lens, recent, global_mode=False, overall=False):
     """Kept sets must be identical except for keys whose oracle score lies within REL_TOL of the
     K-th (boundary) score of a top-K problem the key takes part in.  Returns the number of
     boundary-band differences that were tolerated."""
@@ -76,7 +76,8 @@ def assert_index_sets_match(gpu_idx, gpu_n, ref, modality, seq_lens, recent, glo
             mg = ref["margins"][b, h]
             for t in diff:
                 vis = int(mod[t] != 0)
-                probs = [(0, ref["score_self"]), (1, ref["score_cross"])] if global_mode else \
+                probs = [(0, ref["score_self"] + ref["score_cross"])] if overall else \
+                        [(0, ref["score_self"]), (1, ref["score_cross"])] if global_mode else \
                         [(vis, ref["score_self"]), (2 + vis, ref["score_cross"])]
                 ok = False
                 for pidx, sc in probs:

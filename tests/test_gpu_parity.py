@@ -215,10 +215,11 @@ def _select_case(csp, oracle, B, H, lens, R, budgets, quantise=None, seed=0, tot
     return run.status(), flags
 
 
-@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1), dict(select_mode=1, combine=1)])
+@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1), dict(select_mode=1, combine=1),
+                                  dict(select_mode=2), dict(select_mode=2, combine=1)])
 def test_select_matches_oracle_exactly(csp, oracle, mode):
     lens = (3000, 1500, 777)
-    nb = 2 if mode.get("select_mode") else 4
+    nb = {0: 4, 1: 2, 2: 1}[mode.get("select_mode", 0)]
     budgets = np.random.RandomState(1).randint(0, 400, size=(3, nb))
     _select_case(csp, oracle, 3, 2, lens, 32, budgets, seed=1, **mode)
     _select_case(csp, oracle, 3, 2, lens, 32, budgets, quantise=16, seed=2, **mode)   # heavy ties
@@ -242,6 +243,14 @@ def test_select_identity_capacity_and_short_sequences(csp, oracle):
 def test_select_long_sequence(csp, oracle):
     _select_case(csp, oracle, 1, 2, (32768,), 32, [[1626, 0, 0, 4301]], seed=7)
     _select_case(csp, oracle, 1, 1, (32768,), 32, [[1626, 3, 9, 4301]], quantise=64, seed=8)
+
+
+def test_select_overall_mode_long_caches(csp, oracle):
+    """One top-K on s + c (the ablation's comparison arm), through every selection kernel shape."""
+    _select_case(csp, oracle, 2, 2, (32768, 9000), 32, [[4000], [100000]], seed=12, select_mode=2)
+    _select_case(csp, oracle, 1, 1, (66000,), 32, [[700]], quantise=32, seed=13, select_mode=2)
+    _select_case(csp, oracle, 40, 8, tuple(3000 + 13 * i for i in range(40)), 32, [[300 + i] for i in range(40)],
+                 quantise=64, seed=14, select_mode=2)
 
 
 def test_select_cache_longer_than_cluster_limit(csp, oracle):
@@ -307,17 +316,19 @@ def _run_prune(csp, oracle, cfg, layer=0, with_optional=True, **mode):
     return run, ref
 
 
-@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1)])
+@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1), dict(select_mode=2)])
 def test_prune_layer_small(csp, oracle, mode):
     cfg = _case((900, 300, 517), 4, 2, 128, 32, 32, seed=30, visual_pct=25, text_pct=50)
-    if mode.get("select_mode"):
+    if mode.get("select_mode") == 1:
         cfg.budgets = cfg.budgets[:, [0, 3]].copy()
+    elif mode.get("select_mode") == 2:
+        cfg.budgets = cfg.budgets.sum(axis=1, keepdims=True).astype(np.int32)
     run, ref = _run_prune(csp, oracle, cfg, **mode)
     assert run.status() == 0
     assert_scores_close(run.ss.cpu().numpy(), ref["score_self"], cfg.seq_lens, cfg.recent)
     assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, cfg.recent)
     assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens,
-                            cfg.recent, global_mode=bool(mode.get("select_mode")))
+                            cfg.recent, global_mode=mode.get("select_mode") == 1, overall=mode.get("select_mode") == 2)
     assert_compaction_exact(run, cfg.modality())
     if not mode:
         np.testing.assert_array_equal(run.n_out.cpu().numpy(), ref["n_out"])
