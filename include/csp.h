@@ -150,6 +150,10 @@ csp_status csp_select(const csp_params* p, const float* score_self, const float*
  * Eq. 4: k_out[b,h,j,:] = k[b,h,keep_idx[b,h,j],:] for j < n_out[b,h]; same for v and the labels.
  *   k_out, v_out [B, H_kv, out_capacity, d] (strided); mod_out [B, H_kv, out_capacity] dense, may
  *   be NULL.  Rows j >= n_out are left as they were; units with n_out <= 0 are skipped.
+ * In place (the iteration of Algorithm 1 without a second cache buffer): k_out may be the very tensor k
+ * and v_out the very tensor v (same pointer and strides, both or neither; CSP_ERR_UNSUPPORTED otherwise).
+ * keep_idx is ascending with keep_idx[j] >= j, as csp_select writes it, so rows only move down; mod_out
+ * stays a separate array.  Any other overlap between inputs and outputs is not detected and not allowed.
  */
 csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v,
                        const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,

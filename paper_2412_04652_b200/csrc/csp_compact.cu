@@ -1,5 +1,5 @@
-// Compaction kernel (Eq. 4): gather the kept rows of K and V, and their modality labels, into the
-// compacted cache.  Pure data movement: rows are copied as 16-byte chunks, one row per
+// Compaction kernels (Eq. 4): gather the kept rows of K and V, and their modality labels, into the
+// compacted cache (a second buffer, or the same one: see compact_inplace_kernel).  Pure data movement: rows are copied as 16-byte chunks, one row per
 // (row bytes / 16) consecutive threads, so every load and store is a full 128-bit access and a
 // warp covers whole rows.
 #include "csp_internal.cuh"
@@ -67,11 +67,72 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactA
     }
 }
 
+// In-place variant (k_out is k, v_out is v): row j of a unit moves from position keep_idx[j] >= j down to
+// position j.  One CTA walks a unit's rows in ascending chunks; inside a chunk every load is issued before
+// the CTA barrier and every store after it.  That is enough: a later chunk only reads positions at or beyond
+// its own first row, which no earlier chunk has written, and a chunk's own sources are read before the
+// barrier.  The loads are ordinary (coherent) loads: the kernel writes the memory it reads.
+constexpr int kInplaceThreads = 512;
+
+__global__ void __launch_bounds__(kInplaceThreads) compact_inplace_kernel(const CompactArgs a) {
+    const int u = blockIdx.x, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
+    const int n = a.n_out[u];
+    if (n <= 0) return;
+    const int cpr = a.chunks_per_row;                    // 8, 16 or 32
+    const int rows_per_iter = kInplaceThreads / cpr;
+    const int r_in = threadIdx.x / cpr, c = threadIdx.x % cpr;
+    const int32_t* const idx = a.keep_idx + int64_t(u) * a.out_capacity;
+    uint4* const kio = static_cast<uint4*>(a.k_out) + int64_t(b) * a.ko_sb + int64_t(h) * a.ko_sh;
+    uint4* const vio = static_cast<uint4*>(a.v_out) + int64_t(b) * a.vo_sb + int64_t(h) * a.vo_sh;
+    const int row_end = min(n, a.out_capacity);
+    // labels first: they go to a separate array, so no ordering is needed
+    if (a.mod_out && a.modality) {
+        const uint8_t* const mod = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
+        for (int j = threadIdx.x; j < row_end; j += kInplaceThreads) {
+            const int t = idx[j];
+            if (t >= 0 && t < a.max_len) a.mod_out[int64_t(u) * a.out_capacity + j] = mod[t];
+        }
+    }
+    for (int j0 = 0; j0 < row_end; j0 += 4 * rows_per_iter) {
+        uint4 kv[4], vv[4];
+        int jj[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            jj[q] = j0 + q * rows_per_iter + r_in;
+            if (jj[q] < row_end) {
+                const int t = idx[jj[q]];
+                // a bad index or a source above its destination copies nothing; a row already in place stays
+                if (t > jj[q] && t < a.max_len) {
+                    kv[q] = kio[int64_t(t) * a.ko_st + c];
+                    vv[q] = vio[int64_t(t) * a.vo_st + c];
+                } else {
+                    jj[q] = row_end;
+                }
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (jj[q] < row_end) {
+                kio[int64_t(jj[q]) * a.ko_st + c] = kv[q];
+                vio[int64_t(jj[q]) * a.vo_st + c] = vv[q];
+            }
+    }
+}
+
 }  // namespace
 
 csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_t s) {
     const int units = p.batch * p.n_kv_heads;
     if (units == 0 || p.out_capacity == 0) return CSP_OK;
+    if (a.k == a.k_out || a.v == a.v_out) {
+        // in place: both tensors, with the strides of their inputs
+        if (a.k != a.k_out || a.v != a.v_out || a.k_sb != a.ko_sb || a.k_sh != a.ko_sh || a.k_st != a.ko_st ||
+            a.v_sb != a.vo_sb || a.v_sh != a.vo_sh || a.v_st != a.vo_st)
+            return CSP_ERR_UNSUPPORTED;
+        compact_inplace_kernel<<<units, kInplaceThreads, 0, s>>>(a);
+        return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
+    }
     const long long blocks = (long long)((p.out_capacity + kRowsPerCta - 1) / kRowsPerCta) * units;
     if (blocks > 0x7fffffffLL) return CSP_ERR_UNSUPPORTED;
     const dim3 grid((unsigned)blocks);

@@ -304,6 +304,68 @@ def test_compact_is_bit_exact_with_strides(csp, oracle):
     np.testing.assert_array_equal(run.mod_out.cpu().numpy(), mo)
 
 
+@pytest.mark.parametrize("d,dtype", [(128, torch.bfloat16), (64, torch.bfloat16), (64, torch.float32)])
+def test_compact_in_place_matches_out_of_place(csp, oracle, d, dtype):
+    """k_out is k and v_out is v: rows move down inside the cache.  Dense keeps (many rows shifting by a few
+    positions, across several 128-row chunks) are the hazardous case; an identity prefix and empty units too."""
+    lens = (1500, 700, 333)
+    cfg = _case(lens, 4, 2, d, 16, 16, dtype=dtype, seed=21)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    cap = 1500
+    p = gpu_params(csp, cfg, cap=cap)
+    rng = np.random.RandomState(1)
+    idx = np.full((3, 2, cap), -1, np.int32)
+    n_out = np.array([[1490, 600], [700, 0], [129, 1]], np.int32)      # near-full, sparse, identity, empty, chunk + 1, one
+    for b in range(3):
+        for h in range(2):
+            n = int(n_out[b, h])
+            idx[b, h, :n] = np.sort(rng.choice(lens[b], n, replace=False))
+    idx[0, 1, :200] = np.arange(200)                                    # identity prefix, then a jump
+    idx[0, 1, 200:600] = np.sort(rng.choice(np.arange(200, lens[0]), 400, replace=False))
+    ko, vo, mo = oracle.compact(orc_params(oracle, cfg, cap=cap), k.cpu(), v.cpu(), cfg.modality(), idx, n_out)
+    if ko.dtype == np.float32:
+        ko, vo = ko.view(np.uint32), vo.view(np.uint32)
+    run = GpuRun(csp, p, q, k.clone(), v.clone(), cfg.modality(), cfg.seq_lens, cfg.budgets)
+    run.idx, run.n_out = torch.from_numpy(idx).cuda(), torch.from_numpy(n_out).cuda()
+    run.k_out, run.v_out = run.k, run.v                                 # the same tensors
+    run.compact()
+    kb, vb = bits(run.k), bits(run.v)
+    for b in range(3):
+        for h in range(2):
+            n = int(n_out[b, h])
+            np.testing.assert_array_equal(kb[b, h, :n], ko[b, h, :n])
+            np.testing.assert_array_equal(vb[b, h, :n], vo[b, h, :n])
+            np.testing.assert_array_equal(run.mod_out.cpu().numpy()[b, h, :n], mo[b, h, :n])
+            if n == 0:                                                  # an empty unit is left untouched
+                np.testing.assert_array_equal(kb[b, h, :lens[b]], bits(k)[b, h, :lens[b]])
+    # only one of the two tensors in place is refused
+    run2 = GpuRun(csp, p, q, k.clone(), v.clone(), cfg.modality(), cfg.seq_lens, cfg.budgets)
+    run2.idx, run2.n_out = run.idx, run.n_out
+    run2.k_out = run2.k
+    with pytest.raises(csp.CspError) as e:
+        run2.compact()
+    assert e.value.code == 2
+
+
+def test_prune_layer_in_place(csp, oracle):
+    """Algorithm 1 without a second cache buffer: k_out / v_out are the input tensors."""
+    cfg = _case((1200, 640), 8, 4, 128, 32, 32, seed=22)
+    run, ref = _run_prune(csp, oracle, cfg)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    p = gpu_params(csp, cfg)
+    inp = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget)
+    inp.k_out, inp.v_out = inp.k, inp.v
+    inp.prune()
+    assert inp.status() == 0
+    assert torch.equal(inp.n_out, run.n_out) and torch.equal(inp.idx, run.idx)
+    n_out = run.n_out.cpu().numpy()
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            n = int(n_out[b, h])
+            assert torch.equal(inp.k[b, h, :n], run.k_out[b, h, :n]) and torch.equal(inp.v[b, h, :n], run.v_out[b, h, :n])
+    assert torch.equal(inp.mod_out, run.mod_out)
+
+
 # ------------------------------------------------------------------ Algorithm 1 end to end
 
 def _run_prune(csp, oracle, cfg, layer=0, with_optional=True, **mode):
