@@ -8,7 +8,10 @@ namespace csp {
 namespace {
 
 constexpr int kCompactThreads = 256;
-constexpr int kRowsPerCta = 64;
+// rows per CTA: 128 when that still gives every SM several CTAs (fewer, longer CTAs stream better), else 64
+inline int rows_per_cta(int units, int capacity) {
+    return (long long)units * ((capacity + 127) / 128) >= 8 * 148 ? 128 : 64;
+}
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;
@@ -17,21 +20,22 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+template <int rows_cta, int CPR>   // rows per CTA; 16-byte chunks per row (8, 16 or 32)
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactArgs a) {
-    const int blocks_per_unit = (a.out_capacity + kRowsPerCta - 1) / kRowsPerCta;
+    const int blocks_per_unit = (a.out_capacity + rows_cta - 1) / rows_cta;
     const int u = blockIdx.x / blocks_per_unit, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
     const int n = a.n_out[u];
-    const int row0 = (blockIdx.x % blocks_per_unit) * kRowsPerCta;
+    const int row0 = (blockIdx.x % blocks_per_unit) * rows_cta;
     if (n <= 0 || row0 >= n) return;
-    const int cpr = a.chunks_per_row;                    // 8, 16 or 32
-    const int rows_per_iter = kCompactThreads / cpr;
+    constexpr int cpr = CPR;
+    constexpr int rows_per_iter = kCompactThreads / cpr;
     const int r_in = threadIdx.x / cpr, c = threadIdx.x % cpr;
     const int32_t* const idx = a.keep_idx + int64_t(u) * a.out_capacity;
     const uint4* const kin = static_cast<const uint4*>(a.k) + int64_t(b) * a.k_sb + int64_t(h) * a.k_sh;
     const uint4* const vin = static_cast<const uint4*>(a.v) + int64_t(b) * a.v_sb + int64_t(h) * a.v_sh;
     uint4* const kout = static_cast<uint4*>(a.k_out) + int64_t(b) * a.ko_sb + int64_t(h) * a.ko_sh;
     uint4* const vout = static_cast<uint4*>(a.v_out) + int64_t(b) * a.vo_sb + int64_t(h) * a.vo_sh;
-    const int row_end = min(n, row0 + kRowsPerCta);
+    const int row_end = min(n, row0 + rows_cta);
 
     for (int j0 = row0; j0 < row_end; j0 += 4 * rows_per_iter) {
         // four independent rows per thread in flight
@@ -133,10 +137,17 @@ csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_
         compact_inplace_kernel<<<units, kInplaceThreads, 0, s>>>(a);
         return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
     }
-    const long long blocks = (long long)((p.out_capacity + kRowsPerCta - 1) / kRowsPerCta) * units;
+    const int rpc = rows_per_cta(units, p.out_capacity);
+    const long long blocks = (long long)((p.out_capacity + rpc - 1) / rpc) * units;
     if (blocks > 0x7fffffffLL) return CSP_ERR_UNSUPPORTED;
     const dim3 grid((unsigned)blocks);
-    compact_kernel<<<grid, kCompactThreads, 0, s>>>(a);
+    auto launch = [&](auto kern) { kern<<<grid, kCompactThreads, 0, s>>>(a); };
+    switch (a.chunks_per_row) {
+        case 8: rpc == 128 ? launch(compact_kernel<128, 8>) : launch(compact_kernel<64, 8>); break;
+        case 16: rpc == 128 ? launch(compact_kernel<128, 16>) : launch(compact_kernel<64, 16>); break;
+        case 32: rpc == 128 ? launch(compact_kernel<128, 32>) : launch(compact_kernel<64, 32>); break;
+        default: return CSP_ERR_UNSUPPORTED;
+    }
     return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
 }
 
