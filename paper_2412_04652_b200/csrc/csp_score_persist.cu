@@ -399,17 +399,22 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const uint32_t add_s = same & vis, add_c = ~same & vis;
                 float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
                 const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
+                // The whole row of logits goes to registers first and the buffer is handed back at once: the
+                // tensor core refills it (next unit) while the weights are still being computed here.
                 uint32_t va[16], vb[16];
                 tc_ld_row16(va, row_addr);
+                tc_ld_row16(vb, row_addr + 16u);
+                tc_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);          // the tensor core may refill this buffer
                 // Common case: every window query carries the same label and no column of this tile is
                 // hidden.  Then a key's weights all go to one of the two sums, chosen once per key, and the
                 // columns beyond W add exact zeros (their constant is -inf): plain sums, no selection.
                 const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    tc_wait_ld();
                     uint32_t (&cur)[16] = ch ? vb : va;
-                    if (ch == 0) tc_ld_row16(vb, row_addr + 16u);
                     const float4* cv = reinterpret_cast<const float4*>(cv_team + ch * 16);
                     if (plain) {
 #pragma unroll
@@ -441,9 +446,6 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     s0 = same ? total : 0.f; s1 = 0.f;
                     c0 = same ? 0.f : total; c1 = 0.f;
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);          // the tensor core may refill this buffer
                 if (t < x.N) { out_s[t] = s0 + s1; out_c[t] = c0 + c1; }
             }
             // the label table and Q of this parity may now be restaged
