@@ -54,7 +54,7 @@ constexpr int kPsMaxStages = 8;
 constexpr int kQSets = 3;                               // Q tiles and label tables staged ahead (ring)
 
 struct PsSmemPlan {   // byte offsets from the 1024-aligned base
-    uint32_t q, wstats, cstats, cvec, rmax, dq_mask, dq_val, bars, misc, total;
+    uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
 };
 __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     PsSmemPlan s;
@@ -63,7 +63,6 @@ __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     s.wstats = off;   off += 16u * 32u * 8u;                     // [team][warp][column]
     s.cstats = off;   off += 4u * 8u * 32u * 8u;                  // [unit & 3][rank][row], written by the peers
     s.cvec = off;     off += 2u * 32u * 4u;                      // per team
-    s.rmax = off;     off += 2u * 4u * 32u * 4u;                 // [team][quarter][column]: column maxima of the first tile
     s.dq_mask = off;  off += uint32_t(kQSets) * 32u * 4u;
     s.dq_val = off;   off += uint32_t(kQSets) * 32u * 4u;
     s.bars = off;     off += (2u * kPsMaxStages + 3u * kBufs + 3u * kQSets + 2u) * 8u;
@@ -89,7 +88,6 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     float2* const wstats = reinterpret_cast<float2*>(base_ptr + sp.wstats);
     float2* const cstats = reinterpret_cast<float2*>(base_ptr + sp.cstats);
     float* const cvec = reinterpret_cast<float*>(base_ptr + sp.cvec);
-    float* const rmax_all = reinterpret_cast<float*>(base_ptr + sp.rmax);
     uint32_t* const dq_mask = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_mask);
     uint32_t* const dq_val = reinterpret_cast<uint32_t*>(base_ptr + sp.dq_val);
     const uint32_t full_k = base + sp.bars;
@@ -313,48 +311,9 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             }
 
             // ---------------------------------- pass 1 ----------------------------------
-            // Reference exponent of every window column: its maximum over the first tile this CTA holds of the
-            // unit (for rank 0 that tile contains the first keys of the sequence, where the largest logits of an
-            // attention row usually sit).  Pass 1 then replaces every logit in tensor memory by
-            // e = 2^(x scale2 - r_w), so that pass 2 needs one multiply per element and no exponential.  The
-            // exponent is capped at 2^120: a logit more than 83 nats above the reference would lose accuracy
-            // instead of overflowing.
-            float* const rmax = rmax_all + team * (4 * 32);
-            auto visible = [&](int colw, int t) { return colw < W && t <= first_masked_key + colw; };
-            if (group == 0 && x.my_all > 0) {
-                mbar_wait(my_full, ph, abort_flag);
-                tc_fence_after();
-                const int tile = int(rank);
-                const bool masked = (tile + 1) * kTileKeys > first_masked_key;
-                const int t_base = tile * kTileKeys + quarter * 32 + lr;
-                uint32_t v0[16], v1[16];
-                tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16));
-                tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16));
-                tc_wait_ld();
+            float m_run[8], z_run[8];
 #pragma unroll
-                for (int jj = 0; jj < 8; ++jj) {
-                    const int i4 = (jj >> 1) * 4 + (jj & 1), colw = (jj >> 1) * 8 + lq * 2 + (jj & 1);
-                    float xv[4] = {__uint_as_float(v0[i4]), __uint_as_float(v0[i4 + 2]), __uint_as_float(v1[i4]),
-                                   __uint_as_float(v1[i4 + 2])};
-                    if (masked) {
-#pragma unroll
-                        for (int r = 0; r < 4; ++r)
-                            if (!visible(colw, t_base + (r & 1) * 8 + (r >> 1) * 16)) xv[r] = kNeg;
-                    }
-                    float mx = fmaxf(fmaxf(xv[0], xv[1]), fmaxf(xv[2], xv[3]));
-#pragma unroll
-                    for (int d = 4; d <= 16; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-                    if (lr == 0) rmax[quarter * 32 + colw] = mx > 0.5f * kNeg ? mx * scale2 : kNeg;
-                }
-            }
-            team_sync(team);
-            float r_col[8], z_run[8];
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-                const int colw = (jj >> 1) * 8 + lq * 2 + (jj & 1);
-                r_col[jj] = x.my_all > 0 ? fmaxf(fmaxf(rmax[colw], rmax[32 + colw]), fmaxf(rmax[64 + colw], rmax[96 + colw])) : kNeg;
-                z_run[jj] = 0.f;
-            }
+            for (int jj = 0; jj < 8; ++jj) { m_run[jj] = kNeg; z_run[jj] = 0.f; }
             for (int i = group; i < x.my_all; i += 2) {
                 const int buf = i;
                 const int tile = i * int(csize) + int(rank);
@@ -362,41 +321,23 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 tc_fence_after();
                 const bool masked = (tile + 1) * kTileKeys > first_masked_key;
                 const int t_base = tile * kTileKeys + quarter * 32 + lr;
-                const uint32_t lo = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
-                const uint32_t hi = tmem_base + (uint32_t(quarter * 32 + 16) << 16) + uint32_t(buf * NC);
                 uint32_t v0[16], v1[16];
-                tc_ld_16x32(v0, lo);
-                tc_ld_16x32(v1, hi);
+                tc_ld_16x32(v0, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC));
+                tc_ld_16x32(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + uint32_t(buf * NC));
                 tc_wait_ld();
-#pragma unroll
-                for (int jj = 0; jj < 8; ++jj) {
-                    const int i4 = (jj >> 1) * 4 + (jj & 1);
-                    const float nr = -r_col[jj];
-                    float e[4] = {ex2f(fminf(fmaf(__uint_as_float(v0[i4]), scale2, nr), 120.f)),
-                                  ex2f(fminf(fmaf(__uint_as_float(v0[i4 + 2]), scale2, nr), 120.f)),
-                                  ex2f(fminf(fmaf(__uint_as_float(v1[i4]), scale2, nr), 120.f)),
-                                  ex2f(fminf(fmaf(__uint_as_float(v1[i4 + 2]), scale2, nr), 120.f))};
-                    if (masked) {
-                        const int colw = (jj >> 1) * 8 + lq * 2 + (jj & 1);
-#pragma unroll
-                        for (int r = 0; r < 4; ++r)
-                            if (!visible(colw, t_base + (r & 1) * 8 + (r >> 1) * 16)) e[r] = 0.f;
-                    }
-                    z_run[jj] += (e[0] + e[1]) + (e[2] + e[3]);
-                    v0[i4] = __float_as_uint(e[0]); v0[i4 + 2] = __float_as_uint(e[1]);
-                    v1[i4] = __float_as_uint(e[2]); v1[i4 + 2] = __float_as_uint(e[3]);
-                }
-                tc_st_16x32(lo, v0);
-                tc_st_16x32(hi, v1);
+                if (!masked) stats_block<4>(v0, v1, m_run, z_run, scale2);
+                else stats_block_masked<4>(v0, v1, m_run, z_run, scale2, t_base, first_masked_key, W, lq * 2);
             }
-            tc_wait_st();
-            tc_fence_before();                           // pass 2 (other threads) reads what was stored here
-            // merge: lanes holding the same columns (same reference: plain sums), then warps, then the CTAs
+            // merge: lanes holding the same columns, then warps, then the CTAs of the cluster
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
 #pragma unroll
-                for (int d = 4; d <= 16; d <<= 1) z_run[jj] += __shfl_xor_sync(0xffffffffu, z_run[jj], d);
-                if (lr == 0) wst[tw * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(r_col[jj], z_run[jj]);
+                for (int d = 4; d <= 16; d <<= 1) {
+                    const float om = __shfl_xor_sync(0xffffffffu, m_run[jj], d);
+                    const float oz = __shfl_xor_sync(0xffffffffu, z_run[jj], d);
+                    merge_stats(m_run[jj], z_run[jj], om, oz);
+                }
+                if (lr == 0) wst[tw * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
             }
             team_sync(team);
             const int qs = j % kQSets;
@@ -410,7 +351,6 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 for (int d = 1; d < kTeamWarps; d <<= 1)                  // pairwise tree, fixed order
 #pragma unroll
                     for (int w = 0; w < kTeamWarps; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
-                const float r_mine = v[0].x;             // this CTA's reference of window row `lane`
                 const int slot4 = j & 3;   // a peer can only overwrite a slot four units later, after this CTA's arrive for j + 2
                 const uint32_t mine = smem_u32(&cstats[(slot4 * 8 + int(rank)) * 32 + lane]);
                 for (uint32_t r = 0; r < csize; ++r) st_remote_f2(mine, r, v[0]);
@@ -427,13 +367,12 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 #pragma unroll
                     for (int w = 0; w < 8; w += 2 * d) merge_stats(c8[w].x, c8[w].y, c8[w + d].x, c8[w + d].y);
                 const float m = c8[0].x, z = c8[0].y;
-                // weight of e = 2^(x - r) is 2^(r - m) / (n 2^-m + Z): one factor per window row
+                // weight of 2^(x - m) is 1 / (n 2^-m + Z); fold it and -m into one additive constant
                 const float denom = a.n * ex2f(-m) + z;
-                cv_team[lane] = (lane < W && z > 0.f) ? a.weight * ex2f(r_mine - m) / denom : 0.f;
+                cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
                 mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
             }
             team_sync(team);
-            tc_fence_after();                            // the e values other threads stored in pass 1
 
             // ---------------------------------- pass 2 ----------------------------------
             float* const out_s = a.score_self + (int64_t(x.b) * a.n_kv_heads + x.h) * a.max_len;
@@ -460,8 +399,8 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const uint32_t add_s = same & vis, add_c = ~same & vis;
                 float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
                 const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
-                // The whole row of e values goes to registers first and the buffer is handed back at once: the
-                // tensor core refills it (next unit) while the weights are still being summed here.
+                // The whole row of logits goes to registers first and the buffer is handed back at once: the
+                // tensor core refills it (next unit) while the weights are still being computed here.
                 uint32_t va[16], vb[16];
                 tc_ld_row16(va, row_addr);
                 tc_ld_row16(vb, row_addr + 16u);
@@ -471,7 +410,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 if (lane == 0) mbar_arrive(tmem_empty + 8 * buf);          // the tensor core may refill this buffer
                 // Common case: every window query carries the same label and no column of this tile is
                 // hidden.  Then a key's weights all go to one of the two sums, chosen once per key, and the
-                // columns beyond W add exact zeros (their factor is 0): plain sums, no selection.
+                // columns beyond W add exact zeros (their constant is -inf): plain sums, no selection.
                 const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
@@ -481,10 +420,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 #pragma unroll
                         for (int j4 = 0; j4 < 4; ++j4) {
                             const float4 cc = cv[j4];
-                            s0 = fmaf(__uint_as_float(cur[j4 * 4 + 0]), cc.x, s0);
-                            s1 = fmaf(__uint_as_float(cur[j4 * 4 + 1]), cc.y, s1);
-                            c0 = fmaf(__uint_as_float(cur[j4 * 4 + 2]), cc.z, c0);
-                            c1 = fmaf(__uint_as_float(cur[j4 * 4 + 3]), cc.w, c1);
+                            s0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                            s1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                            c0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                            c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
                         }
                         continue;
                     }
@@ -492,10 +431,10 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 #pragma unroll
                     for (int j4 = 0; j4 < 4; ++j4) {
                         const float4 cc = cv[j4];
-                        const float p0 = __uint_as_float(cur[j4 * 4 + 0]) * cc.x;
-                        const float p1 = __uint_as_float(cur[j4 * 4 + 1]) * cc.y;
-                        const float p2 = __uint_as_float(cur[j4 * 4 + 2]) * cc.z;
-                        const float p3 = __uint_as_float(cur[j4 * 4 + 3]) * cc.w;
+                        const float p0 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
+                        const float p1 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
+                        const float p2 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
+                        const float p3 = ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
                         s0 += (as >> (j4 * 4 + 0)) & 1u ? p0 : 0.f; c0 += (ac >> (j4 * 4 + 0)) & 1u ? p0 : 0.f;
                         s1 += (as >> (j4 * 4 + 1)) & 1u ? p1 : 0.f; c1 += (ac >> (j4 * 4 + 1)) & 1u ? p1 : 0.f;
                         s0 += (as >> (j4 * 4 + 2)) & 1u ? p2 : 0.f; c0 += (ac >> (j4 * 4 + 2)) & 1u ? p2 : 0.f;

@@ -88,6 +88,25 @@ def test_score_many_units_resident_clusters(csp, oracle, lens_hi, n_seq, heads):
     _run_score(csp, oracle, cfg, modality=mod.astype(np.uint8))
 
 
+@pytest.mark.parametrize("later_gain", [6.0, 0.05])
+def test_score_resident_clusters_logits_far_from_the_first_tile(csp, oracle, later_gain):
+    """The resident-cluster kernel stores 2^(x - r) with r taken from a unit's first tile.  Keys after the first
+    tile are scaled so that the largest logits sit about 60 nats above (or far below) that reference."""
+    rng = np.random.RandomState(3)
+    lens = tuple(int(x) for x in rng.randint(200, 900, size=40))
+    cfg = _case(lens, 8, 8, 128, 32, 32, seed=23)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    q = (q.float() * 3.0).to(cfg.dtype)
+    k = k.clone()
+    k[:, :, 128:] = (k[:, :, 128:].float() * later_gain).to(cfg.dtype)
+    p = gpu_params(csp, cfg)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).score()
+    assert run.status() == 0
+    s, c = oracle.score(orc_params(oracle, cfg), q.cpu(), k.cpu(), cfg.modality(), cfg.seq_lens)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent, "self")
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent, "cross")
+
+
 def test_score_mixed_modality_window_and_per_head_labels(csp, oracle):
     cfg = _case((600, 350), 4, 2, 128, 32, 32, seed=5)
     rng = np.random.RandomState(0)
