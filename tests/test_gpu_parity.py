@@ -572,6 +572,43 @@ def test_reprune_round_with_per_head_labels(csp, oracle):
     assert_compaction_exact(run2, mod2.cpu().numpy())
 
 
+def test_reprune_rounds_in_one_buffer(csp, oracle):
+    """Algorithm 1's iteration without a second cache: prune in place, append decode tokens behind the kept rows
+    of the same buffer, prune in place again.  Every round is compared with a two-buffer run on the same bytes."""
+    cfg = _case((800,), 4, 2, 128, 32, 32, seed=42, visual_pct=30, text_pct=40)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    p = gpu_params(csp, cfg)
+    two = GpuRun(csp, p, q, k.clone(), v.clone(), cfg.modality(), cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget).prune()
+    one = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget)
+    one.k_out, one.v_out = one.k, one.v
+    one.prune()
+    n1 = int(two.n_out[0, 0])
+    assert (two.n_out == n1).all() and torch.equal(one.n_out, two.n_out)
+    assert torch.equal(one.k[:, :, :n1], two.k_out[:, :, :n1]) and torch.equal(one.v[:, :, :n1], two.v_out[:, :, :n1])
+    g = torch.Generator(device="cuda").manual_seed(6)
+    bud = np.array([[60, 0, 0, 20]], np.int32)
+    for rnd in range(2):
+        add = 64
+        L2 = n1 + add
+        one.k[:, :, n1:L2] = torch.randn(1, 2, add, 128, device="cuda", generator=g).to(torch.bfloat16)
+        one.v[:, :, n1:L2] = torch.randn(1, 2, add, 128, device="cuda", generator=g).to(torch.bfloat16)
+        mod2 = torch.cat([one.mod_out[:, :, :n1], torch.zeros(1, 2, add, dtype=torch.uint8, device="cuda")], 2)
+        mod2 = torch.cat([mod2, torch.zeros(1, 2, cfg.max_len - L2, dtype=torch.uint8, device="cuda")], 2).contiguous()
+        q2 = torch.randn(1, 4, 32, 128, device="cuda", generator=g).to(torch.bfloat16)
+        two = GpuRun(csp, p, q2, one.k.clone(), one.v.clone(), mod2.cpu().numpy(), [L2], bud).prune()
+        nxt = GpuRun(csp, p, q2, one.k, one.v, mod2.cpu().numpy(), [L2], bud)
+        nxt.k_out, nxt.v_out = nxt.k, nxt.v
+        nxt.prune()
+        assert nxt.status() == 0 and torch.equal(nxt.n_out, two.n_out) and torch.equal(nxt.idx, two.idx)
+        for h in range(2):
+            n = int(two.n_out[0, h])
+            assert torch.equal(nxt.k[0, h, :n], two.k_out[0, h, :n]) and torch.equal(nxt.v[0, h, :n], two.v_out[0, h, :n])
+        assert torch.equal(nxt.mod_out, two.mod_out)
+        if not (two.n_out == two.n_out[0, 0]).all():
+            break                                         # heads diverged: a ragged append needs per-head lengths
+        one, n1 = nxt, int(two.n_out[0, 0])
+
+
 @pytest.mark.parametrize("budget_pct", [5, 40])
 def test_config4_reprune_rounds(csp, oracle, budget_pct):
     """Batched serving shape: prune the prompt cache (round 0), then four times append 64 decode tokens to
