@@ -205,7 +205,8 @@ def run_reference(args, rank, world):
 def kernels_per_call(p) -> int:
     """Kernels one csp_prune_layer call launches: score, select, compact, and, for a bf16 cache with more
     (sequence, head) units than SMs and several sequences, the kernel that orders them by length."""
-    ordered = p.dtype == 1 and 2 <= p.batch <= 4096 and p.batch * p.n_kv_heads > 148
+    units, tiles = p.batch * p.n_kv_heads, (p.max_len + 127) // 128
+    ordered = p.dtype == 1 and 2 <= p.batch <= 4096 and (units > 148 or units * min(tiles, 8) > 120)
     return 4 if ordered else 3
 
 

@@ -570,8 +570,11 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_te
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return CSP_ERR_UNSUPPORTED;
     if (p.dtype == CSP_F32) return launch_t<float>(p, a, tmap, s);
-    // more units than SMs and several sequences: take them longest first
-    if (p.batch >= 2 && p.batch <= 4096 && p.batch * p.n_kv_heads > 148) {
+    // several sequences and more CTAs than fit on the GPU at once (up to 8 per unit, 120 SMs hold clusters
+    // of 8): take the sequences longest first
+    const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
+    const long long units = (long long)p.batch * p.n_kv_heads;
+    if (p.batch >= 2 && p.batch <= 4096 && (units > 148 || units * (max_tiles < 8 ? max_tiles : 8) > 120)) {
         length_order_kernel<<<(p.batch + 255) / 256, 256, 0, s>>>(a.seq_lens, p.batch, p.max_len, a.order_buf);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
         a.order = a.order_buf;
