@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_
         const int shift = 24 - 8 * round;
         uint32_t* const hb = &hist[round & 1][0][0];
         for (int i = tid; i < 4 * 256; i += kCsThreads) hb[i] = 0;
-        if (round > 0) settle(shift + 8);
+        if (round > 0 && (live_s | live_c) != 0u) settle(shift + 8);   // most threads have no live key after a round or two
         __syncthreads();
         if (round == 0) {
             // the top byte (sign, high exponent bits) takes very few values: count this thread's keys
@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_
         }
         __syncthreads();
     }
-    settle(0);
+    if ((live_s | live_c) != 0u) settle(0);
     // live_* now marks the keys equal to their problem's K-th value: krem[p] of the eqcnt[p] such keys
     // are taken, the earliest positions first
 
