@@ -504,6 +504,19 @@ def main():
                 "frac": achieved / peak, "traffic": None if traffic is None else traffic * layers_per_launch,
                 "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": ab_launch[dominant], "us_per_launch": per[dominant] * 1e3}
+    # The scoring kernel takes one exponential per (query head of the group, window row, key): with G >= 3 that
+    # is more special-function work per K byte than the SMs can keep up with at the HBM peak, so the bound of
+    # that kernel is the ex2 rate (16 per clock and SM at the maximum SM clock), each exponential counted once.
+    if dominant == "score":
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        ex2_peak = 16.0 * sms * clocks["sm_max_mhz"] * 1e6 if clocks.get("sm_max_mhz") else None
+        n_exp = float(cfg.group * cfg.window * cfg.n_kv_heads) * float(cfg.seq_lens.sum()) * layers_per_launch
+        if ex2_peak and n_exp / ex2_peak > ab_launch["score"] / (peak * 1e9):
+            ex2_rate = n_exp / (per["score"] * 1e-3)
+            roofline = {"bound": "alu", "kernel": "score", "achieved": ex2_rate / 1e12, "peak": ex2_peak / 1e12,
+                        "unit": "T ex2/s", "frac": ex2_rate / ex2_peak, "traffic": roofline["traffic"],
+                        "peak_kind": "16 ex2 per clock and SM x SM count x maximum SM clock",
+                        "exponentials_per_launch": n_exp, "us_per_launch": per["score"] * 1e3, "hbm": roofline}
     path = {"algorithmic_bytes_per_layer": ab["total"], "us_per_layer": ms_step * 1e3 / n_layers,
             "achieved_gbs": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9,
             "frac_of_hbm_peak": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9 / peak,
