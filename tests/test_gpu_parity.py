@@ -74,13 +74,14 @@ def test_score_matches_oracle(csp, oracle, lens, n_q, n_kv, d, W, R, dtype):
     _run_score(csp, oracle, _case(lens, n_q, n_kv, d, W, R, dtype=dtype, seed=len(lens) + n_q))
 
 
-@pytest.mark.parametrize("lens_hi,n_seq,heads", [(1000, 40, 8), (2500, 20, 16)])
-def test_score_many_units_resident_clusters(csp, oracle, lens_hi, n_seq, heads):
+@pytest.mark.parametrize("lens_hi,n_seq,heads,d", [(1000, 40, 8, 128), (2500, 20, 16, 128), (1800, 40, 8, 64),
+                                                    (5000, 10, 32, 64)])
+def test_score_many_units_resident_clusters(csp, oracle, lens_hi, n_seq, heads, d):
     """More MHA units than clusters fit on the GPU: the resident-cluster kernel walks unit after unit
-    (clusters of 1 and of 4 CTAs), ragged lengths, every unit compared."""
+    (clusters of 1, 2 and 4 CTAs; 256- and 128-byte rows), ragged lengths, every unit compared."""
     rng = np.random.RandomState(lens_hi)
     lens = tuple(int(x) for x in rng.randint(90, lens_hi, size=n_seq))
-    cfg = _case(lens, heads, heads, 128, 32, 32, seed=17)
+    cfg = _case(lens, heads, heads, d, 32, 32, seed=17)
     mod = cfg.modality()
     mod[:, -40:] = (rng.rand(n_seq, 40) < 0.3)          # padding labels and some mixed windows
     for b, L in enumerate(lens):
@@ -512,6 +513,53 @@ def test_config4_sampled_units(csp, oracle):
     rng = np.random.RandomState(0)
     units = [(int(rng.randint(32)), int(rng.randint(32))) for _ in range(4)]
     _sampled_units_check(csp, oracle, cfg, units)
+
+
+def _folded_sampled_units_check(csp, oracle, cfg, n_fold, units):
+    """The bench's default launch: `n_fold` layers stacked on the batch axis of one call, so that the
+    kernels see as many units as there (resident clusters for MHA, clusters of two taken longest first
+    for GQA).  The oracle recomputes sampled (layer, sequence, KV head) units from the same bytes."""
+    parts = [synth.make_layer(cfg, i, "cuda") for i in range(n_fold)]
+    q, k, v = (torch.cat([x[j] for x in parts], 0) for j in range(3))
+    del parts
+    p = gpu_params(csp, cfg)
+    p.batch = cfg.batch * n_fold
+    mod1 = cfg.modality()
+    mod = np.tile(mod1, (n_fold, 1))
+    lens = np.tile(cfg.seq_lens, n_fold)
+    budgets = np.tile(cfg.budgets, (n_fold, 1))
+    total = None if cfg.total_budget is None else np.tile(cfg.total_budget, n_fold)
+    run = GpuRun(csp, p, q, k, v, mod, lens, budgets, total_budget=total).prune()
+    assert run.status() in (0, csp.DEV_K_CLAMPED)
+    G, B = cfg.group, cfg.batch
+    for layer, b, h in units:
+        fb = layer * B + b
+        L = int(cfg.seq_lens[b])
+        op = oracle.Params(1, G, 1, cfg.head_dim, cfg.window, cfg.recent, L, p.out_capacity)
+        ref = oracle.prune_layer(op, q[fb:fb + 1, h * G:(h + 1) * G].cpu(), k[fb:fb + 1, h:h + 1, :L].cpu(),
+                                 v[fb:fb + 1, h:h + 1, :L].cpu(), mod1[b:b + 1, :L], np.array([L], np.int32),
+                                 cfg.budgets[b:b + 1],
+                                 None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
+        assert_scores_close(run.ss[fb:fb + 1, h:h + 1, :L].cpu().numpy(), ref["score_self"], [L], cfg.recent)
+        assert_scores_close(run.sc[fb:fb + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], cfg.recent)
+        assert_index_sets_match(run.idx[fb:fb + 1, h:h + 1].cpu().numpy(),
+                                run.n_out[fb:fb + 1, h:h + 1].cpu().numpy(), ref, mod1[b:b + 1, :L], [L], cfg.recent)
+    assert_compaction_exact(run, mod)
+    # every layer of a sequence keeps the same number of rows (budgets and labels repeat)
+    n = run.n_out.cpu().numpy().reshape(n_fold, B, cfg.n_kv_heads)
+    assert (n > 0).all() and (n == n[0, :, :1]).all()
+
+
+def test_config1_layers_folded_into_one_call(csp, oracle):
+    _folded_sampled_units_check(csp, oracle, synth.config(1), 8, [(0, 0, 0), (3, 0, 17), (7, 0, 31)])
+
+
+def test_config2_layers_folded_into_one_call(csp, oracle):
+    _folded_sampled_units_check(csp, oracle, synth.config(2), 4, [(0, 0, 5), (3, 0, 30)])
+
+
+def test_config3_layers_folded_into_one_call(csp, oracle):
+    _folded_sampled_units_check(csp, oracle, synth.config(3), 5, [(0, 3, 0), (2, 1, 3), (4, 0, 2)])
 
 
 def test_host_buffer_entry_point(csp, oracle):
