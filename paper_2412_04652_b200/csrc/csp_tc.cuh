@@ -85,6 +85,12 @@ __device__ __forceinline__ uint64_t sw128_desc(uint32_t smem_addr) {
     d |= uint64_t(2) << 61;                // SWIZZLE_128B
     return d;
 }
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float lg2f(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -127,19 +133,21 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 template <int NB>
 __device__ __forceinline__ void stats_block(const uint32_t (&v0)[4 * NB], const uint32_t (&v1)[4 * NB],
                                             float (&m)[2 * NB], float (&z)[2 * NB], float scale2) {
-    float mx[2 * NB];
+    float mx[2 * NB];       // largest raw value of the slot (scale2 > 0: scaling keeps the order)
     bool raise = false;
 #pragma unroll
     for (int jj = 0; jj < 2 * NB; ++jj) {
         const int i = (jj >> 1) * 4 + (jj & 1);
-        mx[jj] = fmaxf(fmaxf(__uint_as_float(v0[i]), __uint_as_float(v0[i + 2])),
-                       fmaxf(__uint_as_float(v1[i]), __uint_as_float(v1[i + 2]))) * scale2;
-        raise |= mx[jj] > m[jj] + kLazy;
+        mx[jj] = fmax3(__uint_as_float(v0[i]), __uint_as_float(v0[i + 2]),
+                       fmaxf(__uint_as_float(v1[i]), __uint_as_float(v1[i + 2])));
+        raise |= fmaf(mx[jj], scale2, -m[jj]) > kLazy;
     }
     if (raise) {
 #pragma unroll
-        for (int jj = 0; jj < 2 * NB; ++jj)
-            if (mx[jj] > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - mx[jj]); m[jj] = mx[jj]; }
+        for (int jj = 0; jj < 2 * NB; ++jj) {
+            const float ms = mx[jj] * scale2;
+            if (ms > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - ms); m[jj] = ms; }
+        }
     }
 #pragma unroll
     for (int jj = 0; jj < 2 * NB; ++jj) {
