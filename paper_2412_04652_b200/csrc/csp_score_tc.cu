@@ -399,14 +399,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             };
             // The thread's columns come in chunks of 16: chunk k sits kStep columns after chunk k - 1 (both
             // halves of every head, or this set's half of every head) and uses bits kShift(k) of the masks.
-            // Two chunks per iteration, the load of the next one in flight while one is turned into weights;
-            // kept as a real loop for G > 2 so that the code stays small.
+            // Two chunks per iteration, the load of the next one in flight while one is turned into weights.
+            // Fully unrolled for every G: with 7 heads the rolled loop was 4-8 % slower (address arithmetic
+            // and a branch per 32 exponentials in a loop that is bound by instruction issue).
             constexpr int kChunks = EP::kSplit ? G : 2 * G;
             constexpr int kStep = EP::kSplit ? 32 : 16;
             const float* const cv_mine = cvec + cofs;
             auto shift_of = [&](int k) { return EP::kSplit ? cofs : (k & 1) * 16; };
             if (plain) {
-#pragma unroll(G <= 2 ? G : 1)
+#pragma unroll
                 for (int k = 0; k < kChunks; k += 2) {
                     tc_wait_ld();
                     if (k + 1 < kChunks) tc_ld_row16(vb, row_addr + uint32_t((k + 1) * kStep));
@@ -421,7 +422,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                 s0 = same ? total : 0.f; s1 = 0.f;
                 c0 = same ? 0.f : total; c1 = 0.f;
             } else {
-#pragma unroll(G <= 2 ? G : 1)
+#pragma unroll
                 for (int k = 0; k < kChunks; k += 2) {
                     tc_wait_ld();
                     if (k + 1 < kChunks) tc_ld_row16(vb, row_addr + uint32_t((k + 1) * kStep));
