@@ -363,6 +363,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // the row of 32 G logits is read in chunks of 16 columns; the load of the next chunk is in
             // flight while the current one is turned into weights (two accumulators per score)
             float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
+            float2 p01 = make_float2(0.f, 0.f), p23 = make_float2(0.f, 0.f);   // the plain sums, two-wide
             const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC + cofs);
             uint32_t va[16], vb[16];
             tc_ld_row16(va, row_addr);
@@ -389,12 +390,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             auto chunk_plain = [&](const uint32_t (&cur)[16], const float* cvp) {
                 const float4* cv = reinterpret_cast<const float4*>(cvp);
 #pragma unroll
+                const float2 sc2 = make_float2(scale2, scale2);
                 for (int j4 = 0; j4 < 4; ++j4) {
                     const float4 cc = cv[j4];
-                    s0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
-                    s1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
-                    c0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
-                    c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                    p01 = __fadd2_rn(p01, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 0]), __uint_as_float(cur[j4 * 4 + 1])),
+                                                           sc2, make_float2(cc.x, cc.y))));
+                    p23 = __fadd2_rn(p23, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 2]), __uint_as_float(cur[j4 * 4 + 3])),
+                                                           sc2, make_float2(cc.z, cc.w))));
                 }
             };
             // The thread's columns come in chunks of 16: chunk k sits kStep columns after chunk k - 1 (both
@@ -418,7 +420,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                         chunk_plain(vb, cv_mine + (k + 1) * kStep);
                     }
                 }
-                const float total = (s0 + s1) + (c0 + c1);
+                const float total = (p01.x + p01.y) + (p23.x + p23.y);
                 s0 = same ? total : 0.f; s1 = 0.f;
                 c0 = same ? 0.f : total; c1 = 0.f;
             } else {

@@ -124,6 +124,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     }
 }
 
+__device__ __forceinline__ float2 ex2f2(float2 x) { return make_float2(ex2f(x.x), ex2f(x.y)); }
+
 // ---- pass-1 row statistics of one accumulator block of 32 rows x 8 NB columns ----------------------------
 // v0 / v1: the two 16-row halves as loaded by tc_ld_frag.  Statistic slot jj = 2 nt + e belongs to column
 // 8 nt + 2 (lane % 4) + e of the block; (m, z) is a running (reference, sum of 2^(x scale2 - reference)) over
@@ -149,12 +151,20 @@ __device__ __forceinline__ void stats_block(const uint32_t (&v0)[4 * NB], const 
             if (ms > m[jj] + kLazy) { z[jj] *= ex2f(m[jj] - ms); m[jj] = ms; }
         }
     }
+    // Slots 2 b and 2 b + 1 sit in neighbouring registers of every fragment, so the scaling and the sums run
+    // as two-wide fp32 instructions (same roundings and summation order as the scalar form, half the
+    // instructions to issue).
+    const float2 sc2 = make_float2(scale2, scale2);
 #pragma unroll
-    for (int jj = 0; jj < 2 * NB; ++jj) {
-        const int i = (jj >> 1) * 4 + (jj & 1);
-        const float nm = -m[jj];
-        z[jj] += (ex2f(fmaf(__uint_as_float(v0[i]), scale2, nm)) + ex2f(fmaf(__uint_as_float(v0[i + 2]), scale2, nm))) +
-                 (ex2f(fmaf(__uint_as_float(v1[i]), scale2, nm)) + ex2f(fmaf(__uint_as_float(v1[i + 2]), scale2, nm)));
+    for (int bq = 0; bq < NB; ++bq) {
+        const float2 nm = make_float2(-m[2 * bq], -m[2 * bq + 1]);
+        const float2 ea = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v0[4 * bq]), __uint_as_float(v0[4 * bq + 1])), sc2, nm));
+        const float2 eb = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v0[4 * bq + 2]), __uint_as_float(v0[4 * bq + 3])), sc2, nm));
+        const float2 ec = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v1[4 * bq]), __uint_as_float(v1[4 * bq + 1])), sc2, nm));
+        const float2 ed = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v1[4 * bq + 2]), __uint_as_float(v1[4 * bq + 3])), sc2, nm));
+        const float2 zz = __fadd2_rn(make_float2(z[2 * bq], z[2 * bq + 1]), __fadd2_rn(__fadd2_rn(ea, eb), __fadd2_rn(ec, ed)));
+        z[2 * bq] = zz.x;
+        z[2 * bq + 1] = zz.y;
     }
 }
 // The same for a tile that reaches into the window: key t is visible to window column w iff w < W and
