@@ -398,6 +398,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const uint32_t vis = delta <= 0 ? wmask : (delta >= 32 ? 0u : (wmask & (0xFFFFFFFFu << delta)));
                 const uint32_t add_s = same & vis, add_c = ~same & vis;
                 float s0 = 0.f, s1 = 0.f, c0 = 0.f, c1 = 0.f;
+                float2 p01 = make_float2(0.f, 0.f), p23 = make_float2(0.f, 0.f);   // the plain sums
                 const uint32_t row_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(buf * NC);
                 // The whole row of logits goes to registers first and the buffer is handed back at once: the
                 // tensor core refills it (next unit) while the weights are still being computed here.
@@ -417,13 +418,15 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     uint32_t (&cur)[16] = ch ? vb : va;
                     const float4* cv = reinterpret_cast<const float4*>(cv_team + ch * 16);
                     if (plain) {
+                        // two-wide fp32 instructions: same roundings and order as four scalar sums
+                        const float2 sc2 = make_float2(scale2, scale2);
 #pragma unroll
                         for (int j4 = 0; j4 < 4; ++j4) {
                             const float4 cc = cv[j4];
-                            s0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 0]), scale2, cc.x));
-                            s1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 1]), scale2, cc.y));
-                            c0 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 2]), scale2, cc.z));
-                            c1 += ex2f(fmaf(__uint_as_float(cur[j4 * 4 + 3]), scale2, cc.w));
+                            p01 = __fadd2_rn(p01, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 0]), __uint_as_float(cur[j4 * 4 + 1])),
+                                                                   sc2, make_float2(cc.x, cc.y))));
+                            p23 = __fadd2_rn(p23, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 2]), __uint_as_float(cur[j4 * 4 + 3])),
+                                                                   sc2, make_float2(cc.z, cc.w))));
                         }
                         continue;
                     }
@@ -442,7 +445,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                     }
                 }
                 if (plain) {
-                    const float total = (s0 + s1) + (c0 + c1);
+                    const float total = (p01.x + p01.y) + (p23.x + p23.y);
                     s0 = same ? total : 0.f; s1 = 0.f;
                     c0 = same ? 0.f : total; c1 = 0.f;
                 }
