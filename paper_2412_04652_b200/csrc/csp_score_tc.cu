@@ -31,6 +31,7 @@ using namespace dev;
 template <int G> struct EpiPlan {
     static constexpr bool kSplit = G >= 3;              // two warp sets, each with half of the window columns
     static constexpr int kSets = kSplit ? 2 : 1;
+    static constexpr bool kFmaExp = kSplit;             // one pair of exponentials in eight on the FMA pipe
     static constexpr int kWarps = 8 * kSets;
     static constexpr int kEpiThreads = 32 * kWarps;
     static constexpr int kBlocks = kSplit ? 2 : 4;      // 8-column blocks per head and thread in pass 1
@@ -280,7 +281,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                 tc_ld_frag(v0, tmem_base + (uint32_t(quarter * 32) << 16) + col);
                 tc_ld_frag(v1, tmem_base + (uint32_t(quarter * 32 + 16) << 16) + col);
                 tc_wait_ld();
-                if (!masked) stats_block<NB>(v0, v1, m_run[g], z_run[g], scale2);
+                if (!masked) stats_block<NB, EP::kFmaExp>(v0, v1, m_run[g], z_run[g], scale2);
                 else stats_block_masked<NB>(v0, v1, m_run[g], z_run[g], scale2, t_base, first_masked_key, W, cofs + lq * 2);
             }
             if (i >= kept) {                      // streaming buffer: hand it back to the MMA issuer
@@ -395,8 +396,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
                     const float4 cc = cv[j4];
                     p01 = __fadd2_rn(p01, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 0]), __uint_as_float(cur[j4 * 4 + 1])),
                                                            sc2, make_float2(cc.x, cc.y))));
-                    p23 = __fadd2_rn(p23, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 2]), __uint_as_float(cur[j4 * 4 + 3])),
-                                                           sc2, make_float2(cc.z, cc.w))));
+                    const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 2]), __uint_as_float(cur[j4 * 4 + 3])),
+                                                  sc2, make_float2(cc.z, cc.w));
+                    p23 = __fadd2_rn(p23, (EP::kFmaExp && j4 == 3) ? ex2_fma2(x23) : ex2f2(x23));
                 }
             };
             // The thread's columns come in chunks of 16: chunk k sits kStep columns after chunk k - 1 (both

@@ -125,6 +125,20 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 
 __device__ __forceinline__ float2 ex2f2(float2 x) { return make_float2(ex2f(x.x), ex2f(x.y)); }
+// 2^x for two values on the FMA pipe instead of the special-function unit: x rounded to the nearest integer j
+// with the 1.5 * 2^23 trick, a cubic for 2^f on f = x - j in [-0.5, 0.5] (minimax in the relative error,
+// 7.5e-5), and j added to the exponent field.  x <= 126; below -125 the result stays at about 2^-125.
+__device__ __forceinline__ float2 ex2_fma2(float2 x) {
+    x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
+    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
+    const float2 j = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __ffma2_rn(j, make_float2(-1.f, -1.f), x);
+    float2 p = __ffma2_rn(make_float2(0.0551716648f, 0.0551716648f), f, make_float2(0.2426111251f, 0.2426111251f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677f, 0.6932609677f));
+    p = __ffma2_rn(p, f, make_float2(0.9999280572f, 0.9999280572f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
+}
 
 // ---- pass-1 row statistics of one accumulator block of 32 rows x 8 NB columns ----------------------------
 // v0 / v1: the two 16-row halves as loaded by tc_ld_frag.  Statistic slot jj = 2 nt + e belongs to column
@@ -132,7 +146,8 @@ __device__ __forceinline__ float2 ex2f2(float2 x) { return make_float2(ex2f(x.x)
 // the keys this thread has seen.  The reference is only raised when a value exceeds it by more than kLazy,
 // which is rare after the first tiles: the test is taken once for the whole block, so that the exponentials
 // that follow are straight-line code.  scale2 > 0.
-template <int NB>
+// kFma: one pair of exponentials in eight goes to the FMA pipe (kernels bound by the special-function unit).
+template <int NB, bool kFma = false>
 __device__ __forceinline__ void stats_block(const uint32_t (&v0)[4 * NB], const uint32_t (&v1)[4 * NB],
                                             float (&m)[2 * NB], float (&z)[2 * NB], float scale2) {
     float mx[2 * NB];       // largest raw value of the slot (scale2 > 0: scaling keeps the order)
@@ -161,7 +176,8 @@ __device__ __forceinline__ void stats_block(const uint32_t (&v0)[4 * NB], const 
         const float2 ea = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v0[4 * bq]), __uint_as_float(v0[4 * bq + 1])), sc2, nm));
         const float2 eb = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v0[4 * bq + 2]), __uint_as_float(v0[4 * bq + 3])), sc2, nm));
         const float2 ec = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v1[4 * bq]), __uint_as_float(v1[4 * bq + 1])), sc2, nm));
-        const float2 ed = ex2f2(__ffma2_rn(make_float2(__uint_as_float(v1[4 * bq + 2]), __uint_as_float(v1[4 * bq + 3])), sc2, nm));
+        const float2 xd = __ffma2_rn(make_float2(__uint_as_float(v1[4 * bq + 2]), __uint_as_float(v1[4 * bq + 3])), sc2, nm);
+        const float2 ed = (kFma && (bq & 1)) ? ex2_fma2(xd) : ex2f2(xd);
         const float2 zz = __fadd2_rn(make_float2(z[2 * bq], z[2 * bq + 1]), __fadd2_rn(__fadd2_rn(ea, eb), __fadd2_rn(ec, ed)));
         z[2 * bq] = zz.x;
         z[2 * bq + 1] = zz.y;
