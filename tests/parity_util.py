@@ -92,6 +92,24 @@ def assert_index_sets_match(gpu_idx, gpu_n, ref, modality, seq_lens, recent, glo
     return tolerated
 
 
+def assert_selection_follows_own_scores(orc, op, gpu_ss, gpu_sc, gpu_idx, gpu_n, modality, seq_lens, budgets,
+                                         total_budget=None):
+    """Given the scores the GPU itself produced, its selection must be the exact one: every top-K problem keeps
+    precisely min(k, candidates) keys, the best ones in (score, position) order, combined as the mode says.
+    This is what makes a tolerated boundary-band difference against the oracle's scores harmless: the GPU set is
+    then the exact answer for scores that lie within the score tolerance.  `op` carries the mode switches."""
+    idx, n_out, _, _ = orc.select(op, np.ascontiguousarray(gpu_ss, np.float32), np.ascontiguousarray(gpu_sc, np.float32),
+                                  modality, np.asarray(seq_lens, np.int32), np.asarray(budgets, np.int32),
+                                  None if total_budget is None else np.asarray(total_budget, np.int32))
+    np.testing.assert_array_equal(np.asarray(gpu_n), n_out)
+    B, H = n_out.shape
+    for b in range(B):
+        for h in range(H):
+            n = int(n_out[b, h])
+            if n > 0:
+                np.testing.assert_array_equal(np.asarray(gpu_idx)[b, h, :n], idx[b, h, :n])
+
+
 class GpuRun:
     """Device copies of one layer's inputs plus freshly allocated outputs."""
 

@@ -5,8 +5,8 @@ import pytest
 import torch
 
 import csp_synth as synth
-from parity_util import (GpuRun, assert_compaction_exact, assert_index_sets_match, assert_scores_close,
-                         bits, gpu_params, orc_params)
+from parity_util import (GpuRun, assert_compaction_exact, assert_index_sets_match,
+                         assert_selection_follows_own_scores, assert_scores_close, bits, gpu_params, orc_params)
 
 pytestmark = pytest.mark.gpu
 
@@ -91,8 +91,8 @@ def test_score_many_units_resident_clusters(csp, oracle, lens_hi, n_seq, heads, 
 
 @pytest.mark.parametrize("later_gain", [6.0, 0.05])
 def test_score_resident_clusters_logits_far_from_the_first_tile(csp, oracle, later_gain):
-    """The resident-cluster kernel stores 2^(x - r) with r taken from a unit's first tile.  Keys after the first
-    tile are scaled so that the largest logits sit about 60 nats above (or far below) that reference."""
+    """Keys after a unit's first tile are scaled so that the largest logits sit about 60 nats above (or far
+    below) those of the first tile: the running reference of the resident-cluster kernel has to follow."""
     rng = np.random.RandomState(3)
     lens = tuple(int(x) for x in rng.randint(200, 900, size=40))
     cfg = _case(lens, 8, 8, 128, 32, 32, seed=23)
@@ -411,6 +411,9 @@ def test_prune_layer_small(csp, oracle, mode):
     assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, cfg.recent)
     assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens,
                             cfg.recent, global_mode=mode.get("select_mode") == 1, overall=mode.get("select_mode") == 2)
+    assert_selection_follows_own_scores(oracle, orc_params(oracle, cfg, **mode), run.ss.cpu().numpy(),
+                                        run.sc.cpu().numpy(), run.idx.cpu().numpy(), run.n_out.cpu().numpy(),
+                                        cfg.modality(), cfg.seq_lens, cfg.budgets, cfg.total_budget)
     assert_compaction_exact(run, cfg.modality())
     if not mode:
         np.testing.assert_array_equal(run.n_out.cpu().numpy(), ref["n_out"])
@@ -467,99 +470,136 @@ def test_config1_one_layer_full(csp, oracle):
     assert (run.n_out.cpu().numpy() == 1027).all()
 
 
-def _sampled_units_check(csp, oracle, cfg, units, layer=0):
-    """Full-size GPU run in the launch configuration the bench uses; the oracle recomputes sampled
-    (sequence, KV head) units one by one from the bytes the GPU read."""
-    q, k, v = synth.make_layer(cfg, layer, "cuda")
-    p = gpu_params(csp, cfg)
-    mod = cfg.modality()
-    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, cfg.budgets, total_budget=cfg.total_budget).prune()
-    # budgets above the candidate count are clamped (and flagged); everything else must be clean
-    want = np.zeros(cfg.batch, np.int64)
-    clamped = False
+def _check_units_against_oracle(csp, oracle, cfg, run, q, k, v, units, label_row, budgets, total):
+    """The oracle recomputes the listed units of a finished GPU run from the bytes the GPU read.
+    units: (folded batch index fb, sequence b, KV head h).  The sampled units are laid out as a batch with one
+    KV head per entry so that the oracle, which is parallel across units only, does them in one call.
+    label_row(fb, b, h) -> uint8 labels of that unit, length >= L_b."""
+    G, d, R = cfg.group, cfg.head_dim, cfg.recent
+    n = len(units)
+    all_lens = run.lens.cpu().numpy()
+    lens = np.array([all_lens[fb] for fb, _, _ in units], np.int32)
+    Lm, cap = int(lens.max()), run.p.out_capacity
+    h_ss, h_sc, h_idx, h_n = (t.cpu().numpy() for t in (run.ss, run.sc, run.idx, run.n_out))
+    qs = torch.stack([q[fb, h * G:(h + 1) * G] for fb, _, h in units]).cpu()
+    ks = torch.zeros((n, 1, Lm, d), dtype=k.dtype)
+    vs = torch.zeros((n, 1, Lm, d), dtype=k.dtype)
+    mods = np.zeros((n, Lm), np.uint8)
+    g_ss, g_sc = np.zeros((n, 1, Lm), np.float32), np.zeros((n, 1, Lm), np.float32)
+    g_idx, g_n = np.full((n, 1, cap), -1, np.int32), np.zeros((n, 1), np.int32)
+    for i, (fb, b, h) in enumerate(units):
+        L = int(lens[i])
+        ks[i, 0, :L], vs[i, 0, :L] = k[fb, h, :L].cpu(), v[fb, h, :L].cpu()
+        mods[i, :L] = label_row(fb, b, h)[:L]
+        g_ss[i, 0, :L], g_sc[i, 0, :L] = h_ss[fb, h, :L], h_sc[fb, h, :L]
+        g_idx[i, 0], g_n[i, 0] = h_idx[fb, h], h_n[fb, h]
+    bud = np.stack([budgets[b] for _, b, _ in units]).astype(np.int32)
+    tot = None if total is None else np.array([total[b] for _, b, _ in units], np.int32)
+    op = oracle.Params(n, G, 1, d, cfg.window, R, Lm, cap)
+    ref = oracle.prune_layer(op, qs, ks, vs, mods, lens, bud, tot)
+    assert_scores_close(g_ss, ref["score_self"], lens, R, "self")
+    assert_scores_close(g_sc, ref["score_cross"], lens, R, "cross")
+    tolerated = assert_index_sets_match(g_idx, g_n, ref, mods, lens, R)
+    assert_selection_follows_own_scores(oracle, op, g_ss, g_sc, g_idx, g_n, mods, lens, bud, tot)
+    return tolerated
+
+
+def _expected_rows(cfg, csp):
+    """Rows every head of a sequence keeps when the window is text only (disjoint supports), and whether a
+    budget had to be clamped."""
+    want, clamped = np.zeros(cfg.batch, np.int64), False
     for b, lay in enumerate(cfg.layouts):
         n_text, n_vis = synth.candidate_counts(lay, cfg.recent)
         ks, kc = int(cfg.budgets[b, 0]), int(cfg.budgets[b, 3])
         clamped |= ks > n_text or kc > n_vis
         want[b] = min(ks, n_text) + min(kc, n_vis) + cfg.recent
-    assert run.status() == (csp.DEV_K_CLAMPED if clamped else 0)
-    G = cfg.group
-    for b, h in units:
-        L = int(cfg.seq_lens[b])
-        op = oracle.Params(1, G, 1, cfg.head_dim, cfg.window, cfg.recent, L, p.out_capacity)
-        ref = oracle.prune_layer(op, q[b:b + 1, h * G:(h + 1) * G].cpu(), k[b:b + 1, h:h + 1, :L].cpu(),
-                                 v[b:b + 1, h:h + 1, :L].cpu(), mod[b:b + 1, :L], np.array([L], np.int32),
-                                 cfg.budgets[b:b + 1],
-                                 None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
-        assert_scores_close(run.ss[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_self"], [L], cfg.recent)
-        assert_scores_close(run.sc[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], cfg.recent)
-        assert_index_sets_match(run.idx[b:b + 1, h:h + 1].cpu().numpy(), run.n_out[b:b + 1, h:h + 1].cpu().numpy(),
-                                ref, mod[b:b + 1, :L], [L], cfg.recent)
-    assert_compaction_exact(run, mod)
-    # properties that hold at any size
-    assert (run.n_out.cpu().numpy() == want[:, None]).all()
+    return want, (csp.DEV_K_CLAMPED if clamped else 0)
 
 
-def test_config2_sampled_units(csp, oracle):
-    _sampled_units_check(csp, oracle, synth.config(2), [(0, 0), (0, 17), (0, 31)])
-
-
-def test_config3_sampled_units(csp, oracle):
-    _sampled_units_check(csp, oracle, synth.config(3), [(0, 1), (3, 2)])
-
-
-def test_config4_sampled_units(csp, oracle):
-    cfg = synth.config(4, budget_pct=20)
-    rng = np.random.RandomState(0)
-    units = [(int(rng.randint(32)), int(rng.randint(32))) for _ in range(4)]
-    _sampled_units_check(csp, oracle, cfg, units)
-
-
-def _folded_sampled_units_check(csp, oracle, cfg, n_fold, units):
-    """The bench's default launch: `n_fold` layers stacked on the batch axis of one call, so that the
-    kernels see as many units as there (resident clusters for MHA, clusters of two taken longest first
-    for GQA).  The oracle recomputes sampled (layer, sequence, KV head) units from the same bytes."""
-    parts = [synth.make_layer(cfg, i, "cuda") for i in range(n_fold)]
-    q, k, v = (torch.cat([x[j] for x in parts], 0) for j in range(3))
+def _full_size_check(csp, oracle, cfg, n_fold, n_sampled, first_layer=0, seed=0):
+    """Full-size workload in the launch configuration the bench times: `n_fold` layers stacked on the batch
+    axis of one call (n_fold = 1: one call for one layer).  Layer `first_layer` is compared in full, every
+    (sequence, KV head) unit of it, and `n_sampled` seeded random (layer, sequence, KV head) units of the
+    other layers are recomputed one by one.  Compaction is checked for every unit of the launch."""
+    parts = [synth.make_layer(cfg, first_layer + i, "cuda") for i in range(n_fold)]
+    q, k, v = (torch.cat([x[j] for x in parts], 0) for j in range(3)) if n_fold > 1 else parts[0]
     del parts
     p = gpu_params(csp, cfg)
     p.batch = cfg.batch * n_fold
     mod1 = cfg.modality()
     mod = np.tile(mod1, (n_fold, 1))
     lens = np.tile(cfg.seq_lens, n_fold)
-    budgets = np.tile(cfg.budgets, (n_fold, 1))
     total = None if cfg.total_budget is None else np.tile(cfg.total_budget, n_fold)
-    run = GpuRun(csp, p, q, k, v, mod, lens, budgets, total_budget=total).prune()
-    assert run.status() in (0, csp.DEV_K_CLAMPED)
-    G, B = cfg.group, cfg.batch
-    for layer, b, h in units:
-        fb = layer * B + b
-        L = int(cfg.seq_lens[b])
-        op = oracle.Params(1, G, 1, cfg.head_dim, cfg.window, cfg.recent, L, p.out_capacity)
-        ref = oracle.prune_layer(op, q[fb:fb + 1, h * G:(h + 1) * G].cpu(), k[fb:fb + 1, h:h + 1, :L].cpu(),
-                                 v[fb:fb + 1, h:h + 1, :L].cpu(), mod1[b:b + 1, :L], np.array([L], np.int32),
-                                 cfg.budgets[b:b + 1],
-                                 None if cfg.total_budget is None else cfg.total_budget[b:b + 1])
-        assert_scores_close(run.ss[fb:fb + 1, h:h + 1, :L].cpu().numpy(), ref["score_self"], [L], cfg.recent)
-        assert_scores_close(run.sc[fb:fb + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], cfg.recent)
-        assert_index_sets_match(run.idx[fb:fb + 1, h:h + 1].cpu().numpy(),
-                                run.n_out[fb:fb + 1, h:h + 1].cpu().numpy(), ref, mod1[b:b + 1, :L], [L], cfg.recent)
+    run = GpuRun(csp, p, q, k, v, mod, lens, np.tile(cfg.budgets, (n_fold, 1)), total_budget=total).prune()
+    want, st = _expected_rows(cfg, csp)
+    assert run.status() == st
+    B, H = cfg.batch, cfg.n_kv_heads
+    units = [(b, b, h) for b in range(B) for h in range(H)]                      # the first layer in full
+    rng = np.random.RandomState(seed)
+    while len(units) < B * H + n_sampled and n_fold > 1:
+        layer, b, h = int(rng.randint(1, n_fold)), int(rng.randint(B)), int(rng.randint(H))
+        units.append((layer * B + b, b, h))
+    tolerated = 0
+    for i in range(0, len(units), 256):                                          # bounded host memory per call
+        tolerated += _check_units_against_oracle(csp, oracle, cfg, run, q, k, v, units[i:i + 256],
+                                                 lambda fb, b, h: mod1[b], cfg.budgets, cfg.total_budget)
     assert_compaction_exact(run, mod)
-    # every layer of a sequence keeps the same number of rows (budgets and labels repeat)
-    n = run.n_out.cpu().numpy().reshape(n_fold, B, cfg.n_kv_heads)
-    assert (n > 0).all() and (n == n[0, :, :1]).all()
+    # properties that hold at any size: every layer of a sequence keeps the expected number of rows
+    n = run.n_out.cpu().numpy().reshape(n_fold, B, H)
+    assert (n == want[None, :, None]).all()
+    return len(units), tolerated
 
 
-def test_config1_layers_folded_into_one_call(csp, oracle):
-    _folded_sampled_units_check(csp, oracle, synth.config(1), 8, [(0, 0, 0), (3, 0, 17), (7, 0, 31)])
+def test_config1_all_layers_in_one_call(csp, oracle):
+    n, _ = _full_size_check(csp, oracle, synth.config(1), 32, 64)
+    assert n == 32 + 64
 
 
-def test_config2_layers_folded_into_one_call(csp, oracle):
-    _folded_sampled_units_check(csp, oracle, synth.config(2), 4, [(0, 0, 5), (3, 0, 30)])
+def test_config2_all_layers_in_one_call(csp, oracle):
+    n, _ = _full_size_check(csp, oracle, synth.config(2), 32, 64)
+    assert n == 32 + 64
 
 
-def test_config3_layers_folded_into_one_call(csp, oracle):
-    _folded_sampled_units_check(csp, oracle, synth.config(3), 5, [(0, 3, 0), (2, 1, 3), (4, 0, 2)])
+def test_config3_all_layers_in_one_call(csp, oracle):
+    n, _ = _full_size_check(csp, oracle, synth.config(3), 28, 64)
+    assert n == 16 + 64
+
+
+@pytest.mark.parametrize("budget_pct", [5, 10, 20, 40])
+def test_config4_budget_sweep_round0(csp, oracle, budget_pct):
+    """The serving shape is timed one call per layer over four distinct layer buffers: layer 0 in full
+    (1024 units) and 64 sampled units spread over layers 1-3, at every budget of the sweep."""
+    cfg = synth.config(4, budget_pct=budget_pct)
+    n, _ = _full_size_check(csp, oracle, cfg, 1, 0)
+    assert n == 32 * 32
+    rng = np.random.RandomState(budget_pct)
+    for layer in (1, 2, 3):
+        q, k, v = synth.make_layer(cfg, layer, "cuda")
+        mod1 = cfg.modality()
+        run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod1, cfg.seq_lens, cfg.budgets,
+                     total_budget=cfg.total_budget).prune()
+        assert run.status() == _expected_rows(cfg, csp)[1]
+        units = [(b, b, int(rng.randint(32))) for b in rng.randint(32, size=22)]
+        _check_units_against_oracle(csp, oracle, cfg, run, q, k, v, units, lambda fb, b, h: mod1[b],
+                                    cfg.budgets, cfg.total_budget)
+        assert_compaction_exact(run, mod1)
+        del run, q, k, v
+
+
+@pytest.mark.parametrize("config,units", [(2, [(0, 0), (0, 17), (0, 31)]), (3, [(0, 1), (3, 2), (2, 0)])])
+def test_one_layer_per_call_sampled_units(csp, oracle, config, units):
+    """The other launch configuration (one call per layer: few units, large clusters)."""
+    cfg = synth.config(config)
+    q, k, v = synth.make_layer(cfg, 1, "cuda")
+    mod1 = cfg.modality()
+    run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod1, cfg.seq_lens, cfg.budgets,
+                 total_budget=cfg.total_budget).prune()
+    want, st = _expected_rows(cfg, csp)
+    assert run.status() == st
+    _check_units_against_oracle(csp, oracle, cfg, run, q, k, v, [(b, b, h) for b, h in units],
+                                lambda fb, b, h: mod1[b], cfg.budgets, cfg.total_budget)
+    assert_compaction_exact(run, mod1)
+    assert (run.n_out.cpu().numpy() == want[:, None]).all()
 
 
 def test_host_buffer_entry_point(csp, oracle):

@@ -374,6 +374,80 @@ def test_and_or_on_mixed_window_are_intersection_and_union(oracle):
         assert sets[0][h] == top_s | top_c and sets[1][h] == top_s & top_c
 
 
+def _stable_topk(score, ids, k):
+    """Eq. 2 written with numpy: the first k of `ids` in a stable descending sort of their scores."""
+    k = max(0, min(int(k), len(ids)))
+    return set(ids[np.argsort(-score[ids].astype(np.float64), kind="stable")][:k].tolist())
+
+
+@pytest.mark.parametrize("seed,quantise", [(50, None), (51, None), (52, 8)])
+def test_segmented_select_is_four_independent_topks_on_a_mixed_window(oracle, seed, quantise):
+    """Budgets per key modality: the intra vector s ranks the text keys and, separately, the visual keys; so
+    does the inter vector c.  M^s is the union of the two s problems, M^c of the two c problems; Eq. 3 joins
+    them (union by default, intersection as printed).  With a mixed-modality window both vectors are non-zero
+    on both kinds of key, so a problem ranked by the wrong vector or drawn from the wrong keys changes the set."""
+    p, q, k, v, mod, L = _rand_case(oracle, seed, B=2, Hq=4, Hkv=2, L=(61, 47), W=6, R=5)
+    for b in range(2):                                   # both labels among the window queries
+        mod[b, L[b] - 6:L[b]] = [0, 1, 1, 0, 1, 0]
+    s, c = oracle.score(p, q, k, mod, L)
+    s32, c32 = s.astype(np.float32), c.astype(np.float32)
+    if quantise:                                         # many equal scores: ties go to the lower position
+        s32 = (np.floor(s32 * quantise * 4) / (quantise * 4)).astype(np.float32)
+        c32 = (np.floor(c32 * quantise * 4) / (quantise * 4)).astype(np.float32)
+    for b in range(2):
+        N = L[b] - p.recent
+        text, vis = mod[b, :N] == 0, mod[b, :N] != 0
+        for h in range(p.n_kv_heads):                    # every vector is informative on every kind of key
+            assert (s32[b, h, :N][text] > 0).sum() > 8 and (s32[b, h, :N][vis] > 0).sum() > 8
+            assert (c32[b, h, :N][text] > 0).sum() > 8 and (c32[b, h, :N][vis] > 0).sum() > 8
+    bud = np.array([[7, 5, 4, 9], [3, 30, 6, 2]], np.int32)    # self/text, self/visual, cross/text, cross/visual
+    for comb in (oracle.COMBINE_OR, oracle.COMBINE_AND):
+        p.combine = comb
+        idx, n_out, flags, margins = oracle.select(p, s32, c32, mod, L, bud)
+        for b in range(2):
+            N = int(L[b]) - p.recent
+            text, vis = np.where(mod[b, :N] == 0)[0], np.where(mod[b, :N] != 0)[0]
+            clamped = any(bud[b, j] > len(ids) for j, ids in enumerate((text, vis, text, vis)))
+            for h in range(p.n_kv_heads):
+                st, sv = _stable_topk(s32[b, h], text, bud[b, 0]), _stable_topk(s32[b, h], vis, bud[b, 1])
+                ct, cv = _stable_topk(c32[b, h], text, bud[b, 2]), _stable_topk(c32[b, h], vis, bud[b, 3])
+                ms, mc = st | sv, ct | cv
+                want = sorted(ms & mc if comb == oracle.COMBINE_AND else ms | mc)
+                got = idx[b, h, :n_out[b, h]]
+                np.testing.assert_array_equal(got[:len(want)], want)
+                np.testing.assert_array_equal(got[len(want):], np.arange(N, L[b]))
+                assert bool(flags[b, h] & oracle.FLAG_K_CLAMPED) == clamped
+                # the reported boundary scores belong to the right problem
+                for j, (vec, ids) in enumerate(((s32, text), (s32, vis), (c32, text), (c32, vis))):
+                    kk = min(int(bud[b, j]), len(ids))
+                    ranked = np.sort(vec[b, h][ids].astype(np.float64))[::-1]
+                    if kk >= 1:
+                        assert margins[b, h, j, 0] == np.float32(ranked[kk - 1])
+                    if kk < len(ids):
+                        assert margins[b, h, j, 1] == np.float32(ranked[kk])
+
+
+def test_segmented_select_hand_worked_example(oracle):
+    gold = {}
+    with open(os.path.join(GOLDEN, "segmented_select_L10.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, *vals = line.split()
+                gold[name] = vals
+    mod = np.array([gold["labels"]], np.uint8)
+    s = np.zeros((1, 1, 10), np.float32)
+    c = np.zeros((1, 1, 10), np.float32)
+    s[0, 0, :8] = np.array(gold["s"], np.float32)
+    c[0, 0, :8] = np.array(gold["c"], np.float32)
+    bud = np.array([gold["budgets"]], np.int32)
+    for comb, name in ((oracle.COMBINE_OR, "keep_or"), (oracle.COMBINE_AND, "keep_and")):
+        p = oracle.Params(1, 1, 1, 4, 2, 2, 10, 10, combine=comb)
+        idx, n_out, flags, _ = oracle.select(p, s, c, mod, np.array([10], np.int32), bud)
+        want = np.array(gold[name], np.int32)
+        assert n_out[0, 0] == len(want) and flags[0, 0] == 0
+        np.testing.assert_array_equal(idx[0, 0, :len(want)], want)
+
+
 def test_capacity_overflow_and_clamp_flags(oracle):
     p, q, k, v, mod, L = _rand_case(oracle, 35, B=1, L=(30,), W=3, R=3)
     p.out_capacity = 10
