@@ -22,7 +22,12 @@
  *    buffer.  The library never allocates or frees device memory and, except for
  *    csp_device_status and csp_prune_layer_host, never synchronises: work is enqueued on the
  *    given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
- *  - Inputs are read-only.  Outputs must not overlap inputs or each other.
+ *  - Inputs are read-only.  Outputs must not overlap inputs or each other, with one exception:
+ *    compaction in place (k_out the very tensor k and v_out the very tensor v), see csp_compact.
+ *  - Host threads: entry points may be called from several host threads at once, on the same or on
+ *    different devices, as long as calls that can overlap on the GPU use different workspaces and
+ *    outputs.  What the library remembers between calls (per-device launch settings) is synchronised
+ *    internally.  csp_prune_layer_static is the exception: all its calls share one scratch array.
  *  - Tensors are described by a base pointer and ELEMENT strides; the innermost (head_dim)
  *    axis is contiguous.  Base pointers and row starts must be 16-byte aligned (every stride
  *    times the element size a multiple of 16 bytes).
@@ -149,7 +154,9 @@ csp_status csp_select(const csp_params* p, const float* score_self, const float*
 /*
  * Eq. 4: k_out[b,h,j,:] = k[b,h,keep_idx[b,h,j],:] for j < n_out[b,h]; same for v and the labels.
  *   k_out, v_out [B, H_kv, out_capacity, d] (strided); mod_out [B, H_kv, out_capacity] dense, may
- *   be NULL.  Rows j >= n_out are left as they were; units with n_out <= 0 are skipped.
+ *   be NULL.  Rows j >= n_out are left as they were; units with n_out <= 0 are skipped; an n_out above
+ *   out_capacity copies the first out_capacity rows only (csp_prune_layer also raises CSP_DEV_CAPACITY;
+ *   csp_compact has no status word).  Entries of keep_idx outside [0, max_len) copy nothing.
  * In place (the iteration of Algorithm 1 without a second cache buffer): k_out may be the very tensor k
  * and v_out the very tensor v (same pointer and strides, both or neither; CSP_ERR_UNSUPPORTED otherwise).
  * keep_idx is ascending with keep_idx[j] >= j, as csp_select writes it, so rows only move down; mod_out
@@ -226,8 +233,11 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
  *   - Shapes whose csp_workspace_bytes exceeds the limit are refused with CSP_ERR_WORKSPACE and
  *     nothing is enqueued (8 MiB covers e.g. 32 KV heads x 4096 positions; use csp_prune_layer with
  *     your own workspace beyond that).
+ *   - Arguments are checked as in csp_prune_layer before anything else happens; a call that returns an
+ *     error has enqueued nothing.
  *   - The first call on a device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *     outside any stream capture.  The address is kept for the life of the process (a cudaDeviceReset
+ *     in between is not supported).
  *   - All calls share the one array, which still holds the previous call's contents; the status
  *     area is cleared on the stream at the start of every call.  Two calls whose GPU work can
  *     overlap (different streams, several host threads) race on it: serialise them.

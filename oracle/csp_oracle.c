@@ -118,7 +118,7 @@ int orc_score(const orc_params* p, const void* q, const void* k,
     int bad = 0;
 
     if (p->head_reduce == ORC_HEADS_PER_KV) {
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
         for (int u = 0; u < units; ++u) {
             const int b = u / p->n_kv_heads, h = u % p->n_kv_heads;
             const int64_t L = seq_lens[b];
@@ -137,7 +137,7 @@ int orc_score(const orc_params* p, const void* q, const void* k,
         }
     } else {
         /* the paper's sentence: one attention matrix averaged over every head */
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
         for (int b = 0; b < p->batch; ++b) {
             const int64_t L = seq_lens[b];
             for (int h = 0; h < p->n_kv_heads; ++h) {
@@ -205,7 +205,7 @@ int orc_select(const orc_params* p, const float* score_self, const float* score_
         return -1;
     const int units = p->batch * p->n_kv_heads;
     int bad = 0;
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
     for (int u = 0; u < units; ++u) {
         const int b = u / p->n_kv_heads, h = u % p->n_kv_heads;
         const int64_t L = seq_lens[b];
@@ -297,7 +297,7 @@ int orc_compact(const orc_params* p, const void* k, const void* v,
     const int units = p->batch * p->n_kv_heads;
     const int64_t row = (int64_t)p->head_dim * elem_size(p->dtype);
     int bad = 0;
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
     for (int u = 0; u < units; ++u) {
         const int b = u / p->n_kv_heads, h = u % p->n_kv_heads;
         const char* ku = (const char*)k + (int64_t)u * p->max_len * row;
@@ -345,7 +345,7 @@ int orc_decode_attn(const orc_params* p, const void* q, const void* k, const voi
     const int G = p->n_q_heads / p->n_kv_heads;
     const double scale = p->scale > 0.0 ? p->scale : 1.0 / sqrt((double)d);
     int bad = 0;
-#pragma omp parallel for collapse(2) schedule(dynamic)
+#pragma omp parallel for collapse(2) schedule(dynamic) reduction(|:bad)
     for (int b = 0; b < p->batch; ++b) {
         for (int hq = 0; hq < p->n_q_heads; ++hq) {
             const int hkv = hq / G;

@@ -35,7 +35,8 @@ csp_status check_params(const csp_params* p) {
     if (row_bytes != 128 && row_bytes != 256 && row_bytes != 512) return CSP_ERR_UNSUPPORTED;
     if (p->n_q_heads / p->n_kv_heads > 8) return CSP_ERR_UNSUPPORTED;
     if (p->window > 32) return CSP_ERR_UNSUPPORTED;
-    if (p->n_kv_heads > 65535 || p->batch > 65535) return CSP_ERR_UNSUPPORTED;
+    // one (sequence, KV head) unit per grid row or plane: the product must fit a grid dimension
+    if (int64_t(p->batch) * int64_t(p->n_kv_heads) > 65535) return CSP_ERR_UNSUPPORTED;
     return CSP_OK;
 }
 
@@ -99,7 +100,8 @@ csp_status do_select(const csp_params& p, const float* score_self, const float* 
 
 csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor& v, const uint8_t* modality,
                       int64_t msb, int64_t msh, const int32_t* keep_idx, const int32_t* n_out,
-                      const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, cudaStream_t stream) {
+                      const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, int32_t* status,
+                      cudaStream_t stream) {
     const int64_t es = elem_size(p);
     CompactArgs a;
     a.k = k.ptr; a.v = v.ptr; a.k_out = k_out.ptr; a.v_out = v_out.ptr;
@@ -111,10 +113,43 @@ csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor
     a.keep_idx = keep_idx; a.n_out = n_out;
     a.n_kv_heads = p.n_kv_heads; a.max_len = p.max_len; a.out_capacity = p.out_capacity;
     a.chunks_per_row = int(p.head_dim * es / 16);
+    a.status = status;
     return launch_compact(p, a, stream);
 }
 
 }  // namespace
+
+int sm_count() {
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return kFallbackSms; }
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached) {
+        const int v = cache[dev].load(std::memory_order_relaxed);
+        if (v > 0) return v;
+    }
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return kFallbackSms;
+    }
+    if (cached) cache[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
+csp_status check_prune_layer_args(const csp_params* p, const csp_tensor& q_win, const csp_tensor& k, const csp_tensor& v,
+                                  const uint8_t* modality, const int32_t* seq_lens, const int32_t* budgets,
+                                  const csp_tensor& k_out, const csp_tensor& v_out, const int32_t* n_out) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!modality || !seq_lens || !budgets || !n_out || !q_win.ptr || !k.ptr || !v.ptr || !k_out.ptr || !v_out.ptr)
+        return CSP_ERR_INVALID_ARG;
+    if (!tensor_ok(*p, q_win) || !tensor_ok(*p, k) || !tensor_ok(*p, v) || !tensor_ok(*p, k_out) ||
+        !tensor_ok(*p, v_out))
+        return CSP_ERR_UNSUPPORTED;
+    return check_arch();
+}
+
 }  // namespace csp
 
 using namespace csp;
@@ -175,7 +210,7 @@ csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v, const ui
         return CSP_ERR_UNSUPPORTED;
     if ((st = check_arch()) != CSP_OK) return st;
     return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, keep_idx, n_out, k_out, v_out, mod_out,
-                      static_cast<cudaStream_t>(cuda_stream));
+                      nullptr, static_cast<cudaStream_t>(cuda_stream));
 }
 
 csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
@@ -185,15 +220,9 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes,
                            void* cuda_stream) {
-    csp_status st = check_params(p);
+    csp_status st = check_prune_layer_args(p, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, n_out);
     if (st != CSP_OK) return st;
-    if (!modality || !seq_lens || !budgets || !n_out || !q_win.ptr || !k.ptr || !v.ptr || !k_out.ptr || !v_out.ptr)
-        return CSP_ERR_INVALID_ARG;
-    if (!tensor_ok(*p, q_win) || !tensor_ok(*p, k) || !tensor_ok(*p, v) || !tensor_ok(*p, k_out) ||
-        !tensor_ok(*p, v_out))
-        return CSP_ERR_UNSUPPORTED;
     if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
-    if ((st = check_arch()) != CSP_OK) return st;
     const WorkspaceLayout wl = workspace_layout(*p);
     char* ws = static_cast<char*>(workspace);
     float* ss = score_self_or_null ? score_self_or_null : reinterpret_cast<float*>(ws + wl.score_self);
@@ -206,7 +235,8 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
     if ((st = do_select(*p, ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
                         idx, n_out, workspace, stream)) != CSP_OK)
         return st;
-    return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out, stream);
+    return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
+                      static_cast<int32_t*>(workspace), stream);
 }
 
 // staging layout for the host-buffer variant: every block rounded up to 256 bytes

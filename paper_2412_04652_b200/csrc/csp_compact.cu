@@ -10,7 +10,7 @@ namespace {
 constexpr int kCompactThreads = 256;
 // rows per CTA: 128 when that still gives every SM several CTAs (fewer, longer CTAs stream better), else 64
 inline int rows_per_cta(int units, int capacity) {
-    return (long long)units * ((capacity + 127) / 128) >= 8 * 148 ? 128 : 64;
+    return (long long)units * ((capacity + 127) / 128) >= 8LL * sm_count() ? 128 : 64;
 }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -24,8 +24,12 @@ template <int rows_cta, int CPR>   // rows per CTA; 16-byte chunks per row (8, 1
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactArgs a) {
     const int blocks_per_unit = (a.out_capacity + rows_cta - 1) / rows_cta;
     const int u = blockIdx.x / blocks_per_unit, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
-    const int n = a.n_out[u];
+    int n = a.n_out[u];
     const int row0 = (blockIdx.x % blocks_per_unit) * rows_cta;
+    if (n > a.out_capacity) {          // a row count the outputs cannot hold: copy what fits, say so where possible
+        if (a.status && row0 == 0 && threadIdx.x == 0) atomicOr(a.status, CSP_DEV_CAPACITY);
+        n = a.out_capacity;
+    }
     if (n <= 0 || row0 >= n) return;
     constexpr int cpr = CPR;
     constexpr int rows_per_iter = kCompactThreads / cpr;
@@ -82,6 +86,7 @@ __global__ void __launch_bounds__(kInplaceThreads) compact_inplace_kernel(const 
     const int u = blockIdx.x, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
     const int n = a.n_out[u];
     if (n <= 0) return;
+    if (n > a.out_capacity && a.status && threadIdx.x == 0) atomicOr(a.status, CSP_DEV_CAPACITY);
     const int cpr = a.chunks_per_row;                    // 8, 16 or 32
     const int rows_per_iter = kInplaceThreads / cpr;
     const int r_in = threadIdx.x / cpr, c = threadIdx.x % cpr;

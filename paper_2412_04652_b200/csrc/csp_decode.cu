@@ -335,8 +335,8 @@ int decode_splits(const csp_params& p) {
     const int units = p.batch * p.n_kv_heads;
     const int tiles = (p.out_capacity + kDecTile - 1) / kDecTile;
     if (units <= 0 || tiles <= 0) return 1;
-    // at least about four work items per resident CTA (148), but no item shorter than four tiles
-    int splits = (4 * 148 + units - 1) / units;
+    // at least about four work items per resident CTA (one per SM), but no item shorter than four tiles
+    int splits = (4 * sm_count() + units - 1) / units;
     if (splits > (tiles + 3) / 4) splits = (tiles + 3) / 4;
     return splits < 1 ? 1 : splits;
 }
@@ -375,18 +375,10 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
         const size_t smem = 1024 + size_t(kDecStages) * 2 * NH * kDecBlock + size_t(kDecWarps) * 8 * (p.head_dim + 2) * 4 +
                             16 * kDecStages + 64;
         auto kern = NH == 1 ? decode_attn_kernel<1> : decode_attn_kernel<2>;
-        static bool configured[2][64] = {};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
-        if (dev < 0 || dev >= 64 || !configured[NH - 1][dev]) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
-                cudaGetLastError();
-                return CSP_ERR_CUDA;
-            }
-            if (dev >= 0 && dev < 64) configured[NH - 1][dev] = true;
-        }
-        const int n_items = units * a.splits;
-        kern<<<n_items < 148 ? n_items : 148, kDecThreads, smem, s>>>(tk, tv, a, n_items);
+        static std::atomic<bool> configured[2][kMaxDevices];
+        if (!raise_smem_limit(kern, int(smem), configured[NH - 1])) return CSP_ERR_CUDA;
+        const int n_items = units * a.splits, sms = sm_count();
+        kern<<<n_items < sms ? n_items : sms, kDecThreads, smem, s>>>(tk, tv, a, n_items);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
     }
     decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);

@@ -5,9 +5,38 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "csp.h"
 
 namespace csp {
+
+// ---- per-device host-side caches ----------------------------------------------------------
+// Entry points may be called from several host threads at once.  What the launchers remember between
+// calls (SM count, "this kernel's shared-memory limit has been raised on this device", how many clusters
+// of a size fit on the device) sits in arrays of atomics indexed by the device ordinal: the cached values
+// are the same whoever computes them, so a lost race only repeats an idempotent query.
+constexpr int kMaxDevices = 64;
+constexpr int kFallbackSms = 148;                    // B200; used only when the attribute query fails
+
+// Streaming multiprocessors of the current device.
+int sm_count();
+
+// Raises a kernel's dynamic shared-memory limit the first time it is launched on the current device.
+// `done` is that kernel's own array of per-device flags.
+template <typename Kern>
+inline bool raise_smem_limit(Kern kern, int bytes, std::atomic<bool> (&done)[kMaxDevices]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached && done[dev].load(std::memory_order_acquire)) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    if (cached) done[dev].store(true, std::memory_order_release);
+    return true;
+}
 
 // ---- workspace layout -------------------------------------------------------------------
 // [0, 256)            status area (word 0 = OR of CSP_DEV_* bits)
@@ -71,16 +100,18 @@ struct CompactArgs {
     const uint8_t* modality; int64_t mod_sb, mod_sh; uint8_t* mod_out;
     const int32_t* keep_idx; const int32_t* n_out;
     int32_t n_kv_heads, max_len, out_capacity, chunks_per_row;
+    int32_t* status;                                 // device status word, or null (csp_compact has none)
 };
 
-// Cluster size (CTAs per unit, a power of two <= 8).  At least enough CTAs to occupy the 148 SMs when
+// Cluster size (CTAs per unit, a power of two <= 8).  At least enough CTAs to occupy the `sms` SMs when
 // there are few units; more when that lets every CTA keep all of its tiles' logits on chip
 // (`tiles_kept` tiles per CTA; 0 if the kernel keeps none), which removes the second pass over K.
-// Clusters of 4 and 8 fit on 132 and 120 of the 148 SMs only, so when even 8 CTAs cannot keep the
-// logits the cluster stays small: pairs, which also halves the longest CTA of a ragged batch.
-inline int pick_cluster(int units, int max_tiles, int tiles_kept) {
+// Clusters of 4 and 8 fit on fewer SMs than single CTAs or pairs do (132 and 120 of a B200's 148), so when
+// even 8 CTAs cannot keep the logits the cluster stays small: pairs, which also halves the longest CTA of
+// a ragged batch.
+inline int pick_cluster(int units, int max_tiles, int tiles_kept, int sms) {
     int c = 1;
-    while (c < 8 && units * (c * 2) <= 148 && c * 2 <= max_tiles) c *= 2;
+    while (c < 8 && units * (c * 2) <= sms && c * 2 <= max_tiles) c *= 2;
     if (tiles_kept > 0 && (max_tiles + 7) / 8 <= tiles_kept) {
         while (c < 8 && (max_tiles + c - 1) / c > tiles_kept) c *= 2;
     } else if (tiles_kept > 0 && c < 2 && max_tiles >= 32) {
@@ -88,6 +119,11 @@ inline int pick_cluster(int units, int max_tiles, int tiles_kept) {
     }
     return c;
 }
+
+// Host-visible checks of csp_prune_layer's arguments (everything but the workspace); enqueues nothing.
+csp_status check_prune_layer_args(const csp_params* p, const csp_tensor& q_win, const csp_tensor& k, const csp_tensor& v,
+                                  const uint8_t* modality, const int32_t* seq_lens, const int32_t* budgets,
+                                  const csp_tensor& k_out, const csp_tensor& v_out, const int32_t* n_out);
 
 // ---- host-side launchers (defined next to their kernels) ----------------------------------
 csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s);

@@ -458,16 +458,10 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     if (stages < 2) return CSP_ERR_UNSUPPORTED;
     const size_t smem = smem_plan(NH, G, stages).total + 1024;
     auto kern = score_kernel<T, NH, G>;
-    static bool configured[64] = {};   // per instantiation and device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-            return CSP_ERR_CUDA;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];   // per instantiation and device
+    if (!raise_smem_limit(kern, 227 * 1024, configured)) return CSP_ERR_CUDA;
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
-    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles, 0);
+    const int c = pick_cluster(p.batch * p.n_kv_heads, max_tiles, 0, sm_count());
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
     cfg.blockDim = dim3(kThreads);
@@ -570,11 +564,12 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_te
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return CSP_ERR_UNSUPPORTED;
     if (p.dtype == CSP_F32) return launch_t<float>(p, a, tmap, s);
-    // several sequences and more CTAs than fit on the GPU at once (up to 8 per unit, 120 SMs hold clusters
-    // of 8): take the sequences longest first
+    // several sequences and more CTAs than fit on the GPU at once (up to 8 per unit; clusters of 8 occupy
+    // about 13/16 of the SMs, 120 of a B200's 148): take the sequences longest first
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
     const long long units = (long long)p.batch * p.n_kv_heads;
-    if (p.batch >= 2 && p.batch <= 4096 && (units > 148 || units * (max_tiles < 8 ? max_tiles : 8) > 120)) {
+    const int sms = sm_count();
+    if (p.batch >= 2 && p.batch <= 4096 && (units > sms || units * (max_tiles < 8 ? max_tiles : 8) > sms * 13 / 16)) {
         length_order_kernel<<<(p.batch + 255) / 256, 256, 0, s>>>(a.seq_lens, p.batch, p.max_len, a.order_buf);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
         a.order = a.order_buf;

@@ -479,11 +479,11 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
     if (stages < 2) return CSP_OK;
     const size_t smem = ps_smem_plan(NH, stages).total + 1024;
     auto kern = score_tc_persist_kernel<NH>;
-    static bool configured[64] = {};
-    static int resident[64] = {};      // clusters of this size that fit on the device at once
+    static std::atomic<bool> configured[kMaxDevices];
+    static std::atomic<int> resident[kMaxDevices][4];   // clusters of 1, 2, 4, 8 CTAs that fit on the device at once
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
-    if (dev < 0 || dev >= 64) return CSP_OK;
+    if (dev < 0 || dev >= kMaxDevices) return CSP_OK;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kPsThreads);
     cfg.dynamicSmemBytes = smem;
@@ -492,20 +492,17 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-            return CSP_ERR_CUDA;
-        configured[dev] = true;
-    }
-    static int resident_c[64] = {};
-    if (resident[dev] == 0 || resident_c[dev] != c) {
-        cfg.gridDim = dim3((148 / c) * c, 1, 1);
+    if (!raise_smem_limit(kern, 227 * 1024, configured)) return CSP_ERR_CUDA;
+    const int slot = c == 1 ? 0 : (c == 2 ? 1 : (c == 4 ? 2 : 3));
+    int n_clusters = resident[dev][slot].load(std::memory_order_relaxed);
+    if (n_clusters == 0) {
+        const int sms = sm_count();
+        cfg.gridDim = dim3((sms / c) * c, 1, 1);
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = 148 / c / 2; }
-        resident[dev] = n > 0 ? n : 1;
-        resident_c[dev] = c;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = sms / c / 2; }
+        n_clusters = n > 0 ? n : 1;
+        resident[dev][slot].store(n_clusters, std::memory_order_relaxed);
     }
-    const int n_clusters = resident[dev];
     if (units < 2 * n_clusters) return CSP_OK;           // too few units for a resident loop to pay off
     cfg.gridDim = dim3(n_clusters * c, 1, 1);
     if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages, units, n_clusters) != cudaSuccess) {

@@ -390,8 +390,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
             auto chunk_plain = [&](const uint32_t (&cur)[16], const float* cvp) {
                 const float4* cv = reinterpret_cast<const float4*>(cvp);
-#pragma unroll
                 const float2 sc2 = make_float2(scale2, scale2);
+#pragma unroll
                 for (int j4 = 0; j4 < 4; ++j4) {
                     const float4 cc = cv[j4];
                     p01 = __fadd2_rn(p01, ex2f2(__ffma2_rn(make_float2(__uint_as_float(cur[j4 * 4 + 0]), __uint_as_float(cur[j4 * 4 + 1])),
@@ -475,9 +475,10 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     const int units = p.batch * p.n_kv_heads;
     // Two CTAs per SM when (MHA) every CTA can still keep all its tiles in its half of tensor memory.
     bool shared_sm = false;
-    int c = pick_cluster(units, max_tiles, TmemPlan<G>::kBufs);
+    const int sms = sm_count();
+    int c = pick_cluster(units, max_tiles, TmemPlan<G>::kBufs, sms);
     if (G == 1 && NH <= 2) {
-        const int c2 = pick_cluster(units, max_tiles, TmemPlan<G>::kBufsShared);
+        const int c2 = pick_cluster(units, max_tiles, TmemPlan<G>::kBufsShared, sms);
         if ((max_tiles + c2 - 1) / c2 <= TmemPlan<G>::kBufsShared) { shared_sm = true; c = c2; }
     }
     const int fixed = int(tc_smem_plan(NH, G, 0).total) + 1024;
@@ -486,14 +487,8 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     if (stages < 2) return CSP_ERR_UNSUPPORTED;
     const size_t smem = tc_smem_plan(NH, G, stages).total + 1024;
     auto kern = score_tc_kernel<NH, G>;
-    static bool configured[64] = {};   // per instantiation and device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-            return CSP_ERR_CUDA;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];   // per instantiation and device
+    if (!raise_smem_limit(kern, 227 * 1024, configured)) return CSP_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c, p.n_kv_heads, p.batch);
     cfg.blockDim = dim3(EpiPlan<G>::kThreads);

@@ -234,15 +234,8 @@ csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t 
     if (n_cached > limit) n_cached = limit;
     n_cached = (n_cached + 3) & ~size_t(3);
     const size_t smem = fixed + n_cached * kBytesPerCached;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
-            cudaSuccess)
-            return CSP_ERR_CUDA;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!raise_smem_limit(select_kernel, 227 * 1024 - 2048, configured)) return CSP_ERR_CUDA;
     select_kernel<<<units, kSelThreads, smem, s>>>(a, int(n_cached));
     return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
 }

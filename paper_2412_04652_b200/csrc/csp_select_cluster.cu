@@ -365,8 +365,9 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     const int per_cta = p.max_len <= 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;
-    if (per_cta == 8192) return units * cs >= 2 * 148 ? launch_e<512, 16>(p, a, cs, s) : launch_e<1024, 8>(p, a, cs, s);
-    if (units * cs >= 2 * 148) return launch_e<512, 8>(p, a, cs, s);
+    const int sms = sm_count();
+    if (per_cta == 8192) return units * cs >= 2 * sms ? launch_e<512, 16>(p, a, cs, s) : launch_e<1024, 8>(p, a, cs, s);
+    if (units * cs >= 2 * sms) return launch_e<512, 8>(p, a, cs, s);
     return launch_e<1024, 4>(p, a, cs, s);
 }
 

@@ -20,7 +20,9 @@ constexpr int kMaxDevices = 64;
 void* g_device_address[kMaxDevices] = {};
 std::mutex g_setup_mutex;
 
-// Looks up, once per device and with that device current, where the array lives on it.
+// Looks up, once per device and with that device current, where the array lives on it.  The address is
+// remembered for the life of the process; a cudaDeviceReset, which unloads the library's device image,
+// is not supported between calls.
 csp_status static_workspace(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return CSP_ERR_CUDA; }
@@ -46,11 +48,15 @@ csp_status csp_prune_layer_static(const csp_params* p, csp_tensor q_win, csp_ten
                                   const int32_t* total_budget_or_null, const float* lse_or_null,
                                   csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
                                   int32_t* dev_status_out_or_null, void* cuda_stream) {
+    // Everything the host can reject is rejected before the address lookup and before anything is enqueued:
+    // parameters, null pointers, alignment, the architecture, then the size of the scratch.
+    csp_status st = csp::check_prune_layer_args(p, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, n_out);
+    if (st != CSP_OK) return st;
     const size_t need = csp_workspace_bytes(p);
-    if (need == 0) return p ? CSP_ERR_UNSUPPORTED : CSP_ERR_INVALID_ARG;
+    if (need == 0) return CSP_ERR_UNSUPPORTED;
     if (need > kStaticWorkspaceBytes) return CSP_ERR_WORKSPACE;   // shapes beyond the built-in scratch
     void* ws = nullptr;
-    csp_status st = static_workspace(&ws);
+    st = static_workspace(&ws);
     if (st != CSP_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps whatever the previous call left: the status area must start at zero

@@ -324,6 +324,41 @@ def test_compact_is_bit_exact_with_strides(csp, oracle):
     np.testing.assert_array_equal(run.mod_out.cpu().numpy(), mo)
 
 
+def test_compact_row_count_above_capacity_is_clamped_not_faulted(csp, oracle):
+    """n_out is caller-supplied device data for csp_compact: a count above out_capacity copies the first
+    out_capacity rows and touches nothing behind the unit (canary rows, the next unit's rows, labels)."""
+    cfg = _case((400, 250), 4, 2, 128, 32, 32, seed=24)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    cap = 70                                              # not a multiple of the 64 / 128 rows a CTA covers
+    p = gpu_params(csp, cfg, cap=cap)
+    run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets)
+    rng = np.random.RandomState(2)
+    idx = np.zeros((2, 2, cap), np.int32)
+    for b in range(2):
+        for h in range(2):
+            idx[b, h] = np.sort(rng.choice(int(cfg.seq_lens[b]), cap, replace=False))
+    n_out = np.array([[cap + 5, cap], [cap + 1000, 3]], np.int32)
+    run.idx, run.n_out = torch.from_numpy(idx).cuda(), torch.from_numpy(n_out).cuda()
+    canary = 0x7F7F
+    big_k = torch.full((2, 2, cap + 8, 128), 0, dtype=torch.int16, device="cuda") + canary
+    big_v = big_k.clone()
+    big_m = torch.full((2 * 2 * cap + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+    run.k_out, run.v_out = big_k.view(torch.bfloat16)[:, :, :cap], big_v.view(torch.bfloat16)[:, :, :cap]
+    run.mod_out = big_m[:2 * 2 * cap].view(2, 2, cap)
+    run.compact()
+    torch.cuda.synchronize()
+    assert (big_k[:, :, cap:] == canary).all() and (big_v[:, :, cap:] == canary).all()
+    assert (big_m[2 * 2 * cap:] == 0xEE).all()
+    kb, vb = bits(k), bits(v)
+    for b in range(2):
+        for h in range(2):
+            n = min(int(n_out[b, h]), cap)
+            np.testing.assert_array_equal(bits(run.k_out[b, h, :n]), kb[b, h][idx[b, h, :n]])
+            np.testing.assert_array_equal(bits(run.v_out[b, h, :n]), vb[b, h][idx[b, h, :n]])
+            np.testing.assert_array_equal(run.mod_out[b, h, :n].cpu().numpy(), cfg.modality()[b][idx[b, h, :n]])
+    assert (big_k[1, 1, 3:] == canary).all()              # the short unit wrote its three rows only
+
+
 @pytest.mark.parametrize("d,dtype", [(128, torch.bfloat16), (64, torch.bfloat16), (64, torch.float32)])
 def test_compact_in_place_matches_out_of_place(csp, oracle, d, dtype):
     """k_out is k and v_out is v: rows move down inside the cache.  Dense keeps (many rows shifting by a few
