@@ -213,6 +213,8 @@ size_t csp_host_staging_bytes(const csp_params* p);
  * back and waits for the stream.  All *_host tensors are dense: q [B,H_q,W,d],
  * k, v [B,H_kv,max_len,d], modality [B,max_len] (mod_per_head == 0) or [B,H_kv,max_len],
  * outputs [B,H_kv,out_capacity,(d)].  dev_status_host (may be NULL) receives the status word.
+ * Only the kept rows of V are needed (Eq. 4): when v_host is page-locked memory the device can address, they are
+ * read from it directly by the compaction kernel and V is never copied as a whole; otherwise V is staged in full.
  */
 csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const void* k_host,
                                 const void* v_host, const uint8_t* modality_host, int mod_per_head,

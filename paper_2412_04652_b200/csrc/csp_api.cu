@@ -299,9 +299,23 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
     auto d2h = [&](void* dst, size_t off, size_t bytes) {
         if (bytes) ok = ok && cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     };
+    // V is only ever read at the kept rows.  When the caller's buffer is page-locked memory that this device can
+    // address (cudaHostAlloc / cudaHostRegister), the compaction kernel fetches those rows from it directly and
+    // the copy of the whole tensor is skipped; pageable or misaligned memory is staged in full as before.
+    const void* v_mapped = nullptr;
+    {
+        cudaPointerAttributes at;
+        int can_map = 0, dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&can_map, cudaDevAttrCanMapHostMemory, dev) == cudaSuccess && can_map &&
+            cudaPointerGetAttributes(&at, v_host) == cudaSuccess && at.type == cudaMemoryTypeHost &&
+            at.devicePointer && (uintptr_t(at.devicePointer) % 16 == 0))
+            v_mapped = at.devicePointer;
+        cudaGetLastError();
+    }
     h2d(sl.q, q_host, q_bytes);
     h2d(sl.k, k_host, kv_bytes);
-    h2d(sl.v, v_host, kv_bytes);
+    if (!v_mapped) h2d(sl.v, v_host, kv_bytes);
     h2d(sl.mod, modality_host, mod_bytes);
     h2d(sl.seq, seq_lens_host, size_t(p->batch) * 4);
     h2d(sl.bud, budgets_host, size_t(p->batch) * 4 * nbud);
@@ -312,7 +326,7 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
     const int64_t d_ = p->head_dim;
     csp_tensor q = {d + sl.q, int64_t(p->n_q_heads) * p->window * d_, int64_t(p->window) * d_, d_};
     csp_tensor k = {d + sl.k, int64_t(p->n_kv_heads) * p->max_len * d_, int64_t(p->max_len) * d_, d_};
-    csp_tensor v = {d + sl.v, k.stride_b, k.stride_h, d_};
+    csp_tensor v = {v_mapped ? const_cast<void*>(v_mapped) : static_cast<void*>(d + sl.v), k.stride_b, k.stride_h, d_};
     csp_tensor ko = {d + sl.k_out, int64_t(p->n_kv_heads) * p->out_capacity * d_, int64_t(p->out_capacity) * d_, d_};
     csp_tensor vo = {d + sl.v_out, ko.stride_b, ko.stride_h, d_};
     const int64_t msb = mod_per_head ? int64_t(p->n_kv_heads) * p->max_len : p->max_len;

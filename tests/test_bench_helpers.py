@@ -1,0 +1,37 @@
+"""Host-side logic of bench.py that needs no GPU: where the ncu DRAM-traffic figure of the bench line comes
+from, and the algorithmic byte counts."""
+import os
+import re
+
+import numpy as np
+
+import bench
+import csp_synth as synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_traffic_comes_from_the_committed_summary_of_that_kernel_workload_and_launch():
+    found = 0
+    for name in sorted(os.listdir(os.path.join(ROOT, "profiles"))):
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+        m = re.search(r"^dram_bytes_per_launch:\s*([0-9.eE+]+)", text, re.M)
+        mm = re.match(r"(score|select|compact|decode_attn)[a-z_]*_(configs\d(?:_\d+pct)?)_(all_layers_one_call|one_layer_per_call)\.md$", name)
+        if not (m and mm):
+            continue
+        got, src = bench.ncu_traffic(mm.group(1), mm.group(2), mm.group(3))
+        assert got == float(m.group(1)) and src == os.path.join("profiles", name)
+        found += 1
+    assert found >= 1
+    assert bench.ncu_traffic("score", "configs9", "all_layers_one_call") == (None, None)
+    assert bench.ncu_traffic("score", "configs1", "some_other_launch") == (None, None)
+
+
+def test_algorithmic_bytes_of_the_headline_workload():
+    cfg = synth.config(1)
+    ab = bench.algorithmic_bytes(cfg, cfg.seq_lens, 32 * 1027)
+    k_bytes = 4096 * 32 * 128 * 2
+    assert ab["score"] == k_bytes + 32 * 32 * 128 * 2 + 4096 + 2 * 4 * 4064 * 32
+    assert ab["compact"] == 32 * 1027 * (4 + 2 * 2 * 256 + 2)
+    assert ab["total"] == ab["score"] + ab["select"] + ab["compact"]
+    assert abs(ab["total"] - 70.0e6) < 0.5e6

@@ -39,7 +39,7 @@ def test_two_gloo_ranks_agree_on_the_slowest_time_and_add_their_units():
 def test_reference_arm_prints_on_rank_zero_only():
     env = dict(os.environ, OMP_NUM_THREADS="2")
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0",
-           "--steps", "1", "--warmup", "0", "--ref-units", "1"]
+           "--steps", "1", "--warmup", "0"]
     r0 = subprocess.run(cmd, env=dict(env, RANK="0", WORLD_SIZE="2"), capture_output=True, text=True, timeout=300)
     r1 = subprocess.run(cmd, env=dict(env, RANK="1", WORLD_SIZE="2"), capture_output=True, text=True, timeout=300)
     assert r0.returncode == 0 and r1.returncode == 0

@@ -650,16 +650,29 @@ def test_host_buffer_entry_point(csp, oracle):
     mod_out = pin(torch.zeros(2, 2, cap, dtype=torch.uint8))
     n_out = pin(torch.zeros(2, 2, dtype=torch.int32))
     staging = torch.empty(csp.host_staging_bytes(p), dtype=torch.uint8, device="cuda")
-    status = csp.prune_layer_host(p, pin(q), pin(k), pin(v), mod, lens, bud, k_out, v_out, mod_out, n_out, staging)
-    assert status == 0
     run = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).prune()
-    assert torch.equal(n_out, run.n_out.cpu())
-    for b in range(2):
-        for h in range(2):
-            n = int(n_out[b, h])
-            assert torch.equal(k_out[b, h, :n], run.k_out[b, h, :n].cpu())
-            assert torch.equal(v_out[b, h, :n], run.v_out[b, h, :n].cpu())
-            assert torch.equal(mod_out[b, h, :n], run.mod_out[b, h, :n].cpu())
+    ref = oracle.prune_layer(orc_params(oracle, cfg), q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets)
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, cfg.modality(), cfg.seq_lens, cfg.recent)
+    # page-locked V: its kept rows are read by the compaction kernel straight from host memory;
+    # pageable V (a plain tensor): staged in full.  Same bytes either way.
+    for v_host in (pin(v), v.contiguous()):
+        for t in (k_out, v_out, mod_out, n_out):
+            t.zero_()
+        status = csp.prune_layer_host(p, pin(q), pin(k), v_host, mod, lens, bud, k_out, v_out, mod_out, n_out, staging)
+        assert status == 0
+        assert torch.equal(n_out, run.n_out.cpu())
+        np.testing.assert_array_equal(n_out.numpy(), ref["n_out"])
+        idx = run.idx.cpu().numpy()
+        for b in range(2):
+            for h in range(2):
+                n = int(n_out[b, h])
+                assert torch.equal(k_out[b, h, :n], run.k_out[b, h, :n].cpu())
+                assert torch.equal(v_out[b, h, :n], run.v_out[b, h, :n].cpu())
+                assert torch.equal(mod_out[b, h, :n], run.mod_out[b, h, :n].cpu())
+                np.testing.assert_array_equal(bits(v_out[b, h, :n]), bits(v)[b, h][idx[b, h, :n]])
+                if (idx[b, h, :n] == ref["keep_idx"][b, h, :n]).all():      # same kept set: the oracle's bytes
+                    np.testing.assert_array_equal(bits(k_out[b, h, :n]), ref["k_out"][b, h, :n])
+                    np.testing.assert_array_equal(bits(v_out[b, h, :n]), ref["v_out"][b, h, :n])
 
 
 def test_bad_lengths_are_flagged_not_faulted(csp, oracle):
