@@ -372,3 +372,52 @@ int orc_decode_attn(const orc_params* p, const void* q, const void* k, const voi
     }
     return bad ? -1 : 0;
 }
+
+/* Algorithm 1's iteration loop, one appended token: the decode attention of orc_decode_attn, and the row of
+ * n-softmax weights it is built from added to the running sums of Eq. 1. */
+int orc_decode_step(const orc_params* p, const void* q, const void* k, const void* v, const int32_t* n_rows,
+                    const uint8_t* modality, const uint8_t* query_label, int first,
+                    double* out, double* acc_self, double* acc_cross) {
+    if (!p || !q || !k || !v || !n_rows || !modality || !query_label || !out || !acc_self || !acc_cross) return -1;
+    const int64_t d = p->head_dim, cap = p->out_capacity;
+    const int G = p->n_q_heads / p->n_kv_heads;
+    const double scale = p->scale > 0.0 ? p->scale : 1.0 / sqrt((double)d);
+    const int units = p->batch * p->n_kv_heads;
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
+    for (int u = 0; u < units; ++u) {
+        const int b = u / p->n_kv_heads, h = u % p->n_kv_heads;
+        const int64_t rows = n_rows[u];
+        for (int g = 0; g < G; ++g)
+            for (int64_t c = 0; c < d; ++c) out[((int64_t)b * p->n_q_heads + h * G + g) * d + c] = 0.0;
+        if (rows < 0 || rows > cap) { bad = 1; continue; }
+        double* as = acc_self + (int64_t)u * cap;
+        double* ac = acc_cross + (int64_t)u * cap;
+        /* a new window: every slot of the unit starts at zero, also those of rows still to be appended */
+        if (first) for (int64_t t = 0; t < cap; ++t) { as[t] = 0.0; ac[t] = 0.0; }
+        if (rows == 0) continue;
+        const uint8_t* mod = modality + (int64_t)u * cap;
+        const int64_t kbase = (int64_t)u * cap * d;
+        double* o = (double*)malloc(sizeof(double) * (size_t)rows);
+        double* a = (double*)malloc(sizeof(double) * (size_t)rows);
+        for (int g = 0; g < G; ++g) {
+            const int hq = h * G + g;
+            const int64_t qbase = ((int64_t)b * p->n_q_heads + hq) * d;
+            for (int64_t t = 0; t < rows; ++t) {
+                double acc = 0.0;
+                for (int64_t c = 0; c < d; ++c)
+                    acc += load_elem(q, qbase + c, p->dtype) * load_elem(k, kbase + t * d + c, p->dtype);
+                o[t] = acc * scale;                                   /* Eq. 5 for the one new query */
+            }
+            orc_nsoftmax(o, rows, p->n, a);                            /* Eq. 7 over the rows in the cache */
+            double* o_vec = out + qbase;
+            for (int64_t t = 0; t < rows; ++t) {
+                for (int64_t c = 0; c < d; ++c) o_vec[c] += a[t] * load_elem(v, kbase + t * d + c, p->dtype);
+                if (mod[t] == query_label[b]) as[t] += a[t] / G;       /* Eq. 1, one query row */
+                else ac[t] += a[t] / G;
+            }
+        }
+        free(o); free(a);
+    }
+    return bad ? -1 : 0;
+}

@@ -4,7 +4,8 @@
  * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, double-precision
  * restatement of what the paper defines (Eq. 1-4, Eq. 5, Eq. 7, Algorithm 1).
  * It also holds the plain definition of decode attention with the n-softmax
- * normaliser (Section 3.3).  It exists to check the CUDA library and to be timed as a CPU baseline.  It
+ * normaliser (Section 3.3) and of a decode step that carries the scores of Eq. 1 along
+ * (Algorithm 1's iteration loop).  It exists to check the CUDA library and to be timed as a CPU baseline.  It
  * shares no code with the CUDA library and must never be called from it.
  *
  * Every function has at least one independent pin in the CPU test-suite
@@ -101,6 +102,22 @@ int orc_prune_layer(const orc_params* p, const void* q, const void* k, const voi
  * argument (n_rows outside [0, out_capacity]). */
 int orc_decode_attn(const orc_params* p, const void* q, const void* k, const void* v,
                     const int32_t* n_rows, double* out);
+
+/* One decode step of Algorithm 1's iteration loop: orc_decode_attn for the new token's query, and the same
+ * n-softmax weights added to running intra / inter score vectors.  The query of the token at position p sees
+ * exactly the rows the cache holds at that step (rows 0..p, its own included), so its weights are row p of the
+ * attention matrix and never change afterwards: summed over the last W steps they are the scores of Eq. 1 for
+ * the window made of those W queries, without another pass over the cache.
+ *   a_g[t]       = e^{o_{g,t}} / (n + sum_j e^{o_{g,j}})            (Eq. 7, query head g of the KV group)
+ *   acc_self[t] += (1/G) sum_g a_g[t]   if modality[b,hkv,t] == query_label[b]   (intra, Eq. 1)
+ *   acc_cross[t]+= (1/G) sum_g a_g[t]   otherwise                                 (inter, Eq. 1)
+ * modality: [B, Hkv, out_capacity] labels of the cached rows (per head: after a prune heads differ);
+ * query_label: [B]; acc_self, acc_cross: [B, Hkv, out_capacity] doubles; a step adds to t < n_rows[b,hkv];
+ * first != 0 starts a new window: all out_capacity slots of a unit are cleared first (rows appended later
+ * in the window then start from zero).  Returns 0 or -1. */
+int orc_decode_step(const orc_params* p, const void* q, const void* k, const void* v, const int32_t* n_rows,
+                    const uint8_t* modality, const uint8_t* query_label, int first,
+                    double* out, double* acc_self, double* acc_cross);
 
 /* number of OpenMP threads the unit loops will use */
 int orc_num_threads(void);

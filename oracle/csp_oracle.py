@@ -216,3 +216,20 @@ def decode_attn(p: Params, q, k, v, n_rows):
     if lib().orc_decode_attn(C.byref(cp), _ptr(q), _ptr(k), _ptr(v), _ptr(n_rows), _ptr(out)):
         raise ValueError("orc_decode_attn: bad argument")
     return out
+
+
+def decode_step(p: Params, q, k, v, n_rows, modality, query_label, acc_self, acc_cross, first: bool):
+    """One appended token of the iteration loop: decode attention plus the running sums of Eq. 1.
+    modality uint8 [B, Hkv, out_capacity]; query_label uint8 [B]; acc_self / acc_cross float64
+    [B, Hkv, out_capacity], updated in place (overwritten when `first`).  Returns out float64 [B, Hq, d]."""
+    q, k, v = _np(q, _elem(p)), _np(k, _elem(p)), _np(v, _elem(p))
+    n_rows = _np(n_rows, np.int32)
+    modality, query_label = _np(modality, np.uint8), _np(query_label, np.uint8)
+    assert modality.shape == (p.batch, p.n_kv_heads, p.out_capacity) and query_label.shape == (p.batch,)
+    assert acc_self.dtype == np.float64 and acc_self.flags.c_contiguous and acc_cross.flags.c_contiguous
+    out = np.zeros((p.batch, p.n_q_heads, p.head_dim), np.float64)
+    cp = p.c()
+    if lib().orc_decode_step(C.byref(cp), _ptr(q), _ptr(k), _ptr(v), _ptr(n_rows), _ptr(modality),
+                             _ptr(query_label), int(bool(first)), _ptr(out), _ptr(acc_self), _ptr(acc_cross)):
+        raise ValueError("orc_decode_step: bad argument")
+    return out

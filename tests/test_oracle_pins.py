@@ -599,6 +599,110 @@ def test_decode_bf16_inputs_are_widened_exactly(oracle):
                                   oracle.decode_attn(p32, q.float(), k.float(), v.float(), rows))
 
 
+# ---------------------------------------------------------------- Algorithm 1's iteration loop: scores carried along
+
+def _decode_rounds(oracle, seed, L0, steps, W, G, d, n, labels_new):
+    """A cache of L0 rows, then `steps` appended tokens, one decode step each; a new window starts W steps before
+    the end.  Returns everything needed to recompute the result from scratch."""
+    rng = np.random.RandomState(seed)
+    L = L0 + steps
+    k = rng.randn(1, 1, L, d).astype(np.float32)
+    v = rng.randn(1, 1, L, d).astype(np.float32)
+    q_all = (rng.randn(G, L, d) * 1.5).astype(np.float32)            # only the appended positions are ever used
+    mod = np.zeros((1, 1, L), np.uint8)
+    mod[0, 0, :L0] = rng.rand(L0) < 0.5
+    mod[0, 0, L0:] = labels_new
+    p = oracle.Params(1, G, 1, d, 1, 0, L, L, dtype=oracle.F32, n=n)
+    acc_s, acc_c = np.full((1, 1, L), 7.0), np.full((1, 1, L), -3.0)  # stale contents: the first step must clear them
+    outs = []
+    for i in range(steps):
+        pos = L0 + i                                                  # the new token sits at this position
+        q = torch.from_numpy(q_all[None, :, pos])
+        out = oracle.decode_step(p, q, k, v, np.array([[pos + 1]], np.int32), mod, mod[0, :, pos].copy(),
+                                 acc_s, acc_c, first=(i == steps - W))
+        outs.append(out)
+    return p, k, v, q_all, mod, acc_s, acc_c, outs
+
+
+@pytest.mark.parametrize("seed,L0,steps,W,G,n", [(60, 9, 5, 3, 2, 1.0), (61, 4, 6, 6, 1, 0.0), (62, 12, 7, 4, 3, 2.5)])
+def test_decode_steps_carry_the_scores_of_the_final_window(oracle, seed, L0, steps, W, G, n):
+    """Row p of the causal attention matrix is final once the token at p has been decoded.  So the intra / inter
+    sums collected over the last W decode steps equal Eq. 1 on the final cache with those W queries as the
+    observation window: checked against the full-matrix transcription, and against the from-scratch scorer."""
+    d = 4
+    rng = np.random.RandomState(seed + 100)
+    labels_new = (rng.rand(steps) < 0.4).astype(np.uint8)
+    p, k, v, q_all, mod, acc_s, acc_c, outs = _decode_rounds(oracle, seed, L0, steps, W, G, d, n, labels_new)
+    L = L0 + steps
+    es, ec = _brute_force_scores(q_all.astype(np.float64), k[0, 0].astype(np.float64), mod[0, 0], W, 0, n)
+    np.testing.assert_allclose(acc_s[0, 0], es, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(acc_c[0, 0], ec, rtol=1e-12, atol=1e-15)
+    ps = oracle.Params(1, G, 1, d, W, 0, L, L, dtype=oracle.F32, n=n)
+    s, c = oracle.score(ps, q_all[None, :, L - W:], k, mod[0], np.array([L], np.int32))
+    np.testing.assert_allclose(acc_s[0, 0], s[0, 0], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(acc_c[0, 0], c[0, 0], rtol=1e-12, atol=1e-15)
+    # every step's output is plain n-softmax attention over the rows present at that step
+    for i, out in enumerate(outs):
+        rows = L0 + i + 1
+        for g in range(G):
+            o = k[0, 0, :rows].astype(np.float64) @ q_all[g, rows - 1].astype(np.float64) / np.sqrt(d)
+            a = np.exp(o) / (n + np.exp(o).sum())
+            np.testing.assert_allclose(out[0, g], a @ v[0, 0, :rows].astype(np.float64), rtol=1e-12, atol=1e-15)
+
+
+def test_decode_step_zero_query_closed_form_and_mass(oracle):
+    """q = 0: the token decoded with `rows` rows in the cache gives every row 1 / (n + rows); a text token adds
+    that to the intra sum of text rows and to the inter sum of visual rows.  And for any query the two sums gain,
+    together, the row's whole mass sum_t a_t = 1 - n / (n + Z)."""
+    n, d, G = 2.0, 4, 2
+    rng = np.random.RandomState(63)
+    cap = 11
+    k = rng.randn(2, 1, cap, d).astype(np.float32)
+    v = rng.randn(2, 1, cap, d).astype(np.float32)
+    mod = (rng.rand(2, 1, cap) < 0.5).astype(np.uint8)
+    p = oracle.Params(2, G, 1, d, 1, 0, cap, cap, dtype=oracle.F32, n=n)
+    acc_s, acc_c = np.zeros((2, 1, cap)), np.zeros((2, 1, cap))
+    qlab = np.array([0, 1], np.uint8)
+    for step, rows in enumerate((7, 8, 9)):
+        oracle.decode_step(p, torch.zeros(2, G, d), k, v, np.array([[rows], [rows - 2]], np.int32), mod, qlab,
+                           acc_s, acc_c, first=(step == 0))
+    for b, shift in ((0, 0), (1, 2)):
+        for t in range(cap):
+            want = sum(Fraction(1) / (Fraction(2) + (rows - shift)) for rows in (7, 8, 9) if t < rows - shift)
+            same = mod[b, 0, t] == qlab[b]
+            assert abs(acc_s[b, 0, t] - (float(want) if same else 0.0)) < 1e-15
+            assert abs(acc_c[b, 0, t] - (0.0 if same else float(want))) < 1e-15
+    q = torch.from_numpy(rng.randn(2, G, d).astype(np.float32) * 2)
+    a_s, a_c = np.zeros((2, 1, cap)), np.zeros((2, 1, cap))
+    rows = np.array([[cap], [5]], np.int32)
+    oracle.decode_step(p, q, k, v, rows, mod, qlab, a_s, a_c, first=True)
+    for b in range(2):
+        r = int(rows[b, 0])
+        mass = 0.0
+        for g in range(G):
+            z = np.exp(k[b, 0, :r].astype(np.float64) @ q[b, g].double().numpy() / np.sqrt(d)).sum()
+            mass += (1.0 - n / (n + z)) / G
+        assert abs(a_s[b].sum() + a_c[b].sum() - mass) < 1e-13
+        assert (a_s[b, 0, r:] == 0).all() and (a_c[b, 0, r:] == 0).all()
+
+
+def test_decode_step_first_clears_the_unit_and_later_steps_add(oracle):
+    p, q, k, v, rows = _decode_case(oracle, 64, B=1, Hq=2, Hkv=2, cap=13)
+    mod = np.zeros((1, 2, 13), np.uint8)
+    acc_s, acc_c = np.full((1, 2, 13), 5.0), np.full((1, 2, 13), 5.0)
+    out = oracle.decode_step(p, q, k, v, rows, mod, np.array([0], np.uint8), acc_s, acc_c, first=True)
+    np.testing.assert_array_equal(out, oracle.decode_attn(p, q, k, v, rows))
+    for h in range(2):
+        r = int(rows[0, h])
+        assert (acc_s[0, h, r:] == 0.0).all() and (acc_c[0, h] == 0.0).all() and (acc_s[0, h, :r] > 0).all()
+    before = acc_s.copy()
+    oracle.decode_step(p, q, k, v, rows, mod, np.array([1], np.uint8), acc_s, acc_c, first=False)
+    np.testing.assert_array_equal(acc_s, before)                     # a visual query: everything goes to the inter sum
+    for h in range(2):
+        r = int(rows[0, h])
+        np.testing.assert_allclose(acc_c[0, h, :r], before[0, h, :r], rtol=1e-15)
+
+
 def test_benchmark_shapes_match_their_description():
     c1 = synth.config(1)
     assert c1.seq_lens.tolist() == [4096] and c1.budgets.tolist() == [[304, 0, 0, 691]]
