@@ -771,6 +771,117 @@ def run_decode(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_incremental(args, rank, world, local_rank):
+    """`--incremental`: a re-prune round of the serving shape (configs[4]) two ways.  Every head's compacted cache
+    has grown by 64 decoded tokens and is pruned back to its budget, either by csp_prune_layer (the window's 32
+    queries rescan the whole cache) or from the intra / inter sums that the last 32 decode steps carried along
+    (csp_decode_step), which leaves csp_select + csp_compact.  Four distinct layers folded into one call each;
+    decode calls are timed at the final cache length.  Prints its own JSON line; not the default."""
+    from paper_2412_04652_b200 import binding as csp
+    csp.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    cfg = synth.config(4, budget_pct=args.budget_pct)
+    n_fold, W, R, d, H, Hq = 4, cfg.window, cfg.recent, cfg.head_dim, cfg.n_kv_heads, cfg.n_q_heads
+    B = cfg.batch * n_fold
+    cap0 = cfg.out_capacity()
+    cap2 = cap0 + 64
+    p0 = csp.Params(B, Hq, H, d, W, R, cfg.max_len, cap2)
+    parts = [synth.make_layer(cfg, i, dev) for i in range(n_fold)]
+    q0, k0, v0 = (torch.cat([x[j] for x in parts], 0) for j in range(3))
+    del parts
+    mod0 = torch.from_numpy(cfg.modality()).to(dev).repeat(n_fold, 1)
+    lens0 = torch.from_numpy(cfg.seq_lens).to(dev).repeat(n_fold)
+    bud0 = torch.from_numpy(cfg.budgets).to(dev).repeat(n_fold, 1)
+    tot0 = torch.from_numpy(cfg.total_budget).to(dev).repeat(n_fold)
+    k_c = torch.zeros(B, H, cap2, d, dtype=cfg.dtype, device=dev)
+    v_c = torch.zeros_like(k_c)
+    mod_c = torch.zeros(B, H, cap2, dtype=torch.uint8, device=dev)
+    n0 = torch.zeros(B, H, dtype=torch.int32, device=dev)
+    ws0 = csp.new_workspace(p0, dev)
+    csp.prune_layer(p0, q0, k0, v0, mod0, lens0, bud0, k_c, v_c, mod_c, n0, ws0, total_budget=tot0)   # round 0
+    status = csp.device_status(ws0)
+    del q0, k0, v0, ws0
+    torch.cuda.empty_cache()
+    n_host = n0.cpu().numpy()
+    assert (n_host == n_host[:, :1]).all() and (n_host > 0).all()
+    gen = torch.Generator(device=dev).manual_seed(77)
+    for b in range(B):                                           # 64 decoded text tokens behind the kept rows
+        n = int(n_host[b, 0])
+        k_c[b, :, n:n + 64] = torch.randn(H, 64, d, device=dev, generator=gen).to(cfg.dtype)
+        v_c[b, :, n:n + 64] = torch.randn(H, 64, d, device=dev, generator=gen).to(cfg.dtype)
+        mod_c[b, :, n:n + 64] = 0
+    n_rows = (n0 + 64).contiguous()
+    lens2 = n_rows[:, 0].contiguous()
+    tokens_per_layer = int(lens2.sum().item()) // n_fold
+    qs = torch.randn(W, B, Hq, d, device=dev, generator=gen).to(cfg.dtype)
+    qlab = torch.zeros(B, dtype=torch.uint8, device=dev)
+    pd = csp.Params(B, Hq, H, d, 1, 0, cap2, cap2)
+    out = torch.zeros(B, Hq, d, device=dev)
+    acc_s = torch.zeros(B, H, cap2, device=dev)
+    acc_c = torch.zeros(B, H, cap2, device=dev)
+    wd, wst = csp.new_decode_workspace(pd, dev), csp.new_decode_step_workspace(pd, dev)
+    # the prune that follows: budgets per sequence as in round 0, cache length = kept rows + 64
+    totals = cfg.total_budget.astype(np.int64)
+    budgets = np.array([synth.budgets_from_total(int(t), R) for t in totals], np.int32)
+    bud2 = torch.from_numpy(budgets).to(dev).repeat(n_fold, 1)
+    tot2 = torch.from_numpy(totals.astype(np.int32)).to(dev).repeat(n_fold)
+    p2 = csp.Params(B, Hq, H, d, W, R, cap2, cap0)
+    k_o = torch.empty(B, H, cap0, d, dtype=cfg.dtype, device=dev)
+    v_o = torch.empty_like(k_o)
+    mod_o = torch.empty(B, H, cap0, dtype=torch.uint8, device=dev)
+    n_o = torch.zeros(B, H, dtype=torch.int32, device=dev)
+    idx = torch.empty(B, H, cap0, dtype=torch.int32, device=dev)
+    ws2 = csp.new_workspace(p2, dev)
+    q_win = qs.permute(1, 2, 0, 3).contiguous()
+    pb = PathBench(csp, args, dev, local_rank, None)
+    stream = pb.stream
+    reps = max(3, min(50, args.steps))
+    with torch.cuda.stream(stream):
+        for i in range(W):                                       # the window's decode steps, so the sums are real
+            csp.decode_step(pd, qs[i], k_c, v_c, n_rows, mod_c, qlab, i == 0, out, acc_s, acc_c, wst)
+        stream.synchronize()
+        t_dec = pb.time_graph_of(lambda: csp.decode_attn(pd, qs[0], k_c, v_c, n_rows, out, wd), reps)
+        acc_s2, acc_c2 = acc_s.clone(), acc_c.clone()           # timing replays must not disturb the real sums
+        t_step = pb.time_graph_of(lambda: csp.decode_step(pd, qs[1], k_c, v_c, n_rows, mod_c, qlab, False, out, acc_s2, acc_c2, wst), reps)
+        t_full = pb.time_graph_of(lambda: csp.prune_layer(p2, q_win, k_c, v_c, mod_c, lens2, bud2, k_o, v_o, mod_o, n_o, ws2,
+                                                          total_budget=tot2), reps)
+        n_full = n_o.clone()
+
+        def from_sums():
+            csp.select(p2, acc_s, acc_c, mod_c, lens2, bud2, idx, n_o, ws2, total_budget=tot2)
+            csp.compact(p2, k_c, v_c, mod_c, idx, n_o, k_o, v_o, mod_o)
+        t_inc = pb.time_graph_of(from_sums, reps)
+        status |= csp.device_status(ws2) | csp.device_status(wd) | csp.device_status(wst)
+        same_rows = bool(torch.equal(n_full, n_o))
+    per_layer = lambda ms: ms / n_fold
+    extra_per_step = per_layer(t_step - t_dec)
+    inc_total = per_layer(t_inc) + W * max(extra_per_step, 0.0)
+    es = 2
+    rows_total = int(n_rows.clamp(min=0).sum().item())
+    dec_bytes = rows_total * 2 * d * es
+    peak, peak_kind = measured_peaks()
+    if rank == 0:
+        line = {"metric": METRIC, "value": world * tokens_per_layer / (inc_total * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": reps, "warmup": 3, "ms_per_step": inc_total * cfg.n_layers, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"configs[4] {cfg.name}, re-prune round 1 from the sums the decode steps carried",
+                           "layers_timed": n_fold, "batch": cfg.batch, "kv_heads": H, "head_dim": d,
+                           "sum_seq_len": tokens_per_layer, "window": W, "recent": R,
+                           "launch": "four layers folded into one call of each kind; decode calls timed at the final cache length"},
+                "per_layer_ms": {"decode_attn": per_layer(t_dec), "decode_step": per_layer(t_step),
+                                 "extra_per_decode_step": extra_per_step,
+                                 "select_plus_compact_from_sums": per_layer(t_inc),
+                                 "reprune_incremental_total": inc_total,
+                                 "reprune_full_rescan": per_layer(t_full)},
+                "full_rescan": {"value": world * tokens_per_layer / (per_layer(t_full) * 1e-3), "unit": UNIT},
+                "decode": {"achieved_gbs": dec_bytes / (t_dec * 1e-3) / 1e9, "with_sums_gbs": dec_bytes / (t_step * 1e-3) / 1e9,
+                           "peak": peak, "peak_kind": f"of {peak_kind}"},
+                "same_row_counts_both_ways": same_rows, "device_status": status, "gpu_launches": reps * 9, "e2e": None,
+                "cpu_baseline": None}
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -792,6 +903,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode", action="store_true",
                     help="time the step after the pruning pass instead: n-softmax decode attention over the pruned caches")
+    ap.add_argument("--incremental", action="store_true",
+                    help="a re-prune round of configs[4] from the sums carried by csp_decode_step, against the full rescan")
     ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
     ap.add_argument("--rounds", type=int, default=4, help="re-prune rounds of configs[4] under --all-configs")
     ap.add_argument("--all-configs", action="store_true",
@@ -813,6 +926,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
     if args.decode:
         run_decode(args, rank, world, local_rank)
+        return
+    if args.incremental:
+        run_incremental(args, rank, world, local_rank)
         return
     from paper_2412_04652_b200 import binding as csp
     csp.lib()

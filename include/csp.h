@@ -203,6 +203,33 @@ csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_
                            const int32_t* n_rows, float* out,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Bytes of scratch that csp_decode_step needs: those of csp_decode_attn plus one row of logits per query head
+ * and unit.  The first 256 bytes must be zero before first use (csp_workspace_reset). */
+size_t csp_decode_step_workspace_bytes(const csp_params* p);
+
+/*
+ * Algorithm 1's iteration loop, one appended token: csp_decode_attn for the new token's query, and the scores
+ * of Eq. 1 carried along, so that the next prune needs no pass over the cache of its own.  The query of the
+ * token at position pos sees exactly the n_rows = pos + 1 rows the cache holds at that step, its own included, so
+ * its n-softmax weights (Eq. 7) are row pos of the attention matrix and are final.  They are averaged over the
+ * query heads of the KV group and added to the intra sum of the rows that carry the query's label and to the
+ * inter sum of the others (Eq. 1).  After the last W steps before a prune, started with first_step != 0, the two
+ * arrays hold what csp_score would compute on that cache with those W queries as the observation window;
+ * csp_select and csp_compact then finish the prune (Eq. 2-4).
+ *   q, k, v, n_rows, out   as for csp_decode_attn; the new token's K and V rows are already in the cache
+ *   modality     labels of the cached rows, element (b,h,t) at modality[b*mod_stride_b + h*mod_stride_h + t]
+ *   query_label  [B] uint8: label of each sequence's new token
+ *   first_step   != 0 starts a new window: all out_capacity slots of every unit are overwritten (rows that are
+ *                appended later in the window start from zero); 0 adds to the slots t < n_rows
+ *   acc_self, acc_cross  [B, H_kv, out_capacity] fp32, the layout of csp_select's score vectors with
+ *                max_len = out_capacity
+ * bf16 caches with head_dim 64 or 128.  Nothing is allocated; the caller owns the workspace.
+ */
+csp_status csp_decode_step(const csp_params* p, csp_tensor q, csp_tensor k, csp_tensor v, const int32_t* n_rows,
+                           const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                           const uint8_t* query_label, int32_t first_step, float* out, float* acc_self,
+                           float* acc_cross, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Bytes of device staging that csp_prune_layer_host needs for these parameters. */
 size_t csp_host_staging_bytes(const csp_params* p);
 

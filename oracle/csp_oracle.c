@@ -421,3 +421,87 @@ int orc_decode_step(const orc_params* p, const void* q, const void* k, const voi
     }
     return bad ? -1 : 0;
 }
+
+/* ---- the distribution-gap diagnostic (Section 1) -------------------------------------------------- */
+
+double orc_js_divergence(const int64_t* hp, const int64_t* hq, int bins) {
+    double sp = 0.0, sq = 0.0;
+    for (int j = 0; j < bins; ++j) { sp += (double)hp[j]; sq += (double)hq[j]; }
+    if (sp <= 0.0 || sq <= 0.0) return NAN;
+    double js = 0.0;
+    for (int j = 0; j < bins; ++j) {
+        const double pj = (double)hp[j] / sp, qj = (double)hq[j] / sq, mj = 0.5 * (pj + qj);
+        if (pj > 0.0) js += 0.5 * pj * log(pj / mj);
+        if (qj > 0.0) js += 0.5 * qj * log(qj / mj);
+    }
+    return js;
+}
+
+static int hist_bin(double log2w) {
+    double j = floor((log2w - ORC_HIST_LO) / ORC_HIST_WIDTH);
+    if (!(j >= 0.0)) j = 0.0;                      /* also catches -inf (weight 0) */
+    if (j > ORC_HIST_BINS - 1) j = ORC_HIST_BINS - 1;
+    return (int)j;
+}
+
+int orc_weight_histogram(const orc_params* p, const void* q, const void* k,
+                         const uint8_t* modality, int mod_per_head, const int32_t* seq_lens,
+                         int64_t* hist, int64_t* near, double near_eps, double* js, double* js_all) {
+    if (!p || !q || !k || !modality || !seq_lens || !hist) return -1;
+    if (p->n_kv_heads <= 0 || p->n_q_heads % p->n_kv_heads) return -1;
+    const int G = p->n_q_heads / p->n_kv_heads, W = p->window, d = p->head_dim;
+    const int units = p->batch * p->n_kv_heads;
+    const double scale = p->scale > 0.0 ? p->scale : 1.0 / sqrt((double)d);
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1) reduction(|:bad)
+    for (int u = 0; u < units; ++u) {
+        const int b = u / p->n_kv_heads, h = u % p->n_kv_heads;
+        const int64_t L = seq_lens[b];
+        int64_t* hu = hist + (int64_t)u * 2 * ORC_HIST_BINS;
+        int64_t* nu = near ? near + (int64_t)u * 2 * ORC_HIST_BINS : NULL;
+        for (int j = 0; j < 2 * ORC_HIST_BINS; ++j) { hu[j] = 0; if (nu) nu[j] = 0; }
+        if (js) js[u] = NAN;
+        if (L > p->max_len || L < 0) { bad = 1; continue; }
+        if (unit_is_short(p, L)) continue;
+        const int64_t N = L - p->recent;
+        const uint8_t* mod = mod_row(p, modality, mod_per_head, b, h);
+        double* o = (double*)malloc(sizeof(double) * (size_t)L);
+        double* a = (double*)malloc(sizeof(double) * (size_t)L);
+        const int64_t kbase = (int64_t)u * p->max_len * d;
+        for (int g = 0; g < G; ++g) {
+            const int64_t qbase = (((int64_t)b * p->n_q_heads + h * G + g) * W) * d;
+            for (int w = 0; w < W; ++w) {
+                const int64_t pos = L - W + w;
+                for (int64_t t = 0; t <= pos; ++t) {
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c)
+                        acc += load_elem(q, qbase + (int64_t)w * d + c, p->dtype) * load_elem(k, kbase + t * d + c, p->dtype);
+                    o[t] = acc * scale;                           /* Eq. 5 */
+                }
+                orc_nsoftmax(o, pos + 1, p->n, a);                /* Eq. 7 */
+                for (int64_t t = 0; t < N && t <= pos; ++t) {
+                    const int cls = mod[pos] == mod[t] ? 0 : 1;   /* intra / inter, as in Eq. 1 */
+                    const double l2 = a[t] > 0.0 ? log2(a[t]) : -INFINITY;
+                    hu[cls * ORC_HIST_BINS + hist_bin(l2)] += 1;
+                    if (nu && a[t] > 0.0) {
+                        /* the nearest bin edge above the first and at or below the last bin's lower edge */
+                        const double e = (l2 - ORC_HIST_LO) / ORC_HIST_WIDTH;
+                        const double je = floor(e + 0.5);
+                        if (je >= 1.0 && je <= ORC_HIST_BINS - 1 && fabs(e - je) * ORC_HIST_WIDTH <= near_eps)
+                            nu[cls * ORC_HIST_BINS + (int)je] += 1;
+                    }
+                }
+            }
+        }
+        free(o); free(a);
+        if (js) js[u] = orc_js_divergence(hu, hu + ORC_HIST_BINS, ORC_HIST_BINS);
+    }
+    if (js_all) {
+        int64_t tot[2 * ORC_HIST_BINS];
+        for (int j = 0; j < 2 * ORC_HIST_BINS; ++j) tot[j] = 0;
+        for (int u = 0; u < units; ++u)
+            for (int j = 0; j < 2 * ORC_HIST_BINS; ++j) tot[j] += hist[(int64_t)u * 2 * ORC_HIST_BINS + j];
+        *js_all = orc_js_divergence(tot, tot + ORC_HIST_BINS, ORC_HIST_BINS);
+    }
+    return bad ? -1 : 0;
+}

@@ -119,6 +119,31 @@ int orc_decode_step(const orc_params* p, const void* q, const void* k, const voi
                     const uint8_t* modality, const uint8_t* query_label, int first,
                     double* out, double* acc_self, double* acc_cross);
 
+/* Diagnostic behind the method's motivation (Section 1, the figure on the distribution gap): the attention
+ * weights of the observation window, per query head and not averaged, split into intra-modality pairs (query
+ * and key carry the same label) and inter-modality pairs, each collected in a histogram of log2(weight), and the
+ * Jensen-Shannon divergence between the two normalised histograms.
+ *   weights: A[g,w,t] of Eq. 7 for window row w (position L-W+w), candidate keys t < L-R with t <= L-W+w
+ *   bin j of ORC_HIST_BINS covers log2(A) in [ORC_HIST_LO + j ORC_HIST_WIDTH, ORC_HIST_LO + (j+1) ORC_HIST_WIDTH);
+ *   values below the first bin (and exact zeros) go to bin 0, values above the last to the last
+ *   hist [B,Hkv,2,ORC_HIST_BINS] int64 counts (0: intra, 1: inter)
+ *   near (optional) [B,Hkv,2,ORC_HIST_BINS]: how many weights lie within near_eps (in log2 units) of the lower
+ *        edge of bin j, i.e. could fall on either side of it in another precision
+ *   js   (optional) [B,Hkv]: orc_js_divergence of the unit's two histograms
+ *   js_all (optional) [1]: the same for the histograms summed over all units of the call
+ * The paper plots a kernel density estimate; the binning (half-octave bins from 2^-32 to 1) is this
+ * library's choice and is stated wherever the result is reported. */
+enum { ORC_HIST_BINS = 64 };
+#define ORC_HIST_LO (-32.0)
+#define ORC_HIST_WIDTH 0.5
+int orc_weight_histogram(const orc_params* p, const void* q, const void* k,
+                         const uint8_t* modality, int mod_per_head, const int32_t* seq_lens,
+                         int64_t* hist, int64_t* near, double near_eps, double* js, double* js_all);
+
+/* Jensen-Shannon divergence, in nats, between two histograms normalised to sum 1:
+ * 1/2 KL(P || M) + 1/2 KL(Q || M), M = (P + Q) / 2, 0 log 0 = 0.  NaN if either histogram is empty. */
+double orc_js_divergence(const int64_t* hist_p, const int64_t* hist_q, int bins);
+
 /* number of OpenMP threads the unit loops will use */
 int orc_num_threads(void);
 

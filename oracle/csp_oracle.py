@@ -23,6 +23,7 @@ COMBINE_OR, COMBINE_AND = 0, 1
 SELECT_SEGMENTED, SELECT_GLOBAL, SELECT_OVERALL = 0, 1, 2
 HEADS_PER_KV, HEADS_MEAN_ALL = 0, 1
 FLAG_K_CLAMPED, FLAG_CAPACITY, FLAG_IDENTITY = 1, 2, 4
+HIST_BINS, HIST_LO, HIST_WIDTH = 64, -32.0, 0.5
 
 
 def build(force: bool = False) -> str:
@@ -74,6 +75,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.orc_topk.restype = C.c_int
         _lib.orc_num_threads.restype = C.c_int
+        _lib.orc_js_divergence.restype = C.c_double
     return _lib
 
 
@@ -233,3 +235,27 @@ def decode_step(p: Params, q, k, v, n_rows, modality, query_label, acc_self, acc
                              _ptr(query_label), int(bool(first)), _ptr(out), _ptr(acc_self), _ptr(acc_cross)):
         raise ValueError("orc_decode_step: bad argument")
     return out
+
+
+def js_divergence(hist_p, hist_q) -> float:
+    hp, hq = _np(hist_p, np.int64), _np(hist_q, np.int64)
+    assert hp.shape == hq.shape and hp.ndim == 1
+    return float(lib().orc_js_divergence(_ptr(hp), _ptr(hq), C.c_int(hp.size)))
+
+
+def weight_histogram(p: Params, q, k, modality, seq_lens, near_eps: float = 0.0):
+    """Histograms of log2(attention weight) of the window, intra- and inter-modality, and their JS divergence.
+    Returns (hist int64 [B,Hkv,2,HIST_BINS], near int64 (same shape), js float64 [B,Hkv], js_all float)."""
+    q, k = _np(q, _elem(p)), _np(k, _elem(p))
+    modality = _np(modality, np.uint8)
+    seq_lens = _np(seq_lens, np.int32)
+    per_head = int(modality.ndim == 3)
+    hist = np.zeros((p.batch, p.n_kv_heads, 2, HIST_BINS), np.int64)
+    near = np.zeros_like(hist)
+    js = np.zeros((p.batch, p.n_kv_heads), np.float64)
+    js_all = C.c_double(0.0)
+    cp = p.c()
+    if lib().orc_weight_histogram(C.byref(cp), _ptr(q), _ptr(k), _ptr(modality), per_head, _ptr(seq_lens),
+                                  _ptr(hist), _ptr(near), C.c_double(near_eps), _ptr(js), C.byref(js_all)):
+        raise ValueError("orc_weight_histogram: bad argument")
+    return hist, near, js, float(js_all.value)

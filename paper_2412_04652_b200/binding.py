@@ -26,7 +26,7 @@ DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
 EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_select", "csp_compact",
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
            "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
-           "csp_decode_workspace_bytes", "csp_decode_attn")
+           "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step")
 
 
 class CspError(RuntimeError):
@@ -115,6 +115,10 @@ def lib() -> C.CDLL:
         l.csp_decode_workspace_bytes.argtypes = [P]
         l.csp_decode_attn.restype = C.c_int
         l.csp_decode_attn.argtypes = [P, CTensor, CTensor, CTensor, vp, vp, vp, sz, vp]
+        l.csp_decode_step_workspace_bytes.restype = sz
+        l.csp_decode_step_workspace_bytes.argtypes = [P]
+        l.csp_decode_step.restype = C.c_int
+        l.csp_decode_step.argtypes = [P, CTensor, CTensor, CTensor, vp, vp, i64, i64, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         l.csp_device_status.restype = C.c_int
         l.csp_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         l.csp_status_string.restype = C.c_char_p
@@ -191,6 +195,29 @@ def decode_attn(p: Params, q, k, v, n_rows, out, ws):
     qt = CTensor(q.data_ptr(), q.stride(0), q.stride(1), q.shape[2])
     _check(lib().csp_decode_attn(C.byref(cp), qt, tensor4(k), tensor4(v), _ptr(n_rows), _ptr(out), _ptr(ws),
                                  ws.numel(), _stream()), "csp_decode_attn")
+
+
+def new_decode_step_workspace(p: Params, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and zeroes a workspace for csp_decode_step."""
+    cp = p.c()
+    n = int(lib().csp_decode_step_workspace_bytes(C.byref(cp)))
+    if n == 0:
+        raise CspError(ERR_UNSUPPORTED, "csp_decode_step_workspace_bytes")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def decode_step(p: Params, q, k, v, n_rows, modality, query_label, first_step, out, acc_self, acc_cross, ws):
+    """csp_decode_attn plus the running intra / inter sums: modality uint8 [B, Hkv, cap] (or [B, cap]), query_label
+    uint8 [B], acc_self / acc_cross fp32 [B, Hkv, cap] (dense)."""
+    cp = p.c()
+    assert q.dim() == 3 and q.stride(2) == 1 and out.is_contiguous() and out.dtype == torch.float32
+    assert acc_self.is_contiguous() and acc_cross.is_contiguous() and acc_self.dtype == torch.float32
+    assert query_label.dtype == torch.uint8 and query_label.is_contiguous()
+    qt = CTensor(q.data_ptr(), q.stride(0), q.stride(1), q.shape[2])
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_decode_step(C.byref(cp), qt, tensor4(k), tensor4(v), _ptr(n_rows), _ptr(modality), sb, sh,
+                                 _ptr(query_label), int(bool(first_step)), _ptr(out), _ptr(acc_self), _ptr(acc_cross),
+                                 _ptr(ws), ws.numel(), _stream()), "csp_decode_step")
 
 
 def score(p: Params, q_win, k, modality, seq_lens, score_self, score_cross, ws, lse=None):

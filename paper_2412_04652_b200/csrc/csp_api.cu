@@ -365,6 +365,28 @@ csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_
     return launch_decode_attn(*p, q, k, v, n_rows, out, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t csp_decode_step_workspace_bytes(const csp_params* p) {
+    if (check_params(p) != CSP_OK) return 0;
+    return decode_step_workspace_bytes(*p);
+}
+
+csp_status csp_decode_step(const csp_params* p, csp_tensor q, csp_tensor k, csp_tensor v, const int32_t* n_rows,
+                           const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                           const uint8_t* query_label, int32_t first_step, float* out, float* acc_self,
+                           float* acc_cross, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!q.ptr || !k.ptr || !v.ptr || !n_rows || !out || !modality || !query_label || !acc_self || !acc_cross)
+        return CSP_ERR_INVALID_ARG;
+    if (p->dtype != CSP_BF16 || (p->head_dim != 64 && p->head_dim != 128)) return CSP_ERR_UNSUPPORTED;
+    if (!tensor_ok(*p, q) || !tensor_ok(*p, k) || !tensor_ok(*p, v)) return CSP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < decode_step_workspace_bytes(*p) || (uintptr_t(workspace) % 256))
+        return CSP_ERR_WORKSPACE;
+    if ((st = check_arch()) != CSP_OK) return st;
+    DecodeStepArgs step = {modality, mod_stride_b, mod_stride_h, query_label, acc_self, acc_cross, first_step ? 1 : 0};
+    return launch_decode_attn(*p, q, k, v, n_rows, out, workspace, static_cast<cudaStream_t>(cuda_stream), &step);
+}
+
 csp_status csp_device_status(void* workspace, void* cuda_stream, int32_t* host_out) {
     if (!workspace) return CSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -41,6 +41,14 @@ struct DecodeArgs {
     int32_t* next_item;                            // work counter in the status area: zero between calls
     int32_t n_kv_heads, group, head_dim, capacity, splits, tiles_per_split;
     float n, scale_log2;
+    // csp_decode_step only: the step's logits are kept so that its n-softmax weights can be added to the running
+    // intra / inter sums of Eq. 1 once the row's normaliser is known
+    float* logits;                                 // [units, G, capacity]: o scale log2(e), or null
+    float* rowstat;                                // [units, G, 2]: reference exponent m, weight 1 / (G (n 2^-m + l))
+    const uint8_t* modality; int64_t mod_sb, mod_sh;
+    const uint8_t* query_label;                    // [B]
+    float* acc_self; float* acc_cross;             // [units, capacity]
+    int32_t first_step;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -77,7 +85,7 @@ __device__ __forceinline__ bool consumers_any(bool pred) {
     return r != 0;
 }
 
-template <int NH>   // head_dim = 64 NH
+template <int NH, bool kKeepLogits>   // head_dim = 64 NH; kKeepLogits: also write every logit to a.logits
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const DecodeArgs a, const int n_items) {
@@ -231,6 +239,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 const int r0 = row_w + 2 * qd;
                 float xs[4] = {r0 < rows ? s0[0] * a.scale_log2 : kNeg, r0 + 1 < rows ? s0[1] * a.scale_log2 : kNeg,
                                r0 + 8 < rows ? s1[0] * a.scale_log2 : kNeg, r0 + 9 < rows ? s1[1] * a.scale_log2 : kNeg};
+                if (kKeepLogits && g < G) {
+                    float* const lrow = a.logits + (int64_t(x.u) * G + g) * a.capacity;
+                    if (r0 < rows) lrow[r0] = xs[0];
+                    if (r0 + 1 < rows) lrow[r0 + 1] = xs[1];
+                    if (r0 + 8 < rows) lrow[r0 + 8] = xs[2];
+                    if (r0 + 9 < rows) lrow[r0 + 9] = xs[3];
+                }
                 float mx = fmaxf(fmaxf(xs[0], xs[1]), fmaxf(xs[2], xs[3]));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
@@ -322,11 +337,41 @@ __global__ void decode_merge_kernel(const DecodeArgs a) {
     float l = 0.f;
     for (int s = 0; s < used; ++s) l += part[s * stride + D + 1] * ex2f(part[s * stride + D] - m);
     const float denom = a.n * ex2f(-m) + l;
+    if (a.rowstat && threadIdx.x == 0) {
+        a.rowstat[(int64_t(u) * a.group + g) * 2] = m;
+        a.rowstat[(int64_t(u) * a.group + g) * 2 + 1] = (used > 0 && denom > 0.f) ? 1.0f / (float(a.group) * denom) : 0.f;
+    }
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
         float v = 0.f;
         for (int s = 0; s < used; ++s) v += part[s * stride + c] * ex2f(part[s * stride + D] - m);
         o[c] = (used > 0 && denom > 0.f) ? v / denom : 0.f;
     }
+}
+
+// One query row of Eq. 1: the step's n-softmax weights, averaged over the query heads of the KV group, are added to
+// the intra sum of the cached rows that carry the query's label and to the inter sum of the others.  On the first
+// step of a window every slot of the unit is (over)written, so rows appended later start from zero.
+__global__ void decode_accumulate_kernel(const DecodeArgs a) {
+    const int u = blockIdx.y, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= a.capacity) return;
+    int rows = a.n_rows[u];
+    rows = rows < 0 ? 0 : (rows > a.capacity ? a.capacity : rows);
+    float* const as = a.acc_self + int64_t(u) * a.capacity;
+    float* const ac = a.acc_cross + int64_t(u) * a.capacity;
+    if (t >= rows) {
+        if (a.first_step) { as[t] = 0.f; ac[t] = 0.f; }
+        return;
+    }
+    float w = 0.f;
+    for (int g = 0; g < a.group; ++g) {
+        const float m = a.rowstat[(int64_t(u) * a.group + g) * 2], f = a.rowstat[(int64_t(u) * a.group + g) * 2 + 1];
+        w += ex2f(a.logits[(int64_t(u) * a.group + g) * a.capacity + t] - m) * f;
+    }
+    const bool same = a.modality[int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh + t] == a.query_label[b];
+    const float s0 = a.first_step ? 0.f : as[t], c0 = a.first_step ? 0.f : ac[t];
+    as[t] = s0 + (same ? w : 0.f);
+    ac[t] = c0 + (same ? 0.f : w);
 }
 
 }  // namespace
@@ -347,12 +392,29 @@ size_t decode_workspace_bytes(const csp_params& p) {
     return kStatusBytes + round256(units * size_t(decode_splits(p)) * G * size_t(p.head_dim + 2) * 4);
 }
 
+size_t decode_step_workspace_bytes(const csp_params& p) {
+    const size_t units = size_t(p.batch) * size_t(p.n_kv_heads);
+    const size_t G = size_t(p.n_q_heads / p.n_kv_heads);
+    return decode_workspace_bytes(p) + round256(units * G * size_t(p.out_capacity) * 4) + round256(units * G * 8);
+}
+
 csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
-                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s) {
+                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s, const DecodeStepArgs* step) {
     if (p.dtype != CSP_BF16 || (p.head_dim != 64 && p.head_dim != 128)) return CSP_ERR_UNSUPPORTED;
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     DecodeArgs a;
+    a.logits = nullptr; a.rowstat = nullptr; a.modality = nullptr; a.mod_sb = a.mod_sh = 0; a.query_label = nullptr;
+    a.acc_self = a.acc_cross = nullptr; a.first_step = 0;
+    if (step) {
+        char* const extra = static_cast<char*>(ws) + decode_workspace_bytes(p);
+        a.logits = reinterpret_cast<float*>(extra);
+        a.rowstat = reinterpret_cast<float*>(extra + round256(size_t(units) * (p.n_q_heads / p.n_kv_heads) *
+                                                              size_t(p.out_capacity) * 4));
+        a.modality = step->modality; a.mod_sb = step->mod_sb; a.mod_sh = step->mod_sh;
+        a.query_label = step->query_label; a.acc_self = step->acc_self; a.acc_cross = step->acc_cross;
+        a.first_step = step->first_step;
+    }
     a.q = q.ptr; a.q_sb = q.stride_b; a.q_sh = q.stride_h;
     a.n_rows = n_rows;
     a.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
@@ -374,15 +436,21 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
         const int NH = p.head_dim / 64;
         const size_t smem = 1024 + size_t(kDecStages) * 2 * NH * kDecBlock + size_t(kDecWarps) * 8 * (p.head_dim + 2) * 4 +
                             16 * kDecStages + 64;
-        auto kern = NH == 1 ? decode_attn_kernel<1> : decode_attn_kernel<2>;
-        static std::atomic<bool> configured[2][kMaxDevices];
-        if (!raise_smem_limit(kern, int(smem), configured[NH - 1])) return CSP_ERR_CUDA;
+        auto kern = step ? (NH == 1 ? decode_attn_kernel<1, true> : decode_attn_kernel<2, true>)
+                         : (NH == 1 ? decode_attn_kernel<1, false> : decode_attn_kernel<2, false>);
+        static std::atomic<bool> configured[4][kMaxDevices];
+        if (!raise_smem_limit(kern, int(smem), configured[(step ? 2 : 0) + NH - 1])) return CSP_ERR_CUDA;
         const int n_items = units * a.splits, sms = sm_count();
         kern<<<n_items < sms ? n_items : sms, kDecThreads, smem, s>>>(tk, tv, a, n_items);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
     }
     decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);
-    return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
+    if (step && p.out_capacity > 0) {
+        decode_accumulate_kernel<<<dim3((p.out_capacity + 255) / 256, units), 256, 0, s>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
+    }
+    return CSP_OK;
 }
 
 }  // namespace csp

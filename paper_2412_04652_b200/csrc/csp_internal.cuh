@@ -146,7 +146,16 @@ bool make_cache_tensor_map(CUtensorMap* map, const csp_tensor& t, int dtype, int
 // decode attention over the pruned cache (csp_decode.cu)
 int decode_splits(const csp_params& p);
 size_t decode_workspace_bytes(const csp_params& p);
+// what csp_decode_step adds to a decode call: the labels and the running sums of Eq. 1
+struct DecodeStepArgs {
+    const uint8_t* modality; int64_t mod_sb, mod_sh;
+    const uint8_t* query_label;
+    float* acc_self; float* acc_cross;
+    int32_t first_step;
+};
+size_t decode_step_workspace_bytes(const csp_params& p);
 csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
-                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s);
+                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s,
+                              const DecodeStepArgs* step = nullptr);
 
 }  // namespace csp

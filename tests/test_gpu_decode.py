@@ -136,3 +136,122 @@ def test_decode_bad_row_count_is_flagged_and_host_errors(csp, oracle):
     with pytest.raises(csp.CspError) as e:      # fp32 caches are not supported by this entry point
         csp.decode_attn(p32, q.cuda().float(), k.cuda().float(), v.cuda().float(), rows.cuda(), out, ws)
     assert e.value.code == 2
+
+
+# ------------------------------------------------------------------ Algorithm 1's iteration loop: csp_decode_step
+
+def _score_tolerance_ok(got, want, what):
+    """The score tolerance of the pruning pass: |gpu - oracle| <= 2e-3 |oracle| + 1e-6 max|oracle| per unit."""
+    for u in range(want.shape[0]):
+        w = want[u].astype(np.float64)
+        tol = 2e-3 * np.abs(w) + 1e-6 * np.abs(w).max()
+        bad = np.abs(got[u] - w) > tol
+        assert not bad.any(), f"{what} unit {u}: {bad.sum()} of {w.size} sums off; worst {np.abs(got[u] - w).max()}"
+        assert (got[u][w == 0.0] == 0.0).all(), f"{what} unit {u}: structural zeros must be exactly 0"
+
+
+@pytest.mark.parametrize("Hq,Hkv,d,L0,steps,W", [(4, 2, 128, (700, 333), 40, 32), (7, 1, 64, (150,), 20, 16),
+                                                 (8, 8, 128, (64, 1, 129, 40, 300, 77, 2, 500), 33, 32)])
+def test_decode_steps_carry_the_scores_and_the_reprune_follows(csp, oracle, Hq, Hkv, d, L0, steps, W):
+    """Tokens are appended one at a time to a cache of ragged per-sequence lengths; every step runs csp_decode_step.
+    Checked: each step's attention output against the oracle; the running intra / inter sums against the oracle's
+    (element by element) and against csp_score run from scratch on the final cache with the last W queries as the
+    window; then csp_select on the carried sums is the exact selection for those sums and agrees with the
+    selection from the from-scratch scores except at boundary ties."""
+    B, G = len(L0), Hq // Hkv
+    cap = max(L0) + steps
+    gen = torch.Generator().manual_seed(7 * Hq + steps)
+    k = torch.randn(B, Hkv, cap, d, generator=gen).to(torch.bfloat16)
+    v = torch.randn(B, Hkv, cap, d, generator=gen).to(torch.bfloat16)
+    mod = (torch.rand(B, Hkv, cap, generator=gen) < 0.5).to(torch.uint8)          # labels differ per head after a prune
+    qs = (torch.randn(steps, B, Hq, d, generator=gen) * 1.5).to(torch.bfloat16)
+    new_label = (torch.rand(steps, B, generator=gen) < 0.3).to(torch.uint8)        # some appended tokens are visual
+    for b in range(B):                                                              # appended rows carry their token's label
+        for i in range(steps):
+            mod[b, :, L0[b] + i] = new_label[i, b]
+    p = csp.Params(B, Hq, Hkv, d, 1, 0, cap, cap)
+    po = oracle.Params(B, Hq, Hkv, d, 1, 0, cap, cap, dtype=oracle.BF16)
+    kd, vd, modd = k.cuda(), v.cuda(), mod.cuda()
+    for b in range(B):                               # rows not yet appended are unspecified: make them hostile
+        kd[b, :, L0[b]:] = float("nan")
+        vd[b, :, L0[b]:] = float("inf")
+    acc_s = torch.full((B, Hkv, cap), 9.0, device="cuda")
+    acc_c = torch.full((B, Hkv, cap), -9.0, device="cuda")
+    o_s, o_c = np.full((B, Hkv, cap), 9.0), np.full((B, Hkv, cap), -9.0)
+    out = torch.zeros(B, Hq, d, device="cuda")
+    ws = csp.new_decode_step_workspace(p)
+    for i in range(steps):
+        rows = torch.tensor([[L0[b] + i + 1] * Hkv for b in range(B)], dtype=torch.int32)
+        for b in range(B):                           # the new token's K and V rows enter the cache first
+            kd[b, :, L0[b] + i] = k[b, :, L0[b] + i].cuda()
+            vd[b, :, L0[b] + i] = v[b, :, L0[b] + i].cuda()
+        first = i == steps - W
+        csp.decode_step(p, qs[i].cuda(), kd, vd, rows.cuda(), modd, new_label[i].cuda(), first, out, acc_s, acc_c, ws)
+        want = oracle.decode_step(po, qs[i], k, v, rows.numpy(), mod.numpy(), new_label[i].numpy(), o_s, o_c, first)
+        if i % 7 == 0 or i == steps - 1:
+            got = out.cpu().numpy().astype(np.float64)
+            tol = REL * np.abs(want) + ABS * float(v.float().abs().max())
+            assert (np.abs(got - want) <= tol).all(), f"step {i}: attention output off by {np.abs(got - want).max()}"
+    assert csp.device_status(ws) == 0
+    g_s, g_c = acc_s.cpu().numpy(), acc_c.cpu().numpy()
+    _score_tolerance_ok(g_s.reshape(B * Hkv, cap), o_s.reshape(B * Hkv, cap), "intra")
+    _score_tolerance_ok(g_c.reshape(B * Hkv, cap), o_c.reshape(B * Hkv, cap), "inter")
+
+    # from scratch on the final cache: the last W queries are the observation window
+    lens = torch.tensor([L0[b] + steps for b in range(B)], dtype=torch.int32)
+    R = W
+    q_win = qs[steps - W:].permute(1, 2, 0, 3).contiguous()                        # [B, Hq, W, d]
+    ps = csp.Params(B, Hq, Hkv, d, W, R, cap, cap)
+    ss = torch.zeros(B, Hkv, cap, device="cuda")
+    sc = torch.zeros(B, Hkv, cap, device="cuda")
+    wsp = csp.new_workspace(ps)
+    csp.score(ps, q_win.cuda(), kd, modd, lens.cuda(), ss, sc, wsp)
+    assert csp.device_status(wsp) == 0
+    for b in range(B):
+        N = int(lens[b]) - R
+        if N <= 0:
+            continue
+        _score_tolerance_ok(g_s[b, :, :N], ss[b, :, :N].cpu().numpy(), "carried vs from-scratch intra")
+        _score_tolerance_ok(g_c[b, :, :N], sc[b, :, :N].cpu().numpy(), "carried vs from-scratch inter")
+
+    # the prune that follows: Eq. 2-4 on the carried sums
+    bud = torch.tensor([[max(1, (L0[b] + steps) // 9), 5, 3, max(1, (L0[b] + steps) // 7)] for b in range(B)], dtype=torch.int32)
+    idx = torch.full((B, Hkv, cap), -1, dtype=torch.int32, device="cuda")
+    n_out = torch.zeros(B, Hkv, dtype=torch.int32, device="cuda")
+    csp.select(ps, acc_s, acc_c, modd, lens.cuda(), bud.cuda(), idx, n_out, wsp)
+    assert csp.device_status(wsp) & ~csp.DEV_K_CLAMPED == 0
+    pos = oracle.Params(B, Hq, Hkv, d, W, R, cap, cap, dtype=oracle.BF16)
+    i_ref, n_ref, _, _ = oracle.select(pos, g_s, g_c, mod.numpy(), lens.numpy(), bud.numpy())
+    np.testing.assert_array_equal(n_out.cpu().numpy(), n_ref)
+    for b in range(B):
+        for h in range(Hkv):
+            n = int(n_ref[b, h])
+            np.testing.assert_array_equal(idx[b, h, :n].cpu().numpy(), i_ref[b, h, :n])
+    k_out, v_out = torch.zeros_like(kd), torch.zeros_like(vd)
+    mod_out = torch.zeros_like(modd)
+    csp.compact(ps, kd, vd, modd, idx, n_out, k_out, v_out, mod_out)
+    for b in range(B):
+        for h in range(Hkv):
+            n = int(n_ref[b, h])
+            ii = i_ref[b, h, :n]
+            np.testing.assert_array_equal(bits(k_out[b, h, :n]), bits(k)[b, h][ii])
+            np.testing.assert_array_equal(bits(v_out[b, h, :n]), bits(v)[b, h][ii])
+            np.testing.assert_array_equal(mod_out[b, h, :n].cpu().numpy(), mod[b, h].numpy()[ii])
+
+
+def test_decode_step_rejects_bad_arguments(csp):
+    p = csp.Params(1, 2, 2, 128, 1, 0, 64, 64)
+    z = torch.zeros(1, 2, 64, 128, dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    rows = torch.zeros(1, 2, dtype=torch.int32, device="cuda")
+    mod = torch.zeros(1, 2, 64, dtype=torch.uint8, device="cuda")
+    lab = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    acc = torch.zeros(1, 2, 64, device="cuda")
+    out = torch.zeros(1, 2, 128, device="cuda")
+    small = csp.new_decode_workspace(p)              # the workspace of the plain decode call is too small
+    with pytest.raises(csp.CspError) as e:
+        csp.decode_step(p, q, z, z, rows, mod, lab, True, out, acc, acc.clone(), small)
+    assert e.value.code == csp.ERR_WORKSPACE
+    ws = csp.new_decode_step_workspace(p)
+    csp.decode_step(p, q, z, z, rows, mod, lab, True, out, acc, acc.clone(), ws)     # zero rows: zeros everywhere
+    assert csp.device_status(ws) == 0 and (out == 0).all() and (acc == 0).all()

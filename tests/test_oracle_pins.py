@@ -703,6 +703,85 @@ def test_decode_step_first_clears_the_unit_and_later_steps_add(oracle):
         np.testing.assert_allclose(acc_c[0, h, :r], before[0, h, :r], rtol=1e-15)
 
 
+# ---------------------------------------------------------------- Section 1: the distribution-gap diagnostic
+
+def test_js_divergence_closed_forms_and_library(oracle):
+    from scipy.spatial.distance import jensenshannon
+    a = np.array([5, 0, 3, 9, 0, 1], np.int64)
+    assert oracle.js_divergence(a, a) == 0.0
+    assert oracle.js_divergence(a, 7 * a) == 0.0                      # only the normalised shapes matter
+    b = np.array([0, 4, 0, 0, 2, 0], np.int64)                        # disjoint supports: ln 2
+    assert abs(oracle.js_divergence(a, b) - np.log(2.0)) < 1e-15
+    rng = np.random.RandomState(70)
+    for _ in range(5):
+        x, y = rng.randint(0, 50, 64).astype(np.int64), rng.randint(0, 50, 64).astype(np.int64)
+        want = jensenshannon(x / x.sum(), y / y.sum()) ** 2          # scipy returns the square root, natural log
+        assert abs(oracle.js_divergence(x, y) - want) < 1e-13
+        assert abs(oracle.js_divergence(x, y) - oracle.js_divergence(y, x)) < 1e-16
+    assert np.isnan(oracle.js_divergence(a, np.zeros(6, np.int64)))
+    # a worked case: P = (1, 0), Q = (1/2, 1/2): M = (3/4, 1/4)
+    want = 0.5 * np.log(1 / 0.75) + 0.5 * (0.5 * np.log(0.5 / 0.75) + 0.5 * np.log(0.5 / 0.25))
+    assert abs(oracle.js_divergence(np.array([2, 0]), np.array([3, 3])) - want) < 1e-15
+
+
+def _weights_per_head(q_full, k, n):
+    """Causal n-softmax matrix of every head (the full-matrix transcription, not averaged)."""
+    H, L, d = q_full.shape
+    A = np.zeros((H, L, L))
+    for h in range(H):
+        O = q_full[h] @ k.T / np.sqrt(d)
+        for i in range(L):
+            e = np.exp(O[i, :i + 1])
+            A[h, i, :i + 1] = e / (n + e.sum())
+    return A
+
+
+@pytest.mark.parametrize("seed,L,W,R,G,n", [(71, 40, 5, 7, 2, 1.0), (72, 33, 4, 4, 1, 0.0), (73, 25, 6, 2, 3, 4.0)])
+def test_weight_histogram_against_the_full_matrix(oracle, seed, L, W, R, G, n):
+    rng = np.random.RandomState(seed)
+    d = 4
+    q_full = (rng.randn(G, L, d) * 3).astype(np.float32)
+    k = rng.randn(L, d).astype(np.float32)
+    mod = (rng.rand(L) < 0.5).astype(np.uint8)
+    p = oracle.Params(1, G, 1, d, W, R, L, L, dtype=oracle.F32, n=n)
+    hist, near, js, js_all = oracle.weight_histogram(p, q_full[None, :, L - W:], k[None, None], mod[None],
+                                                     np.array([L], np.int32), near_eps=0.05)
+    A = _weights_per_head(q_full.astype(np.float64), k.astype(np.float64), n)
+    want = np.zeros((2, oracle.HIST_BINS), np.int64)
+    close = np.zeros((2, oracle.HIST_BINS), np.int64)
+    for g in range(G):
+        for i in range(L - W, L):
+            for t in range(min(L - R, i + 1)):
+                cls = 0 if mod[i] == mod[t] else 1
+                x = (np.log2(A[g, i, t]) - oracle.HIST_LO) / oracle.HIST_WIDTH
+                want[cls, int(np.clip(np.floor(x), 0, oracle.HIST_BINS - 1))] += 1
+                je = int(np.floor(x + 0.5))
+                if 1 <= je <= oracle.HIST_BINS - 1 and abs(x - je) * oracle.HIST_WIDTH <= 0.05:
+                    close[cls, je] += 1
+    np.testing.assert_array_equal(hist[0, 0], want)
+    np.testing.assert_array_equal(near[0, 0], close)
+    assert want.sum() == G * sum(min(L - R, i + 1) for i in range(L - W, L))
+    assert abs(js[0, 0] - oracle.js_divergence(want[0], want[1])) < 1e-15 and abs(js_all - js[0, 0]) < 1e-15
+
+
+def test_weight_histogram_zero_query_closed_form_and_pooling(oracle):
+    """q = 0: row w gives every key it sees 1 / (n + L - W + w + 1); with L = 20, W = 2, n = 1 those are 1/20 and
+    1/21, both in the bin that holds log2 in [-4.5, -4): bin 55.  Counts follow from the labels alone."""
+    L, W, R, G = 20, 2, 3, 2
+    mod = np.zeros((2, L), np.uint8)
+    mod[0, 3:9] = 1                                  # sequence 0: six visual candidates, text window
+    mod[1, :] = 1                                    # sequence 1: everything visual -> no inter pairs
+    p = oracle.Params(2, G, 1, 4, W, R, L, L, dtype=oracle.F32, n=1.0)
+    k = torch.randn(2, 1, L, 4, generator=torch.Generator().manual_seed(1))
+    hist, near, js, js_all = oracle.weight_histogram(p, torch.zeros(2, G, W, 4), k, mod, np.array([L, L], np.int32))
+    N = L - R
+    assert hist[0, 0, 0, 55] == G * W * (N - 6) and hist[0, 0, 1, 55] == G * W * 6
+    assert hist[1, 0, 0, 55] == G * W * N and hist[1, 0, 1].sum() == 0
+    assert hist.sum() == 2 * G * W * N
+    assert js[0, 0] == 0.0 and np.isnan(js[1, 0])    # same shape -> 0; an empty histogram -> undefined
+    assert js_all == 0.0                             # pooled over both units: both classes sit in the same bin
+
+
 def test_benchmark_shapes_match_their_description():
     c1 = synth.config(1)
     assert c1.seq_lens.tolist() == [4096] and c1.budgets.tolist() == [[304, 0, 0, 691]]
