@@ -174,8 +174,9 @@ class LayerBuffers:
 class Call:
     """One csp_prune_layer call of a step."""
 
-    def __init__(self, p, lb, mod, lens, bud, tot, layers):
+    def __init__(self, p, lb, mod, lens, bud, tot, layers, lse=None):
         self.p, self.lb, self.mod, self.lens, self.bud, self.tot, self.layers = p, lb, mod, lens, bud, tot, layers
+        self.lse = lse        # log of the window rows' exponential sums, if an upstream attention kernel supplies it
 
 
 def oracle_params(orc, cfg, batch, max_len, cap):
@@ -256,7 +257,7 @@ class PathBench:
     def prune(self, c: Call, w):
         lb = c.lb
         self.csp.prune_layer(c.p, lb.q, lb.k, lb.v, c.mod, c.lens, c.bud, lb.k_out, lb.v_out, lb.mod_out, lb.n_out, w,
-                             total_budget=c.tot)
+                             total_budget=c.tot, lse=c.lse)
 
     def capture(self, calls, n_chains, wss):
         """A CUDA graph of one step: chain c prunes calls c, c + n_chains, ... on its own stream."""
@@ -317,6 +318,25 @@ class PathBench:
         stream.synchronize()
         return k0.elapsed_time(k1) / reps
 
+    def ex2_rates(self):
+        """Exponentials per second of this GPU, measured once: on the special-function unit and through the FMA pipe."""
+        if getattr(self, "_ex2", None) is None:
+            csp, stream = self.csp, self.stream
+            sink = torch.zeros(2 * self.sms * 1024, device=self.dev)
+            res = {}
+            with torch.cuda.stream(stream):
+                for name, fma in (("special_function_unit", False), ("fma_pipe_two_wide", True)):
+                    csp.probe_ex2_rate(fma, 256, sink)
+                    stream.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    n = csp.probe_ex2_rate(fma, 4096, sink)
+                    e1.record(stream)
+                    stream.synchronize()
+                    res[name] = n / (e0.elapsed_time(e1) * 1e-3)
+            self._ex2 = res
+        return self._ex2
+
     # ---- one workload
     def measure(self, cfg, calls, n_chains, tokens_per_layer, n_layers, workload_name, launch_name, launch_tag,
                 labels_per_head=False, want_extras=True, lens_per_layer=None):
@@ -357,7 +377,7 @@ class PathBench:
 
             def score_all():
                 for c in calls:
-                    csp.score(c.p, c.lb.q, c.lb.k, c.mod, c.lens, c.lb.ss, c.lb.sc, ws)
+                    csp.score(c.p, c.lb.q, c.lb.k, c.mod, c.lens, c.lb.ss, c.lb.sc, ws, lse=c.lse)
 
             def select_all():
                 for c in calls:
@@ -391,16 +411,22 @@ class PathBench:
         # SMs: 16 ex2 per clock and SM on the special-function unit (the documented rate of sm_100) at the
         # maximum SM clock.
         if dominant == "score" and clocks and clocks.get("sm_max_mhz"):
-            ex2_peak = 16.0 * self.sms * clocks["sm_max_mhz"] * 1e6
-            n_exp = 2.0 * float(cfg.group * cfg.window * cfg.n_kv_heads) * float(np.asarray(lens, np.int64).sum()) * lpl
+            derived = 16.0 * self.sms * clocks["sm_max_mhz"] * 1e6
+            probe = self.ex2_rates()
+            ex2_peak = probe["special_function_unit"] if probe else derived
+            passes = 1.0 if calls[0].lse is not None else 2.0       # a supplied LSE removes the pass for the row sums
+            n_exp = passes * float(cfg.group * cfg.window * cfg.n_kv_heads) * float(np.asarray(lens, np.int64).sum()) * lpl
             if n_exp / ex2_peak > ab_launch["score"] / (peak * 1e9):
                 ex2_rate = n_exp / (per["score"] * 1e-3)
                 roofline = {"bound": "alu", "kernel": "score", "achieved": ex2_rate / 1e12, "peak": ex2_peak / 1e12,
                             "unit": "T ex2/s", "frac": ex2_rate / ex2_peak, "traffic": traffic,
                             "traffic_source": traffic_src,
-                            "peak_kind": "derived: 16 ex2 per clock and SM x SM count x maximum SM clock",
+                            "peak_kind": ("measured: csp_probe_ex2_rate, ex2.approx.ftz.f32 in registers only" if probe else
+                                          "derived: 16 ex2 per clock and SM x SM count x maximum SM clock"),
+                            "peak_derived": derived / 1e12, "probe": probe,
                             "exponentials_per_launch": n_exp,
-                            "exponentials_counted": "2 G W per key: one for the row sums, one for the weights",
+                            "exponentials_counted": ("G W per key: the weights (row sums supplied)" if passes == 1.0 else
+                                                     "2 G W per key: one for the row sums, one for the weights"),
                             "us_per_launch": per["score"] * 1e3, "hbm": roofline}
         path = {"algorithmic_bytes_per_layer": ab["total"], "us_per_layer": ms_step * 1e3 / n_layers,
                 "achieved_gbs": ab["total"] / (ms_step * 1e-3 / n_layers) / 1e9,
@@ -513,7 +539,7 @@ class PathBench:
         return base, parity
 
 
-def make_calls(csp, cfg, dev, fold, n_buf, n_layers):
+def make_calls(csp, cfg, dev, fold, n_buf, n_layers, with_lse=False):
     """The library calls of one step.  fold: one call for all layers (layer axis on the batch axis); else one
     call per layer over n_buf distinct layer buffers (views into one folded allocation)."""
     cap = cfg.out_capacity()
@@ -529,8 +555,31 @@ def make_calls(csp, cfg, dev, fold, n_buf, n_layers):
     fold_call = Call(pf, folded, mod.repeat(n_buf, 1), lens.repeat(n_buf), bud.repeat(n_buf, 1),
                      None if tot is None else tot.repeat(n_buf), n_buf)
     views = [folded.layer_view(i, cfg.batch) for i in range(n_buf)]
-    layer_calls = [Call(p, views[i % n_buf], mod, lens, bud, tot, 1) for i in range(n_layers)]
+    lse_views = [None] * n_buf
+    if with_lse:
+        fold_call.lse = window_lse(cfg, folded.q, folded.k, lens.repeat(n_buf))
+        lse_views = [fold_call.lse[i * cfg.batch:(i + 1) * cfg.batch] for i in range(n_buf)]
+    layer_calls = [Call(p, views[i % n_buf], mod, lens, bud, tot, 1, lse_views[i % n_buf]) for i in range(n_layers)]
     return p, fold_call, layer_calls, (mod, lens, bud, tot)
+
+
+def window_lse(cfg, q, k, lens):
+    """Natural log of sum_t e^{o_t} of every window row over the keys it sees: what the attention kernel that
+    produced the window's outputs already holds.  Input preparation (plain torch, untimed), not part of the path."""
+    B, Hq, W, d = q.shape
+    G = cfg.group
+    out = torch.empty(B, Hq, W, dtype=torch.float32, device=q.device)
+    lens_h = lens.cpu().numpy()
+    for b in range(B):
+        L = int(lens_h[b])
+        kk = k[b, :, :L].float()                                        # [Hkv, L, d]
+        qq = q[b].float().view(cfg.n_kv_heads, G * W, d)                # heads of a group share their KV head
+        o = torch.bmm(qq, kk.transpose(1, 2)) / float(np.sqrt(d))       # [Hkv, G W, L]
+        pos = (L - W + torch.arange(W, device=q.device)).repeat(G)      # position of each window row
+        hidden = torch.arange(L, device=q.device)[None, :] > pos[:, None]
+        o.masked_fill_(hidden[None], float("-inf"))
+        out[b] = torch.logsumexp(o, dim=2).view(Hq, W)
+    return out
 
 
 def append_round(csp, cfg, dev, prev_calls, n_buf, gen, totals, budgets):
@@ -597,8 +646,9 @@ def run_config(pb: PathBench, csp, args, config_index, rank, world, dev, budget_
     if huge and args.layers <= 0:
         n_buf = 4
     fold = args.fold_layers and n_buf == n_layers
-    p, fold_call, layer_calls, (mod, lens, bud, tot) = make_calls(csp, cfg, dev, fold, n_buf, n_layers)
-    wl = f"configs{config_index}" + (f"_{budget_pct or args.budget_pct}pct" if config_index == 4 else "")
+    p, fold_call, layer_calls, (mod, lens, bud, tot) = make_calls(csp, cfg, dev, fold, n_buf, n_layers, args.with_lse)
+    wl = f"configs{config_index}" + (f"_{budget_pct or args.budget_pct}pct" if config_index == 4 else "") + \
+        ("_lse" if args.with_lse else "")
     n_chains = max(1, min(args.streams, n_layers))
     per_layer_name = f"cuda graph of one step, {n_chains} concurrent chains of one csp_prune_layer call per layer"
     fold_name = "one csp_prune_layer call for all layers (layer axis folded into the batch axis)"
@@ -624,10 +674,10 @@ def run_config(pb: PathBench, csp, args, config_index, rank, world, dev, budget_
         ws1 = csp.new_workspace(first.p, dev)
         csp.prune_layer(first.p, first.lb.q, first.lb.k, first.lb.v, first.mod, first.lens, first.bud, first.lb.k_out,
                         first.lb.v_out, first.lb.mod_out, first.lb.n_out, ws1, total_budget=first.tot,
-                        score_self=first.lb.ss, score_cross=first.lb.sc, keep_idx=first.lb.idx)
+                        score_self=first.lb.ss, score_cross=first.lb.sc, keep_idx=first.lb.idx, lse=first.lse)
         pb.stream.synchronize()
     e2e = None
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and not args.with_lse:
         e2e = pb.e2e(cfg, p, [c.lb for c in layer_calls[:min(n_buf, 4 if not huge else 2)]], mod, lens, bud, tot, n_layers,
                      sum_l, args.e2e_steps)
     cpu_baseline = parity = None
@@ -635,6 +685,8 @@ def run_config(pb: PathBench, csp, args, config_index, rank, world, dev, budget_
         cpu_baseline, parity = pb.cpu_baseline(cfg, first, cfg.batch, cfg.max_len, p.out_capacity, sum_l,
                                                seconds=args.cpu_seconds)
     lines.append(bench_line(cfg, args, world, config_index, m, e2e, cpu_baseline, parity, n_layers, n_buf, sum_l, extra))
+    if args.with_lse:
+        lines[-1]["config"]["workload"] += ", log-sum-exp of the window rows supplied by the caller (no pass for the row sums)"
 
     # ---- the serving shape's re-prune rounds: 64 decode tokens appended to every head's compacted cache, four times
     if config_index == 4 and args.rounds > 0 and not default_line:
@@ -905,6 +957,9 @@ def main():
                     help="time the step after the pruning pass instead: n-softmax decode attention over the pruned caches")
     ap.add_argument("--incremental", action="store_true",
                     help="a re-prune round of configs[4] from the sums carried by csp_decode_step, against the full rescan")
+    ap.add_argument("--with-lse", action="store_true",
+                    help="supply the log-sum-exp of the window rows (as an upstream attention kernel would): csp_score then "
+                         "skips the pass that computes the row sums; a separate, labelled line")
     ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
     ap.add_argument("--rounds", type=int, default=4, help="re-prune rounds of configs[4] under --all-configs")
     ap.add_argument("--all-configs", action="store_true",

@@ -203,6 +203,31 @@ csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_
                            const int32_t* n_rows, float* out,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * The measurement behind the method (Section 1, the figure on the gap between self- and cross-attention): the
+ * window's attention weights, per query head and not averaged, collected in two histograms, one for pairs whose
+ * query and key carry the same modality label (intra) and one for the others (inter), and the Jensen-Shannon
+ * divergence between the two.  Which weights: A[g,w,t] of Eq. 7 for window row w and every candidate key
+ * t < L_b - R that the row sees, i.e. exactly the entries that Eq. 1 sums.  Bin j of CSP_HIST_BINS covers
+ * log2(A) in [CSP_HIST_LO + j CSP_HIST_WIDTH, CSP_HIST_LO + (j + 1) CSP_HIST_WIDTH); smaller weights (and zeros)
+ * count in bin 0.  The paper shows a kernel density estimate; the half-octave bins are this library's choice.
+ *   hist   [B, H_kv, 2, CSP_HIST_BINS] uint32 (0: intra, 1: inter); cleared and filled by the call
+ *   js_or_null     [B, H_kv] fp32: 1/2 KL(P || M) + 1/2 KL(Q || M) in nats, M = (P + Q) / 2, P and Q the two
+ *                  histograms of the unit normalised to sum 1; NaN when either is empty
+ *   js_all_or_null [1] fp32: the same for the histograms summed over all units of the call (one layer's figure
+ *                  when the call is one layer)
+ * Other arguments as for csp_score; workspace of csp_workspace_bytes (it also receives the scores).  bf16 caches,
+ * CSP_HEADS_PER_KV only.  A diagnostic, several times slower than csp_score: every weight is binned.
+ */
+#define CSP_HIST_BINS 64
+#define CSP_HIST_LO (-32.0f)
+#define CSP_HIST_WIDTH 0.5f
+csp_status csp_weight_histogram(const csp_params* p, csp_tensor q_win, csp_tensor k,
+                                const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                                const int32_t* seq_lens, const float* lse_or_null,
+                                uint32_t* hist, float* js_or_null, float* js_all_or_null,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Bytes of scratch that csp_decode_step needs: those of csp_decode_attn plus one row of logits per query head
  * and unit.  The first 256 bytes must be zero before first use (csp_workspace_reset). */
 size_t csp_decode_step_workspace_bytes(const csp_params* p);
@@ -283,6 +308,19 @@ csp_status csp_prune_layer_static(const csp_params* p, csp_tensor q_win, csp_ten
 
 /* Size in bytes of the built-in scratch array used by csp_prune_layer_static. */
 size_t csp_static_workspace_limit(void);
+
+/*
+ * No counterpart in the paper: a measuring aid.  With G >= 3 query heads per KV head the scoring kernel (Eq. 5,
+ * Eq. 7) is bound by exponentials, not by memory, so its roofline needs this GPU's exponential rate.  Enqueues a
+ * registers-only kernel (two CTAs of 1024 threads per SM, eight independent chains per thread) that evaluates
+ * *exponentials_host_out base-2 exponentials in total; the caller times it with events on the stream.
+ *   fma_pipe    0: ex2.approx.ftz.f32 on the special-function unit (what the scoring kernels issue);
+ *               1: the two-wide FMA-pipe evaluation the G >= 3 kernels use for one pair in eight
+ *   iterations  1 .. 2^20 loop trips (8 exponentials per thread and trip)
+ *   sink        device array that receives one float per thread (keeps the loop alive); may be NULL
+ */
+csp_status csp_probe_ex2_rate(int32_t fma_pipe, int32_t iterations, float* sink, size_t sink_elems,
+                              int64_t* exponentials_host_out, void* cuda_stream);
 
 /* Waits for the stream, copies the status word to *host_out (may be NULL), clears it, and returns
  * CSP_ERR_TIMEOUT if CSP_DEV_TIMEOUT was set, else CSP_OK. */

@@ -26,7 +26,9 @@ DEV_K_CLAMPED, DEV_CAPACITY, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8
 EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_select", "csp_compact",
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
            "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
-           "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step")
+           "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step",
+           "csp_weight_histogram", "csp_probe_ex2_rate")
+HIST_BINS, HIST_LO, HIST_WIDTH = 64, -32.0, 0.5
 
 
 class CspError(RuntimeError):
@@ -119,6 +121,10 @@ def lib() -> C.CDLL:
         l.csp_decode_step_workspace_bytes.argtypes = [P]
         l.csp_decode_step.restype = C.c_int
         l.csp_decode_step.argtypes = [P, CTensor, CTensor, CTensor, vp, vp, i64, i64, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
+        l.csp_probe_ex2_rate.restype = C.c_int
+        l.csp_probe_ex2_rate.argtypes = [C.c_int32, C.c_int32, vp, sz, C.POINTER(C.c_int64), vp]
+        l.csp_weight_histogram.restype = C.c_int
+        l.csp_weight_histogram.argtypes = [P, CTensor, CTensor, vp, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         l.csp_device_status.restype = C.c_int
         l.csp_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         l.csp_status_string.restype = C.c_char_p
@@ -226,6 +232,24 @@ def score(p: Params, q_win, k, modality, seq_lens, score_self, score_cross, ws, 
     _check(lib().csp_score(C.byref(cp), tensor4(q_win), tensor4(k), _ptr(modality), sb, sh, _ptr(seq_lens),
                            _ptr(lse), _ptr(score_self), _ptr(score_cross), _ptr(ws), ws.numel(), _stream()),
            "csp_score")
+
+
+def weight_histogram(p: Params, q_win, k, modality, seq_lens, hist, ws, js=None, js_all=None, lse=None):
+    """hist uint32-as-int32 [B, Hkv, 2, HIST_BINS]; js fp32 [B, Hkv]; js_all fp32 [1]."""
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    assert hist.is_contiguous() and hist.element_size() == 4
+    _check(lib().csp_weight_histogram(C.byref(cp), tensor4(q_win), tensor4(k), _ptr(modality), sb, sh, _ptr(seq_lens),
+                                      _ptr(lse), _ptr(hist), _ptr(js), _ptr(js_all), _ptr(ws), ws.numel(), _stream()),
+           "csp_weight_histogram")
+
+
+def probe_ex2_rate(fma_pipe: bool, iterations: int, sink: Optional[torch.Tensor] = None) -> int:
+    """Enqueues the exponential-throughput probe on the current stream; returns how many exponentials it evaluates."""
+    n = C.c_int64(0)
+    _check(lib().csp_probe_ex2_rate(int(bool(fma_pipe)), int(iterations), _ptr(sink), 0 if sink is None else sink.numel(),
+                                    C.byref(n), _stream()), "csp_probe_ex2_rate")
+    return int(n.value)
 
 
 def select(p: Params, score_self, score_cross, modality, seq_lens, budgets, keep_idx, n_out, ws,

@@ -54,7 +54,7 @@ csp_status check_workspace(const csp_params& p, void* ws, size_t bytes) {
 
 csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const uint8_t* modality,
                     int64_t msb, int64_t msh, const int32_t* seq_lens, const float* lse, float* score_self,
-                    float* score_cross, void* ws, cudaStream_t stream) {
+                    float* score_cross, void* ws, cudaStream_t stream, uint32_t* hist = nullptr) {
     if (p.batch == 0 || p.max_len == 0) return CSP_OK;
     const WorkspaceLayout wl = workspace_layout(p);
     const bool mean_all = p.head_reduce == CSP_HEADS_MEAN_ALL && p.n_kv_heads > 1;
@@ -68,6 +68,7 @@ csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& 
     a.status = static_cast<int32_t*>(ws);
     a.order_buf = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + wl.order);
     a.order = nullptr;
+    a.hist = hist;
     a.n_kv_heads = p.n_kv_heads; a.group = p.n_q_heads / p.n_kv_heads;
     a.window = p.window; a.recent = p.recent; a.max_len = p.max_len;
     a.n = p.n;
@@ -363,6 +364,47 @@ csp_status csp_decode_attn(const csp_params* p, csp_tensor q, csp_tensor k, csp_
         return CSP_ERR_WORKSPACE;
     if ((st = check_arch()) != CSP_OK) return st;
     return launch_decode_attn(*p, q, k, v, n_rows, out, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+csp_status csp_weight_histogram(const csp_params* p, csp_tensor q_win, csp_tensor k, const uint8_t* modality,
+                                int64_t mod_stride_b, int64_t mod_stride_h, const int32_t* seq_lens,
+                                const float* lse_or_null, uint32_t* hist, float* js_or_null, float* js_all_or_null,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!modality || !seq_lens || !hist || !q_win.ptr || !k.ptr) return CSP_ERR_INVALID_ARG;
+    if (p->dtype != CSP_BF16 || p->head_reduce != CSP_HEADS_PER_KV) return CSP_ERR_UNSUPPORTED;
+    if (!tensor_ok(*p, q_win) || !tensor_ok(*p, k)) return CSP_ERR_UNSUPPORTED;
+    if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
+    if ((st = check_arch()) != CSP_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t units = size_t(p->batch) * p->n_kv_heads;
+    if (units == 0) return CSP_OK;
+    if (cudaMemsetAsync(hist, 0, units * 2 * CSP_HIST_BINS * sizeof(uint32_t), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return CSP_ERR_CUDA;
+    }
+    // the scores themselves are a by-product here: they land in the workspace
+    const WorkspaceLayout wl = workspace_layout(*p);
+    char* ws = static_cast<char*>(workspace);
+    if (p->max_len > 0) {
+        st = do_score(*p, q_win, k, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null,
+                      reinterpret_cast<float*>(ws + wl.score_self), reinterpret_cast<float*>(ws + wl.score_cross),
+                      workspace, stream, hist);
+        if (st != CSP_OK) return st;
+    }
+    return launch_hist_js(*p, hist, js_or_null, js_all_or_null, stream);
+}
+
+csp_status csp_probe_ex2_rate(int32_t fma_pipe, int32_t iterations, float* sink, size_t sink_elems,
+                              int64_t* exponentials_host_out, void* cuda_stream) {
+    if (iterations <= 0 || iterations > (1 << 20) || !exponentials_host_out) return CSP_ERR_INVALID_ARG;
+    csp_status st = check_arch();
+    if (st != CSP_OK) return st;
+    long long n = 0;
+    st = launch_ex2_probe(fma_pipe ? 1 : 0, iterations, sink, sink ? sink_elems : 0, &n, static_cast<cudaStream_t>(cuda_stream));
+    *exponentials_host_out = n;
+    return st;
 }
 
 size_t csp_decode_step_workspace_bytes(const csp_params* p) {

@@ -44,7 +44,6 @@ struct DecodeArgs {
     // csp_decode_step only: the step's logits are kept so that its n-softmax weights can be added to the running
     // intra / inter sums of Eq. 1 once the row's normaliser is known
     float* logits;                                 // [units, G, capacity]: o scale log2(e), or null
-    float* rowstat;                                // [units, G, 2]: reference exponent m, weight 1 / (G (n 2^-m + l))
     const uint8_t* modality; int64_t mod_sb, mod_sh;
     const uint8_t* query_label;                    // [B]
     float* acc_self; float* acc_cross;             // [units, capacity]
@@ -337,10 +336,6 @@ __global__ void decode_merge_kernel(const DecodeArgs a) {
     float l = 0.f;
     for (int s = 0; s < used; ++s) l += part[s * stride + D + 1] * ex2f(part[s * stride + D] - m);
     const float denom = a.n * ex2f(-m) + l;
-    if (a.rowstat && threadIdx.x == 0) {
-        a.rowstat[(int64_t(u) * a.group + g) * 2] = m;
-        a.rowstat[(int64_t(u) * a.group + g) * 2 + 1] = (used > 0 && denom > 0.f) ? 1.0f / (float(a.group) * denom) : 0.f;
-    }
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
         float v = 0.f;
         for (int s = 0; s < used; ++s) v += part[s * stride + c] * ex2f(part[s * stride + D] - m);
@@ -348,30 +343,55 @@ __global__ void decode_merge_kernel(const DecodeArgs a) {
     }
 }
 
-// One query row of Eq. 1: the step's n-softmax weights, averaged over the query heads of the KV group, are added to
-// the intra sum of the cached rows that carry the query's label and to the inter sum of the others.  On the first
-// step of a window every slot of the unit is (over)written, so rows appended later start from zero.
-__global__ void decode_accumulate_kernel(const DecodeArgs a) {
-    const int u = blockIdx.y, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= a.capacity) return;
+// csp_decode_step: the merge of decode_merge_kernel for all query heads of one unit, and then one query row of
+// Eq. 1: the step's n-softmax weights, averaged over the query heads of the KV group, are added to the intra sum of
+// the cached rows that carry the query's label and to the inter sum of the others.  On the first step of a window
+// every slot of the unit is (over)written, so rows appended later start from zero.  One block per unit: the
+// normalisers stay in shared memory, the logits are read once.
+constexpr int kStepThreads = 256;
+__global__ void __launch_bounds__(kStepThreads) decode_merge_accumulate_kernel(const DecodeArgs a) {
+    __shared__ float ref[8], wgt[8];                 // per query head: reference exponent, 1 / (G (n 2^-m + l))
+    const int u = blockIdx.x, b = u / a.n_kv_heads, h = u % a.n_kv_heads;
+    const int D = a.head_dim, G = a.group;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.next_item = 0;     // the work counter is zero again for the next call
     int rows = a.n_rows[u];
+    if ((rows < 0 || rows > a.capacity) && threadIdx.x == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
     rows = rows < 0 ? 0 : (rows > a.capacity ? a.capacity : rows);
+    const int tiles = (rows + kDecTile - 1) / kDecTile;
+    const int used = (tiles + a.tiles_per_split - 1) / a.tiles_per_split;
+    const int64_t stride = int64_t(G) * (D + 2);
+    for (int g = 0; g < G; ++g) {
+        float* const o = a.out + (int64_t(b) * a.n_kv_heads * G + h * G + g) * D;
+        const float* const part = a.partial + (int64_t(u) * a.splits * G + g) * (D + 2);
+        float m = kNeg;
+        for (int s = 0; s < used; ++s) m = fmaxf(m, part[s * stride + D]);
+        float l = 0.f;
+        for (int s = 0; s < used; ++s) l += part[s * stride + D + 1] * ex2f(part[s * stride + D] - m);
+        const float denom = a.n * ex2f(-m) + l;
+        const bool ok = used > 0 && denom > 0.f;
+        if (threadIdx.x == 0) { ref[g] = m; wgt[g] = ok ? 1.0f / (float(G) * denom) : 0.f; }
+        for (int c = threadIdx.x; c < D; c += kStepThreads) {
+            float v = 0.f;
+            for (int s = 0; s < used; ++s) v += part[s * stride + c] * ex2f(part[s * stride + D] - m);
+            o[c] = ok ? v / denom : 0.f;
+        }
+    }
+    __syncthreads();
     float* const as = a.acc_self + int64_t(u) * a.capacity;
     float* const ac = a.acc_cross + int64_t(u) * a.capacity;
-    if (t >= rows) {
-        if (a.first_step) { as[t] = 0.f; ac[t] = 0.f; }
-        return;
+    const uint8_t* const mod = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
+    const uint32_t qlab = a.query_label[b];
+    const float* const lg = a.logits + int64_t(u) * G * a.capacity;
+    const int end = a.first_step ? a.capacity : rows;
+    for (int t = threadIdx.x; t < end; t += kStepThreads) {
+        if (t >= rows) { as[t] = 0.f; ac[t] = 0.f; continue; }
+        float w = 0.f;
+        for (int g = 0; g < G; ++g) w += ex2f(lg[int64_t(g) * a.capacity + t] - ref[g]) * wgt[g];
+        const bool same = mod[t] == qlab;
+        const float s0 = a.first_step ? 0.f : as[t], c0 = a.first_step ? 0.f : ac[t];
+        as[t] = s0 + (same ? w : 0.f);
+        ac[t] = c0 + (same ? 0.f : w);
     }
-    float w = 0.f;
-    for (int g = 0; g < a.group; ++g) {
-        const float m = a.rowstat[(int64_t(u) * a.group + g) * 2], f = a.rowstat[(int64_t(u) * a.group + g) * 2 + 1];
-        w += ex2f(a.logits[(int64_t(u) * a.group + g) * a.capacity + t] - m) * f;
-    }
-    const bool same = a.modality[int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh + t] == a.query_label[b];
-    const float s0 = a.first_step ? 0.f : as[t], c0 = a.first_step ? 0.f : ac[t];
-    as[t] = s0 + (same ? w : 0.f);
-    ac[t] = c0 + (same ? 0.f : w);
 }
 
 }  // namespace
@@ -395,7 +415,7 @@ size_t decode_workspace_bytes(const csp_params& p) {
 size_t decode_step_workspace_bytes(const csp_params& p) {
     const size_t units = size_t(p.batch) * size_t(p.n_kv_heads);
     const size_t G = size_t(p.n_q_heads / p.n_kv_heads);
-    return decode_workspace_bytes(p) + round256(units * G * size_t(p.out_capacity) * 4) + round256(units * G * 8);
+    return decode_workspace_bytes(p) + round256(units * G * size_t(p.out_capacity) * 4);
 }
 
 csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
@@ -404,13 +424,10 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     DecodeArgs a;
-    a.logits = nullptr; a.rowstat = nullptr; a.modality = nullptr; a.mod_sb = a.mod_sh = 0; a.query_label = nullptr;
+    a.logits = nullptr; a.modality = nullptr; a.mod_sb = a.mod_sh = 0; a.query_label = nullptr;
     a.acc_self = a.acc_cross = nullptr; a.first_step = 0;
     if (step) {
-        char* const extra = static_cast<char*>(ws) + decode_workspace_bytes(p);
-        a.logits = reinterpret_cast<float*>(extra);
-        a.rowstat = reinterpret_cast<float*>(extra + round256(size_t(units) * (p.n_q_heads / p.n_kv_heads) *
-                                                              size_t(p.out_capacity) * 4));
+        a.logits = reinterpret_cast<float*>(static_cast<char*>(ws) + decode_workspace_bytes(p));
         a.modality = step->modality; a.mod_sb = step->mod_sb; a.mod_sh = step->mod_sh;
         a.query_label = step->query_label; a.acc_self = step->acc_self; a.acc_cross = step->acc_cross;
         a.first_step = step->first_step;
@@ -444,13 +461,9 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
         kern<<<n_items < sms ? n_items : sms, kDecThreads, smem, s>>>(tk, tv, a, n_items);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
     }
-    decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
-    if (step && p.out_capacity > 0) {
-        decode_accumulate_kernel<<<dim3((p.out_capacity + 255) / 256, units), 256, 0, s>>>(a);
-        if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
-    }
-    return CSP_OK;
+    if (step) decode_merge_accumulate_kernel<<<units, kStepThreads, 0, s>>>(a);
+    else decode_merge_kernel<<<units * a.group, 128, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
 }
 
 }  // namespace csp

@@ -81,6 +81,7 @@ struct ScoreArgs {
     const int32_t* order;                            // null, or the sequences by descending length
     int32_t n_kv_heads, group, window, recent, max_len;
     float n, scale_log2, weight;                     // weight = 1/G or 1/Hq
+    uint32_t* hist;                                  // null, or [B, Hkv, 2, CSP_HIST_BINS] counts to add to
 };
 
 struct SelectArgs {
@@ -130,6 +131,8 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tenso
 csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s);
 csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
                                 bool* taken);
+csp_status launch_ex2_probe(int fma_pipe, int iters, float* sink, size_t sink_elems, long long* n_exp, cudaStream_t s);
+csp_status launch_hist_js(const csp_params& p, const uint32_t* hist, float* js, float* js_all, cudaStream_t s);
 csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,
                             float* score_self, float* score_cross, const int32_t* seq_lens,
                             cudaStream_t s);

@@ -431,6 +431,51 @@ __global__ void head_mean_kernel(const float* __restrict__ part_self, const floa
     }
 }
 
+// Jensen-Shannon divergence (nats) between the intra and the inter histogram of every unit (blocks 0 .. units-1)
+// and of their sums over all units (block `units`): 1/2 KL(P || M) + 1/2 KL(Q || M), M = (P + Q) / 2, with P and Q
+// normalised to sum 1 and 0 log 0 = 0; NaN when either histogram is empty.  One thread per bin.
+__global__ void __launch_bounds__(CSP_HIST_BINS) hist_js_kernel(const uint32_t* __restrict__ hist, int units,
+                                                                float* __restrict__ js, float* __restrict__ js_all) {
+    constexpr int NB = CSP_HIST_BINS;
+    __shared__ double red[2][NB];
+    const int j = threadIdx.x, u = blockIdx.x;
+    const bool pooled = u == units;
+    if ((pooled && !js_all) || (!pooled && !js)) return;
+    double cp = 0.0, cq = 0.0;
+    if (pooled) {
+        for (int v = 0; v < units; ++v) {
+            cp += double(hist[(int64_t(v) * 2) * NB + j]);
+            cq += double(hist[(int64_t(v) * 2 + 1) * NB + j]);
+        }
+    } else {
+        cp = double(hist[(int64_t(u) * 2) * NB + j]);
+        cq = double(hist[(int64_t(u) * 2 + 1) * NB + j]);
+    }
+    auto block_sums = [&](double x, double y, double& sx, double& sy) {     // fixed-order tree over the bins
+        red[0][j] = x; red[1][j] = y;
+        __syncthreads();
+        for (int d = NB / 2; d > 0; d >>= 1) {
+            if (j < d) { red[0][j] += red[0][j + d]; red[1][j] += red[1][j + d]; }
+            __syncthreads();
+        }
+        sx = red[0][0]; sy = red[1][0];
+        __syncthreads();
+    };
+    double sp, sq;
+    block_sums(cp, cq, sp, sq);
+    double term = 0.0, unused = 0.0, total, dummy;
+    if (sp > 0.0 && sq > 0.0) {
+        const double pj = cp / sp, qj = cq / sq, mj = 0.5 * (pj + qj);
+        if (pj > 0.0) term += 0.5 * pj * log(pj / mj);
+        if (qj > 0.0) term += 0.5 * qj * log(qj / mj);
+    }
+    block_sums(term, unused, total, dummy);
+    if (j == 0) {
+        const float r = (sp > 0.0 && sq > 0.0) ? float(total) : __int_as_float(0x7fc00000);
+        if (pooled) *js_all = r; else js[u] = r;
+    }
+}
+
 // ---- host side --------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -579,6 +624,13 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_te
     const csp_status ps = launch_score_persist(p, a, tmap, s, &taken);
     if (ps != CSP_OK || taken) return ps;
     return launch_score_tc(p, a, tmap, s);
+}
+
+csp_status launch_hist_js(const csp_params& p, const uint32_t* hist, float* js, float* js_all, cudaStream_t s) {
+    const int units = p.batch * p.n_kv_heads;
+    if (!js && !js_all) return CSP_OK;
+    hist_js_kernel<<<units + 1, CSP_HIST_BINS, 0, s>>>(hist, units, js, js_all);
+    return cudaGetLastError() == cudaSuccess ? CSP_OK : CSP_ERR_CUDA;
 }
 
 csp_status launch_head_mean(const csp_params& p, const float* part_self, const float* part_cross,

@@ -519,7 +519,7 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
 csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
                                 bool* taken) {
     *taken = false;
-    if (a.group != 1 || a.lse != nullptr) return CSP_OK;
+    if (a.group != 1 || a.lse != nullptr || a.hist != nullptr) return CSP_OK;
     const int row_bytes = p.head_dim * 2;
     if (row_bytes != 128 && row_bytes != 256) return CSP_OK;
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;

@@ -57,9 +57,10 @@ template <int G> struct TmemPlan {
 };
 
 struct TcSmemPlan {   // byte offsets from the 1024-aligned base
-    uint32_t q, wstats, cstats, cvec, xchg, dq_mask, dq_val, bars, misc, total;
+    uint32_t q, wstats, cstats, cvec, xchg, dq_mask, dq_val, bars, misc, hist, total;
 };
-__host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
+constexpr int kHistBins = CSP_HIST_BINS;
+__host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages, bool with_hist) {
     TcSmemPlan s;
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
     s.q = off;        off += uint32_t(nh) * uint32_t(g) * 32u * 128u;
@@ -71,11 +72,14 @@ __host__ __device__ inline TcSmemPlan tc_smem_plan(int nh, int g, int stages) {
     s.dq_val = off;   off += 32u * 4u;
     s.bars = off;     off += (2u * kMaxStages + 2u * kMaxTmemBufs + 1u) * 8u;
     s.misc = off;     off += 16u;                       // tmem base, abort flag, n distinct query labels
+    s.hist = off;     off += with_hist ? 16u * 2u * uint32_t(kHistBins) * 4u : 0u;   // [epilogue warp][intra, inter][bin]
     s.total = off;
     return s;
 }
 
-template <int NH, int G>
+// kHist: the distribution diagnostic (csp_weight_histogram) rides on pass 2; a separate instantiation, so that
+// the scoring kernels proper carry none of its code
+template <int NH, int G, bool kHist>
 __global__ void __launch_bounds__(EpiPlan<G>::kThreads, (G == 1 && NH <= 2) ? 2 : 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, const int n_stages,
                 const int tmem_cols) {
@@ -92,7 +96,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const TcSmemPlan sp = tc_smem_plan(NH, G, n_stages);
+    constexpr bool want_hist = kHist;
+    const TcSmemPlan sp = tc_smem_plan(NH, G, n_stages, want_hist);
     const uint32_t q_s = base + sp.q;
     float2* const wstats = reinterpret_cast<float2*>(base_ptr + sp.wstats);
     float2* const cstats = reinterpret_cast<float2*>(base_ptr + sp.cstats);
@@ -258,6 +263,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
 
         const float scale2 = a.scale_log2;
         const int first_masked_key = L - W;       // keys beyond this may be hidden from some window row
+        // histogram of log2(weight) per query head: the exponent of pass 2 is log2(weight x mean factor)
+        uint32_t* const whist = reinterpret_cast<uint32_t*>(base_ptr + sp.hist) + warp * 2 * kHistBins;
+        const float hist_shift = want_hist ? -lg2f(a.weight) - CSP_HIST_LO : 0.f;
+        if (want_hist)
+            for (int j = lane; j < 2 * kHistBins; j += 32) whist[j] = 0u;
 
         // ---------------------------------- pass 1 ----------------------------------
         constexpr int NB = EP::kBlocks;
@@ -371,6 +381,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // weights of 16 columns: cur = logits, cv = their additive constants, as/ac = which columns count
             auto chunk = [&](const uint32_t (&cur)[16], const float* cvp, uint32_t as, uint32_t ac) {
                 const float4* cv = reinterpret_cast<const float4*>(cvp);
+                if (want_hist) {
+                    // one count per (query head, window row, key) the scores take in: its class is the sum it goes
+                    // to, its bin the half-octave of log2(weight).  Lanes with the same (class, bin) are counted
+                    // together, one shared-memory add per distinct value.
+#pragma unroll 1
+                    for (int j = 0; j < 16; ++j) {
+                        const bool counted = t < N && (((as | ac) >> j) & 1u);
+                        const float e = (fmaf(__uint_as_float(cur[j]), scale2, cvp[j]) + hist_shift) * (1.0f / CSP_HIST_WIDTH);
+                        const int bin = min(max(int(floorf(fmaxf(e, 0.f))), 0), kHistBins - 1);
+                        const uint32_t key = counted ? uint32_t(((ac >> j) & 1u) * kHistBins + bin) : 0xFFFFu;
+                        const uint32_t peers = __match_any_sync(0xffffffffu, key);
+                        if (counted && lane == __ffs(peers) - 1) atomicAdd(&whist[key], uint32_t(__popc(peers)));
+                    }
+                }
 #pragma unroll
                 for (int j4 = 0; j4 < 4; ++j4) {
                     const float4 cc = cv[j4];
@@ -387,7 +411,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             // Common case: every window query carries the same label and no column of this tile is hidden.
             // Then a key's weights all go to one of the two sums, chosen once per key, and the columns
             // beyond W add exact zeros (their constant is -inf): plain sums, no per-column selection.
-            const bool plain = ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
+            const bool plain = !want_hist && ndq == 1 && (i * int(csize) + int(rank) + 1) * kTileKeys <= first_masked_key;
             auto chunk_plain = [&](const uint32_t (&cur)[16], const float* cvp) {
                 const float4* cv = reinterpret_cast<const float4*>(cvp);
                 const float2 sc2 = make_float2(scale2, scale2);
@@ -455,6 +479,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
             }
             if (set == 0 && t < N) { out_s[t] = s; out_c[t] = c; }
         }
+        if (want_hist) {
+            // the warps' counts of this CTA go to the unit's histogram (the CTAs of the cluster add up there)
+            epi_sync();
+            const uint32_t* const all = reinterpret_cast<const uint32_t*>(base_ptr + sp.hist);
+            uint32_t* const dst = a.hist + (int64_t(b) * a.n_kv_heads + h) * 2 * kHistBins;
+            for (int j = tid; j < 2 * kHistBins; j += EP::kEpiThreads) {
+                uint32_t c = 0;
+                for (int w = 0; w < EP::kWarps; ++w) c += all[w * 2 * kHistBins + j];
+                if (c) atomicAdd(&dst[j], c);
+            }
+        }
         if (*abort_flag && tid == 0) atomicOr(a.status, CSP_DEV_TIMEOUT);
     }
 
@@ -469,7 +504,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     cluster_wait();
 }
 
-template <int NH, int G>
+template <int NH, int G, bool kHist>
 csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
     const int units = p.batch * p.n_kv_heads;
@@ -481,12 +516,13 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
         const int c2 = pick_cluster(units, max_tiles, TmemPlan<G>::kBufsShared, sms);
         if ((max_tiles + c2 - 1) / c2 <= TmemPlan<G>::kBufsShared) { shared_sm = true; c = c2; }
     }
-    const int fixed = int(tc_smem_plan(NH, G, 0).total) + 1024;
+    constexpr bool with_hist = kHist;
+    const int fixed = int(tc_smem_plan(NH, G, 0, with_hist).total) + 1024;
     int stages = ((shared_sm ? 113 : 227) * 1024 - fixed) / (NH * kBlockBytes);
     if (stages > 6) stages = 6;
     if (stages < 2) return CSP_ERR_UNSUPPORTED;
-    const size_t smem = tc_smem_plan(NH, G, stages).total + 1024;
-    auto kern = score_tc_kernel<NH, G>;
+    const size_t smem = tc_smem_plan(NH, G, stages, with_hist).total + 1024;
+    auto kern = score_tc_kernel<NH, G, kHist>;
     static std::atomic<bool> configured[kMaxDevices];   // per instantiation and device
     if (!raise_smem_limit(kern, 227 * 1024, configured)) return CSP_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -505,22 +541,50 @@ csp_status launch_inst(const csp_params& p, const ScoreArgs& a, const CUtensorMa
     return CSP_OK;
 }
 
+// Registers-only loop of base-2 exponentials, for csp_probe_ex2_rate: eight independent chains per thread, either
+// on the special-function unit (ex2.approx.ftz.f32, the instruction of the scoring kernels) or through the
+// two-wide FMA-pipe evaluation that the G >= 3 kernels use for one pair in eight.
+template <bool kFmaPipe>
+__global__ void __launch_bounds__(1024) ex2_probe_kernel(int iters, float* sink, size_t sink_elems) {
+    float2 x[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) x[i] = make_float2(0.1f * float(threadIdx.x & 7) + 0.05f * i, 0.3f + 0.07f * i);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 neg = make_float2(-x[i].x, -x[i].y);      // x <- 2^-x stays in (0.5, 1]
+            x[i] = kFmaPipe ? ex2_fma2(neg) : ex2f2(neg);
+        }
+    }
+    const size_t gtid = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (gtid < sink_elems) sink[gtid] = (x[0].x + x[0].y) + (x[1].x + x[1].y) + (x[2].x + x[2].y) + (x[3].x + x[3].y);
+}
+
 template <int NH>
 csp_status launch_g(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
     switch (a.group) {
-        case 1: return launch_inst<NH, 1>(p, a, tmap, s);
-        case 2: return launch_inst<NH, 2>(p, a, tmap, s);
-        case 3: return launch_inst<NH, 3>(p, a, tmap, s);
-        case 4: return launch_inst<NH, 4>(p, a, tmap, s);
-        case 5: return launch_inst<NH, 5>(p, a, tmap, s);
-        case 6: return launch_inst<NH, 6>(p, a, tmap, s);
-        case 7: return launch_inst<NH, 7>(p, a, tmap, s);
-        case 8: return launch_inst<NH, 8>(p, a, tmap, s);
+        case 1: return a.hist ? launch_inst<NH, 1, true>(p, a, tmap, s) : launch_inst<NH, 1, false>(p, a, tmap, s);
+        case 2: return a.hist ? launch_inst<NH, 2, true>(p, a, tmap, s) : launch_inst<NH, 2, false>(p, a, tmap, s);
+        case 3: return a.hist ? launch_inst<NH, 3, true>(p, a, tmap, s) : launch_inst<NH, 3, false>(p, a, tmap, s);
+        case 4: return a.hist ? launch_inst<NH, 4, true>(p, a, tmap, s) : launch_inst<NH, 4, false>(p, a, tmap, s);
+        case 5: return a.hist ? launch_inst<NH, 5, true>(p, a, tmap, s) : launch_inst<NH, 5, false>(p, a, tmap, s);
+        case 6: return a.hist ? launch_inst<NH, 6, true>(p, a, tmap, s) : launch_inst<NH, 6, false>(p, a, tmap, s);
+        case 7: return a.hist ? launch_inst<NH, 7, true>(p, a, tmap, s) : launch_inst<NH, 7, false>(p, a, tmap, s);
+        case 8: return a.hist ? launch_inst<NH, 8, true>(p, a, tmap, s) : launch_inst<NH, 8, false>(p, a, tmap, s);
         default: return CSP_ERR_UNSUPPORTED;
     }
 }
 
 }  // namespace
+
+csp_status launch_ex2_probe(int fma_pipe, int iters, float* sink, size_t sink_elems, long long* n_exp, cudaStream_t s) {
+    const int blocks = 2 * sm_count();
+    if (fma_pipe) ex2_probe_kernel<true><<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
+    else ex2_probe_kernel<false><<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
+    if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
+    *n_exp = (long long)blocks * 1024LL * 8LL * (long long)iters;
+    return CSP_OK;
+}
 
 csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
     switch (p.head_dim * 2) {

@@ -1,0 +1,139 @@
+"""GPU parity of csp_weight_histogram (Section 1: the gap between intra- and inter-modality attention weights)
+against the fp64 oracle, through the C interface.
+
+A bin is an integer decided by a floating-point value.  The kernel decides it from its own fp32 logits, the
+oracle from fp64 ones, so a weight that lies within the kernel's error of a bin edge may be counted on either
+side.  The comparison is therefore: totals identical; and at every bin edge the number of weights below the
+edge differs by no more than the number of oracle weights within `EDGE_EPS` of that edge.  EDGE_EPS follows
+from the score tolerance of the pass: a weight within 2e-3 relative is within 2e-3 / ln 2 = 2.9e-3 in log2.
+The divergence is compared with the one recomputed in fp64 from the kernel's own counts (1e-5) and with the
+oracle's within what the movable counts can change."""
+import numpy as np
+import pytest
+import torch
+
+import csp_synth as synth
+from parity_util import gpu_params, orc_params
+
+pytestmark = pytest.mark.gpu
+
+EDGE_EPS = 3e-3
+
+
+@pytest.fixture(scope="module")
+def csp():
+    from paper_2412_04652_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _js(p, q):
+    p, q = p.astype(np.float64), q.astype(np.float64)
+    if p.sum() == 0 or q.sum() == 0:
+        return np.nan
+    p, q = p / p.sum(), q / q.sum()
+    m = 0.5 * (p + q)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        return 0.5 * np.where(p > 0, p * np.log(p / m), 0).sum() + 0.5 * np.where(q > 0, q * np.log(q / m), 0).sum()
+
+
+def _check(csp, oracle, cfg, modality=None, q_gain=1.0, n=1.0):
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    if q_gain != 1.0:
+        q = (q.float() * q_gain).to(cfg.dtype)
+    mod = cfg.modality() if modality is None else modality
+    p = gpu_params(csp, cfg, n=n)
+    B, H = cfg.batch, cfg.n_kv_heads
+    hist = torch.full((B, H, 2, csp.HIST_BINS), 12345, dtype=torch.int32, device="cuda")     # must be cleared by the call
+    js = torch.full((B, H), -1.0, device="cuda")
+    js_all = torch.full((1,), -1.0, device="cuda")
+    ws = csp.new_workspace(p)
+    csp.weight_histogram(p, q, k, torch.from_numpy(mod).cuda(), torch.from_numpy(cfg.seq_lens).cuda(), hist, ws,
+                         js=js, js_all=js_all)
+    assert csp.device_status(ws) == 0
+    want, near, js_o, js_all_o = oracle.weight_histogram(orc_params(oracle, cfg, n=n), q.cpu(), k.cpu(), mod, cfg.seq_lens,
+                                                         near_eps=EDGE_EPS)
+    got = hist.cpu().numpy().astype(np.int64)
+    G, W, R = cfg.group, cfg.window, cfg.recent
+    for b in range(B):
+        L = int(cfg.seq_lens[b])
+        pairs = 0 if (L < W or L < R) else G * sum(min(L - R, L - W + w + 1) for w in range(W))
+        for h in range(H):
+            assert got[b, h].sum() == pairs == want[b, h].sum()
+            for cls in range(2):
+                assert got[b, h, cls].sum() == want[b, h, cls].sum()
+                below_g, below_o = np.cumsum(got[b, h, cls])[:-1], np.cumsum(want[b, h, cls])[:-1]   # below edge j + 1
+                slack = near[b, h, cls, 1:]
+                assert (np.abs(below_g - below_o) <= slack).all(), (b, h, cls, np.abs(below_g - below_o).max())
+            mine = _js(got[b, h, 0], got[b, h, 1])
+            j = float(js[b, h])
+            if np.isnan(mine):
+                assert np.isnan(j) and np.isnan(js_o[b, h])
+            else:
+                assert abs(j - mine) < 1e-5
+                moved = near[b, h, 0].sum() / max(want[b, h, 0].sum(), 1) + near[b, h, 1].sum() / max(want[b, h, 1].sum(), 1)
+                assert abs(j - js_o[b, h]) <= np.log(2.0) * moved + 1e-5
+    pooled = _js(got[:, :, 0].sum(axis=(0, 1)), got[:, :, 1].sum(axis=(0, 1)))
+    if np.isnan(pooled):
+        assert np.isnan(float(js_all))
+    else:
+        assert abs(float(js_all) - pooled) < 1e-5
+    return got, js.cpu().numpy()
+
+
+def _case(lens, n_q, n_kv, d, W, R, seed, img=(2, 50)):
+    lays = []
+    for i, L in enumerate(lens):
+        rng = np.random.RandomState(seed + i)
+        if L < 60:                                   # too short for images: text only
+            lays.append([(synth.TEXT, L)])
+            continue
+        img_len = max(1, min(img[1], (L - 40) // img[0]))
+        text = L - img[0] * img_len
+        cuts = np.sort(rng.randint(0, text - 40 + 1, size=img[0]))
+        spans = np.diff(np.concatenate([[0], cuts, [text - 40]])).tolist()
+        spans[-1] += 40
+        lays.append(synth.interleaved_layout(spans, img_len))
+    return synth.small_config("diag", lays, n_q, n_kv, d, W, R, seed=seed)
+
+
+@pytest.mark.parametrize("lens,n_q,n_kv,d,W,R", [
+    ((300,), 2, 2, 128, 32, 32),             # MHA, three tiles
+    ((517, 130, 1029), 4, 4, 128, 32, 32),   # ragged batch
+    ((700, 257), 12, 4, 128, 32, 32),        # G = 3: two sets of epilogue warps
+    ((1300, 640), 7, 1, 128, 32, 32),        # G = 7: tiles recomputed in the second pass
+    ((450,), 5, 1, 64, 32, 32),              # 128-byte rows
+    ((260,), 2, 2, 128, 5, 9),               # odd window, R > W
+    ((260,), 2, 2, 128, 32, 7),              # R < W: the causal mask cuts into the candidates
+    ((20, 300), 2, 2, 128, 32, 32),          # a sequence too short for a window: empty histograms, NaN
+])
+def test_histograms_and_divergence_match_the_oracle(csp, oracle, lens, n_q, n_kv, d, W, R):
+    _check(csp, oracle, _case(lens, n_q, n_kv, d, W, R, seed=len(lens) + n_q))
+
+
+def test_histograms_with_mixed_windows_per_head_labels_and_sharp_rows(csp, oracle):
+    cfg = _case((600, 350), 4, 2, 128, 32, 32, seed=5)
+    rng = np.random.RandomState(0)
+    mod = (rng.rand(2, 2, cfg.max_len) < 0.5).astype(np.uint8)          # per head, random including the window
+    _check(csp, oracle, cfg, modality=mod)
+    _check(csp, oracle, cfg, modality=mod, q_gain=5.0, n=0.0)            # peaked rows: weights spread over many bins
+    one = np.zeros((2, cfg.max_len), np.uint8)                           # a single label: no inter pairs at all
+    got, js = _check(csp, oracle, cfg, modality=one)
+    assert got[:, :, 1].sum() == 0 and np.isnan(js).all()
+
+
+def test_many_units_take_the_cluster_kernel_not_the_resident_one(csp, oracle):
+    """With many MHA units the scores come from the resident-cluster kernel; the diagnostic keeps to the
+    one-cluster-per-unit kernel, which carries the histogram code."""
+    rng = np.random.RandomState(11)
+    lens = tuple(int(x) for x in rng.randint(90, 700, size=40))
+    _check(csp, oracle, _case(lens, 8, 8, 128, 32, 32, seed=17))
+
+
+def test_config1_layer_pooled_divergence(csp, oracle):
+    """One layer of the LLaVA-shaped workload: visual keys carry a +0.5 shift on every channel, so the inter
+    weights (text queries on visual keys) are distributed differently from the intra ones: the divergence is
+    well above zero and the kernel and the oracle agree on it."""
+    cfg = synth.config(1)
+    got, js = _check(csp, oracle, cfg)
+    assert (js > 0).all() and js.mean() > 1e-3

@@ -20,7 +20,7 @@ def csp():
 
 def test_every_declared_symbol_is_exported(csp):
     header = open(os.path.join(ROOT, "include", "csp.h")).read()
-    declared = set(re.findall(r"\b(csp_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(csp_[a-z0-9_]+)\s*\(", header))
     assert declared == set(csp.EXPORTS)
     for name in declared:
         assert hasattr(csp.lib(), name), name
