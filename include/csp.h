@@ -181,6 +181,41 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
                            int32_t* keep_idx_or_null,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * A paged cache: K and V rows live in fixed-size pages of a pool instead of one dense run per sequence, and a
+ * table says which page holds which stretch of a sequence (the layout serving engines use so that caches can grow
+ * and shrink without copying).  Algorithm 1's loop prunes such a cache again and again; pruning it where it lies
+ * frees whole pages at the end of every sequence.
+ *   pool tensors  k_pool, v_pool [n_pages, H_kv, page_rows, d]: stride_b is the page stride
+ *   page_table    [B, max_pages] int32 device: rows [i page_rows, (i+1) page_rows) of sequence b are page
+ *                 page_table[b, i]; entries beyond a sequence's length are not read.  A page number outside
+ *                 [0, n_pages) never faults: its rows score as zeros and are not copied, and the call is
+ *                 flagged CSP_DEV_BAD_LEN.
+ *   page_rows     a multiple of 128; max_pages * page_rows >= max_len
+ * Labels, scores and keep_idx stay dense arrays over logical positions.
+ */
+typedef struct {
+    const int32_t* page_table;
+    int32_t max_pages, page_rows, n_pages;
+} csp_pages;
+
+/*
+ * csp_prune_layer on a paged cache (Algorithm 1; Eq. 1-5, 7 unchanged, only the addressing differs).
+ *   k_out, v_out  either dense [B, H_kv, out_capacity, d], or the pools themselves (same pointers and strides):
+ *                 then the kept rows move down inside each sequence's own pages (logical row j goes to page
+ *                 page_table[b, j / page_rows]), and pages past n_out rows can be returned to the pool.
+ * bf16 caches, CSP_HEADS_PER_KV.  Everything else as for csp_prune_layer.
+ */
+csp_status csp_prune_layer_paged(const csp_params* p, csp_tensor q_win, csp_tensor k_pool, csp_tensor v_pool,
+                                 const csp_pages* pages,
+                                 const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                                 const int32_t* seq_lens, const int32_t* budgets,
+                                 const int32_t* total_budget_or_null, const float* lse_or_null,
+                                 csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
+                                 float* score_self_or_null, float* score_cross_or_null,
+                                 int32_t* keep_idx_or_null,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Bytes of scratch that csp_decode_attn needs (status word + per-split partial results).  The first
  * 256 bytes must be zero before first use (csp_workspace_reset). */
 size_t csp_decode_workspace_bytes(const csp_params* p);

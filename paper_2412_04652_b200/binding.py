@@ -27,7 +27,7 @@ EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_selec
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
            "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
            "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step",
-           "csp_weight_histogram", "csp_probe_ex2_rate")
+           "csp_weight_histogram", "csp_probe_ex2_rate", "csp_prune_layer_paged")
 HIST_BINS, HIST_LO, HIST_WIDTH = 64, -32.0, 0.5
 
 
@@ -39,6 +39,10 @@ class CspError(RuntimeError):
 
 class CTensor(C.Structure):
     _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
+
+
+class CPages(C.Structure):
+    _fields_ = [("page_table", C.c_void_p), ("max_pages", C.c_int32), ("page_rows", C.c_int32), ("n_pages", C.c_int32)]
 
 
 class CParams(C.Structure):
@@ -121,6 +125,9 @@ def lib() -> C.CDLL:
         l.csp_decode_step_workspace_bytes.argtypes = [P]
         l.csp_decode_step.restype = C.c_int
         l.csp_decode_step.argtypes = [P, CTensor, CTensor, CTensor, vp, vp, i64, i64, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
+        l.csp_prune_layer_paged.restype = C.c_int
+        l.csp_prune_layer_paged.argtypes = [P, CTensor, CTensor, CTensor, C.POINTER(CPages), vp, i64, i64, vp, vp, vp, vp,
+                                            CTensor, CTensor, vp, vp, vp, vp, vp, vp, sz, vp]
         l.csp_probe_ex2_rate.restype = C.c_int
         l.csp_probe_ex2_rate.argtypes = [C.c_int32, C.c_int32, vp, sz, C.POINTER(C.c_int64), vp]
         l.csp_weight_histogram.restype = C.c_int
@@ -278,6 +285,21 @@ def prune_layer(p: Params, q_win, k, v, modality, seq_lens, budgets, k_out, v_ou
                                  tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
                                  _ptr(score_self), _ptr(score_cross), _ptr(keep_idx),
                                  _ptr(ws), ws.numel(), _stream()), "csp_prune_layer")
+
+
+def prune_layer_paged(p: Params, q_win, k_pool, v_pool, page_table, modality, seq_lens, budgets, k_out, v_out, mod_out,
+                      n_out, ws, total_budget=None, lse=None, score_self=None, score_cross=None, keep_idx=None):
+    """k_pool, v_pool [n_pages, Hkv, page_rows, d]; page_table int32 [B, max_pages] (dense).  k_out / v_out dense
+    [B, Hkv, cap, d], or the pools themselves for pruning in place."""
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    assert page_table.dtype == torch.int32 and page_table.is_contiguous() and page_table.dim() == 2
+    pg = CPages(page_table.data_ptr(), page_table.shape[1], k_pool.shape[2], k_pool.shape[0])
+    _check(lib().csp_prune_layer_paged(C.byref(cp), tensor4(q_win), tensor4(k_pool), tensor4(v_pool), C.byref(pg),
+                                       _ptr(modality), sb, sh, _ptr(seq_lens), _ptr(budgets), _ptr(total_budget),
+                                       _ptr(lse), tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
+                                       _ptr(score_self), _ptr(score_cross), _ptr(keep_idx), _ptr(ws), ws.numel(),
+                                       _stream()), "csp_prune_layer_paged")
 
 
 def static_workspace_limit() -> int:

@@ -54,7 +54,8 @@ csp_status check_workspace(const csp_params& p, void* ws, size_t bytes) {
 
 csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const uint8_t* modality,
                     int64_t msb, int64_t msh, const int32_t* seq_lens, const float* lse, float* score_self,
-                    float* score_cross, void* ws, cudaStream_t stream, uint32_t* hist = nullptr) {
+                    float* score_cross, void* ws, cudaStream_t stream, uint32_t* hist = nullptr,
+                    const csp_pages* pages = nullptr) {
     if (p.batch == 0 || p.max_len == 0) return CSP_OK;
     const WorkspaceLayout wl = workspace_layout(p);
     const bool mean_all = p.head_reduce == CSP_HEADS_MEAN_ALL && p.n_kv_heads > 1;
@@ -75,7 +76,7 @@ csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& 
     const float scale = p.scale > 0.f ? p.scale : 1.0f / sqrtf(float(p.head_dim));
     a.scale_log2 = scale * 1.4426950408889634f;
     a.weight = p.head_reduce == CSP_HEADS_MEAN_ALL ? 1.0f / float(p.n_q_heads) : 1.0f / float(a.group);
-    csp_status st = launch_score(p, a, k, stream);
+    csp_status st = launch_score(p, a, k, stream, pages);
     if (st != CSP_OK) return st;
     if (mean_all) st = launch_head_mean(p, a.score_self, a.score_cross, score_self, score_cross, seq_lens, stream);
     return st;
@@ -102,7 +103,7 @@ csp_status do_select(const csp_params& p, const float* score_self, const float* 
 csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor& v, const uint8_t* modality,
                       int64_t msb, int64_t msh, const int32_t* keep_idx, const int32_t* n_out,
                       const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, int32_t* status,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, const csp_pages* pages = nullptr) {
     const int64_t es = elem_size(p);
     CompactArgs a;
     a.k = k.ptr; a.v = v.ptr; a.k_out = k_out.ptr; a.v_out = v_out.ptr;
@@ -115,6 +116,10 @@ csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor
     a.n_kv_heads = p.n_kv_heads; a.max_len = p.max_len; a.out_capacity = p.out_capacity;
     a.chunks_per_row = int(p.head_dim * es / 16);
     a.status = status;
+    a.page_table = pages ? pages->page_table : nullptr;
+    a.max_pages = pages ? pages->max_pages : 0;
+    a.page_rows = pages ? pages->page_rows : 1;
+    a.n_pages = pages ? pages->n_pages : 0;
     return launch_compact(p, a, stream);
 }
 
@@ -238,6 +243,42 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
         return st;
     return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
                       static_cast<int32_t*>(workspace), stream);
+}
+
+// A page table must cover max_len positions with pages of whole 128-key tiles.
+static csp_status check_pages(const csp_params& p, const csp_pages* pg) {
+    if (!pg || !pg->page_table) return CSP_ERR_INVALID_ARG;
+    if (pg->page_rows <= 0 || pg->page_rows % 128 || pg->max_pages <= 0 || pg->n_pages <= 0) return CSP_ERR_INVALID_ARG;
+    if (int64_t(pg->max_pages) * pg->page_rows < p.max_len) return CSP_ERR_INVALID_ARG;
+    if (p.dtype != CSP_BF16 || p.head_reduce != CSP_HEADS_PER_KV) return CSP_ERR_UNSUPPORTED;
+    return CSP_OK;
+}
+
+csp_status csp_prune_layer_paged(const csp_params* p, csp_tensor q_win, csp_tensor k_pool, csp_tensor v_pool,
+                                 const csp_pages* pages, const uint8_t* modality, int64_t mod_stride_b,
+                                 int64_t mod_stride_h, const int32_t* seq_lens, const int32_t* budgets,
+                                 const int32_t* total_budget_or_null, const float* lse_or_null, csp_tensor k_out,
+                                 csp_tensor v_out, uint8_t* mod_out, int32_t* n_out, float* score_self_or_null,
+                                 float* score_cross_or_null, int32_t* keep_idx_or_null, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_prune_layer_args(p, q_win, k_pool, v_pool, modality, seq_lens, budgets, k_out, v_out, n_out);
+    if (st != CSP_OK) return st;
+    if ((st = check_pages(*p, pages)) != CSP_OK) return st;
+    if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
+    const WorkspaceLayout wl = workspace_layout(*p);
+    char* ws = static_cast<char*>(workspace);
+    float* ss = score_self_or_null ? score_self_or_null : reinterpret_cast<float*>(ws + wl.score_self);
+    float* sc = score_cross_or_null ? score_cross_or_null : reinterpret_cast<float*>(ws + wl.score_cross);
+    int32_t* idx = keep_idx_or_null ? keep_idx_or_null : reinterpret_cast<int32_t*>(ws + wl.keep_idx);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if ((st = do_score(*p, q_win, k_pool, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null, ss, sc,
+                       workspace, stream, nullptr, pages)) != CSP_OK)
+        return st;
+    if ((st = do_select(*p, ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
+                        idx, n_out, workspace, stream)) != CSP_OK)
+        return st;
+    return do_compact(*p, k_pool, v_pool, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
+                      static_cast<int32_t*>(workspace), stream, pages);
 }
 
 // staging layout for the host-buffer variant: every block rounded up to 256 bytes

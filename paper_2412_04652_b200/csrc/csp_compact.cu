@@ -20,6 +20,15 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+// Offset (in 16-byte units, before the chunk index) of row t of unit (b, h) in a source with strides (sb, sh, st):
+// dense, or through the page table.  -1 for a row whose page number is outside the pool.
+__device__ __forceinline__ int64_t row_offset(const CompactArgs& a, int b, int h, int t, int64_t sb, int64_t sh, int64_t st) {
+    if (!a.page_table) return int64_t(b) * sb + int64_t(h) * sh + int64_t(t) * st;
+    const int page = a.page_table[int64_t(b) * a.max_pages + t / a.page_rows];
+    if (page < 0 || page >= a.n_pages) return -1;
+    return int64_t(page) * sb + int64_t(h) * sh + int64_t(t % a.page_rows) * st;
+}
+
 template <int rows_cta, int CPR>   // rows per CTA; 16-byte chunks per row (8, 16 or 32)
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactArgs a) {
     const int blocks_per_unit = (a.out_capacity + rows_cta - 1) / rows_cta;
@@ -35,8 +44,8 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactA
     constexpr int rows_per_iter = kCompactThreads / cpr;
     const int r_in = threadIdx.x / cpr, c = threadIdx.x % cpr;
     const int32_t* const idx = a.keep_idx + int64_t(u) * a.out_capacity;
-    const uint4* const kin = static_cast<const uint4*>(a.k) + int64_t(b) * a.k_sb + int64_t(h) * a.k_sh;
-    const uint4* const vin = static_cast<const uint4*>(a.v) + int64_t(b) * a.v_sb + int64_t(h) * a.v_sh;
+    const uint4* const kin = static_cast<const uint4*>(a.k);
+    const uint4* const vin = static_cast<const uint4*>(a.v);
     uint4* const kout = static_cast<uint4*>(a.k_out) + int64_t(b) * a.ko_sb + int64_t(h) * a.ko_sh;
     uint4* const vout = static_cast<uint4*>(a.v_out) + int64_t(b) * a.vo_sb + int64_t(h) * a.vo_sh;
     const int row_end = min(n, row0 + rows_cta);
@@ -51,9 +60,10 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactA
             if (jj[q] < row_end) {
                 const int t = idx[jj[q]];
                 const bool ok = t >= 0 && t < a.max_len;   // a bad index copies nothing
-                if (ok) {
-                    kv[q] = ld_stream(kin + int64_t(t) * a.k_st + c);
-                    vv[q] = ld_stream(vin + int64_t(t) * a.v_st + c);
+                const int64_t ko = ok ? row_offset(a, b, h, t, a.k_sb, a.k_sh, a.k_st) : -1;
+                if (ko >= 0) {
+                    kv[q] = ld_stream(kin + ko + c);
+                    vv[q] = ld_stream(vin + row_offset(a, b, h, t, a.v_sb, a.v_sh, a.v_st) + c);
                 } else {
                     jj[q] = row_end;
                 }
@@ -91,8 +101,8 @@ __global__ void __launch_bounds__(kInplaceThreads) compact_inplace_kernel(const 
     const int rows_per_iter = kInplaceThreads / cpr;
     const int r_in = threadIdx.x / cpr, c = threadIdx.x % cpr;
     const int32_t* const idx = a.keep_idx + int64_t(u) * a.out_capacity;
-    uint4* const kio = static_cast<uint4*>(a.k_out) + int64_t(b) * a.ko_sb + int64_t(h) * a.ko_sh;
-    uint4* const vio = static_cast<uint4*>(a.v_out) + int64_t(b) * a.vo_sb + int64_t(h) * a.vo_sh;
+    uint4* const kio = static_cast<uint4*>(a.k_out);
+    uint4* const vio = static_cast<uint4*>(a.v_out);
     const int row_end = min(n, a.out_capacity);
     // labels first: they go to a separate array, so no ordering is needed
     if (a.mod_out && a.modality) {
@@ -111,9 +121,10 @@ __global__ void __launch_bounds__(kInplaceThreads) compact_inplace_kernel(const 
             if (jj[q] < row_end) {
                 const int t = idx[jj[q]];
                 // a bad index or a source above its destination copies nothing; a row already in place stays
-                if (t > jj[q] && t < a.max_len) {
-                    kv[q] = kio[int64_t(t) * a.ko_st + c];
-                    vv[q] = vio[int64_t(t) * a.vo_st + c];
+                const int64_t ko = (t > jj[q] && t < a.max_len) ? row_offset(a, b, h, t, a.ko_sb, a.ko_sh, a.ko_st) : -1;
+                if (ko >= 0) {
+                    kv[q] = kio[ko + c];
+                    vv[q] = vio[row_offset(a, b, h, t, a.vo_sb, a.vo_sh, a.vo_st) + c];
                 } else {
                     jj[q] = row_end;
                 }
@@ -123,8 +134,11 @@ __global__ void __launch_bounds__(kInplaceThreads) compact_inplace_kernel(const 
 #pragma unroll
         for (int q = 0; q < 4; ++q)
             if (jj[q] < row_end) {
-                kio[int64_t(jj[q]) * a.ko_st + c] = kv[q];
-                vio[int64_t(jj[q]) * a.vo_st + c] = vv[q];
+                const int64_t ko = row_offset(a, b, h, jj[q], a.ko_sb, a.ko_sh, a.ko_st);
+                if (ko >= 0) {                       // the destination page of a kept row is one of the sequence's own
+                    kio[ko + c] = kv[q];
+                    vio[row_offset(a, b, h, jj[q], a.vo_sb, a.vo_sh, a.vo_st) + c] = vv[q];
+                }
             }
     }
 }

@@ -82,7 +82,25 @@ struct ScoreArgs {
     int32_t n_kv_heads, group, window, recent, max_len;
     float n, scale_log2, weight;                     // weight = 1/G or 1/Hq
     uint32_t* hist;                                  // null, or [B, Hkv, 2, CSP_HIST_BINS] counts to add to
+    // paged cache: tile i of sequence b lies in page page_table[b * max_pages + i / tiles_per_page] of the pool,
+    // at rows (i % tiles_per_page) * 128; null for a dense cache
+    const int32_t* page_table; int32_t max_pages, tiles_per_page, n_pages;
 };
+
+// Coordinates of key tile `tile` of sequence `b` in the K tensor map: (first row, index on the outermost axis).
+// Dense cache: (tile * 128, b).  Paged: a row inside the page that holds the tile, and that page.  A page
+// number outside the pool gives an out-of-range coordinate: the copy then delivers zeros, it cannot fault; the
+// call is flagged CSP_DEV_BAD_LEN.
+__device__ __forceinline__ void tile_coords(const ScoreArgs& a, int tile, int b, int& row, int& outer) {
+    if (a.page_table) {
+        outer = a.page_table[int64_t(b) * a.max_pages + tile / a.tiles_per_page];
+        row = (tile % a.tiles_per_page) * 128;
+        if (outer < 0 || outer >= a.n_pages) { atomicOr(a.status, CSP_DEV_BAD_LEN); outer = a.n_pages; }
+    } else {
+        outer = b;
+        row = tile * 128;
+    }
+}
 
 struct SelectArgs {
     const float* score_self; const float* score_cross;
@@ -102,6 +120,9 @@ struct CompactArgs {
     const int32_t* keep_idx; const int32_t* n_out;
     int32_t n_kv_heads, max_len, out_capacity, chunks_per_row;
     int32_t* status;                                 // device status word, or null (csp_compact has none)
+    // paged source (and, in place, destination): row t of sequence b lies in page page_table[b * max_pages +
+    // t / page_rows] at row t % page_rows; k_sb / v_sb are then the page strides.  Null for a dense cache.
+    const int32_t* page_table; int32_t max_pages, page_rows, n_pages;
 };
 
 // Cluster size (CTAs per unit, a power of two <= 8).  At least enough CTAs to occupy the `sms` SMs when
@@ -127,7 +148,8 @@ csp_status check_prune_layer_args(const csp_params* p, const csp_tensor& q_win, 
                                   const csp_tensor& k_out, const csp_tensor& v_out, const int32_t* n_out);
 
 // ---- host-side launchers (defined next to their kernels) ----------------------------------
-csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s);
+csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s,
+                        const csp_pages* pages = nullptr);
 csp_status launch_score_tc(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s);
 csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
                                 bool* taken);

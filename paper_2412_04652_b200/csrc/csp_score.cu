@@ -584,21 +584,31 @@ bool make_cache_tensor_map(CUtensorMap* map, const csp_tensor& t, int dtype, int
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_tensor& k, cudaStream_t s) {
+csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_tensor& k, cudaStream_t s,
+                        const csp_pages* pages) {
     ScoreArgs a = a_in;
+    a.page_table = nullptr; a.max_pages = 0; a.tiles_per_page = 1; a.n_pages = 0;
+    // a paged cache: the tensor map describes the page pool [pages, heads, page_rows, head_dim]
+    const int map_rows = pages ? pages->page_rows : p.max_len;
+    const int map_outer = pages ? pages->n_pages : p.batch;
+    if (pages) {
+        if (p.dtype != CSP_BF16 || p.head_reduce != CSP_HEADS_PER_KV) return CSP_ERR_UNSUPPORTED;
+        a.page_table = pages->page_table; a.max_pages = pages->max_pages; a.tiles_per_page = pages->page_rows / kTileKeys;
+        a.n_pages = pages->n_pages;
+    }
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return CSP_ERR_CUDA;
     const uint64_t es = p.dtype == CSP_F32 ? 4 : 2;
     const uint64_t row_bytes = uint64_t(p.head_dim) * es;
     // sizes of 1 carry no usable stride: give them a legal one
     const uint64_t st = uint64_t(k.stride_t) * es;
-    const uint64_t sh = p.n_kv_heads > 1 ? uint64_t(k.stride_h) * es : st * uint64_t(p.max_len);
-    const uint64_t sb = p.batch > 1 ? uint64_t(k.stride_b) * es : sh * uint64_t(p.n_kv_heads);
+    const uint64_t sh = p.n_kv_heads > 1 ? uint64_t(k.stride_h) * es : st * uint64_t(map_rows);
+    const uint64_t sb = map_outer > 1 ? uint64_t(k.stride_b) * es : sh * uint64_t(p.n_kv_heads);
     if (k.stride_t < p.head_dim || (st % 16) || (sh % 16) || (sb % 16) || (uintptr_t(k.ptr) % 16))
         return CSP_ERR_UNSUPPORTED;
     CUtensorMap tmap;
-    const cuuint64_t dims[4] = {cuuint64_t(p.head_dim), cuuint64_t(p.max_len), cuuint64_t(p.n_kv_heads),
-                                cuuint64_t(p.batch)};
+    const cuuint64_t dims[4] = {cuuint64_t(p.head_dim), cuuint64_t(map_rows), cuuint64_t(p.n_kv_heads),
+                                cuuint64_t(map_outer)};
     const cuuint64_t strides[3] = {st, sh, sb};
     const cuuint32_t box[4] = {cuuint32_t(128 / es), cuuint32_t(kTileKeys), 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};

@@ -177,16 +177,19 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 const int u = unit_at(j);
                 if (u < 0) break;
                 const Unit x = unit_of(u);
+                int row = 0, outer = x.b;          // where the next tile lies (a paged cache looks it up one tile ahead)
+                if (x.my_all > 0) tile_coords(a, int(rank), x.b, row, outer);
                 for (int i = 0; i < x.my_all; ++i, ++it) {
                     const int slot = it % n_stages;
+                    const int row_now = row, outer_now = outer;
+                    if (i + 1 < x.my_all) tile_coords(a, (i + 1) * int(csize) + int(rank), x.b, row, outer);
                     mbar_wait(empty_k + 8 * slot, (uint32_t(it / n_stages) & 1u) ^ 1u, abort_flag);
                     if (*abort_flag) break;
                     mbar_expect_tx(full_k + 8 * slot, kStageBytes);
-                    const int tile = i * int(csize) + int(rank);
 #pragma unroll
                     for (int hb = 0; hb < NH; ++hb)
                         tma_load_4d(base + slot * kStageBytes + hb * kBlockBytes, &tmap, full_k + 8 * slot,
-                                    hb * 64, tile * kTileKeys, x.h, x.b);
+                                    hb * 64, row_now, x.h, outer_now);
                 }
             }
             if (*abort_flag) {

@@ -162,17 +162,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
         cluster_arrive();                         // cluster barrier 1: nothing of ours to publish
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            auto tile_of = [&](int it) { return (it < my_all ? it : it - my_all + kept) * int(csize) + int(rank); };
+            int row = 0, outer = b;                // where the next tile lies (a paged cache looks it up one tile ahead)
+            if (total > 0) tile_coords(a, tile_of(0), b, row, outer);
             for (int it = 0; it < total; ++it) {
                 const int slot = it % n_stages;
                 const uint32_t round = uint32_t(it / n_stages);
-                const int tile = (it < my_all ? it : it - my_all + kept) * int(csize) + int(rank);
+                const int row_now = row, outer_now = outer;
+                if (it + 1 < total) tile_coords(a, tile_of(it + 1), b, row, outer);
                 mbar_wait(empty_k + 8 * slot, (round & 1u) ^ 1u, abort_flag);
                 if (*abort_flag) break;
                 mbar_expect_tx(full_k + 8 * slot, kStageBytes);
 #pragma unroll
                 for (int hb = 0; hb < NH; ++hb)
                     tma_load_4d(base + slot * kStageBytes + hb * kBlockBytes, &tmap, full_k + 8 * slot,
-                                hb * 64, tile * kTileKeys, h, b);
+                                hb * 64, row_now, h, outer_now);
             }
             if (*abort_flag) {
                 // let copies that were issued land before the CTA's shared memory is given up

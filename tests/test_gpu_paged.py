@@ -1,0 +1,136 @@
+"""GPU parity of csp_prune_layer_paged: the pass on a cache whose rows live in pages of a pool.  Paging changes
+addressing only, so the result must be bit-identical to the dense entry point on the same rows, and it is compared
+with the CPU oracle (run on the dense rows) under the tolerances of the pass."""
+import numpy as np
+import pytest
+import torch
+
+import csp_synth as synth
+from parity_util import (GpuRun, assert_compaction_exact, assert_index_sets_match, assert_scores_close, bits,
+                         gpu_params, orc_params)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def csp():
+    from paper_2412_04652_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _layouts(lens, seed):
+    lays = []
+    for i, L in enumerate(lens):
+        rng = np.random.RandomState(seed + i)
+        img = max(1, min(50, (L - 40) // 2))
+        text = L - 2 * img
+        cuts = np.sort(rng.randint(0, text - 40 + 1, size=2))
+        spans = np.diff(np.concatenate([[0], cuts, [text - 40]])).tolist()
+        spans[-1] += 40
+        lays.append(synth.interleaved_layout(spans, img))
+    return lays
+
+
+def _paged_copy(k, v, lens, page_rows, seed):
+    """Scatters dense [B, H, Lm, d] caches into a shuffled page pool; unused pages hold NaN, unused table
+    entries point outside the pool."""
+    B, H, Lm, d = k.shape
+    per_seq = [-(-int(L) // page_rows) for L in lens]
+    max_pages = -(-Lm // page_rows)
+    n_pages = sum(per_seq) + 3
+    order = np.random.RandomState(seed).permutation(n_pages)
+    table = np.full((B, max_pages), 10 ** 6, np.int32)
+    k_pool = torch.full((n_pages, H, page_rows, d), float("nan"), dtype=k.dtype, device=k.device)
+    v_pool = torch.full((n_pages, H, page_rows, d), float("nan"), dtype=k.dtype, device=k.device)
+    nxt = 0
+    for b in range(B):
+        for i in range(per_seq[b]):
+            pg = int(order[nxt]); nxt += 1
+            table[b, i] = pg
+            r0, r1 = i * page_rows, min((i + 1) * page_rows, int(lens[b]))
+            k_pool[pg, :, :r1 - r0] = k[b, :, r0:r1]
+            v_pool[pg, :, :r1 - r0] = v[b, :, r0:r1]
+    return k_pool, v_pool, torch.from_numpy(table).to(k.device)
+
+
+@pytest.mark.parametrize("lens,n_q,n_kv,page_rows", [
+    ((700, 333, 129), 4, 2, 128),            # ragged batch, one tile per page
+    ((1500, 900), 4, 4, 256),                # two tiles per page
+    ((1300, 640), 7, 1, 128),                # G = 7: tiles recomputed in the second pass go through the table again
+    (tuple(200 + 37 * i for i in range(40)), 8, 8, 128),    # many MHA units: the resident-cluster kernel
+    ((5000, 4097), 2, 2, 512),               # long caches, clusters of several CTAs
+])
+def test_paged_prune_matches_the_dense_one_and_the_oracle(csp, oracle, lens, n_q, n_kv, page_rows):
+    cfg = synth.small_config("paged", _layouts(lens, 3), n_q, n_kv, 128, 32, 32, seed=len(lens) + n_q)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    p = gpu_params(csp, cfg)
+    mod = cfg.modality()
+    dense = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, cfg.budgets).prune()
+    assert dense.status() == 0
+    k_pool, v_pool, table = _paged_copy(k, v, cfg.seq_lens, page_rows, seed=11)
+    pp = gpu_params(csp, cfg)
+    pp.max_len = table.shape[1] * page_rows                      # logical length covered by the table
+    paged = GpuRun(csp, pp, q, k, v, np.pad(mod, ((0, 0), (0, pp.max_len - mod.shape[1]))), cfg.seq_lens, cfg.budgets)
+    csp.prune_layer_paged(pp, paged.q, k_pool, v_pool, table, paged.mod, paged.lens, paged.bud, paged.k_out, paged.v_out,
+                          paged.mod_out, paged.n_out, paged.ws, score_self=paged.ss, score_cross=paged.sc, keep_idx=paged.idx)
+    assert paged.status() == 0
+    assert torch.equal(paged.n_out, dense.n_out) and torch.equal(paged.idx, dense.idx)
+    B, H = cfg.batch, cfg.n_kv_heads
+    for b in range(B):
+        N = int(cfg.seq_lens[b]) - 32
+        assert torch.equal(paged.ss[b, :, :N], dense.ss[b, :, :N]) and torch.equal(paged.sc[b, :, :N], dense.sc[b, :, :N])
+        for h in range(H):
+            n = int(dense.n_out[b, h])
+            assert torch.equal(paged.k_out[b, h, :n], dense.k_out[b, h, :n])
+            assert torch.equal(paged.v_out[b, h, :n], dense.v_out[b, h, :n])
+            assert torch.equal(paged.mod_out[b, h, :n], dense.mod_out[b, h, :n])
+    # the oracle on the dense rows
+    ref = oracle.prune_layer(orc_params(oracle, cfg), q.cpu(), k.cpu(), v.cpu(), mod, cfg.seq_lens, cfg.budgets)
+    assert_scores_close(paged.ss.cpu().numpy()[:, :, :cfg.max_len], ref["score_self"], cfg.seq_lens, 32, "self")
+    assert_scores_close(paged.sc.cpu().numpy()[:, :, :cfg.max_len], ref["score_cross"], cfg.seq_lens, 32, "cross")
+    assert_index_sets_match(paged.idx.cpu().numpy(), paged.n_out.cpu().numpy(), ref, mod, cfg.seq_lens, 32)
+
+    # in place: the kept rows move down inside each sequence's own pages
+    kp, vp = k_pool.clone(), v_pool.clone()
+    inpl = GpuRun(csp, pp, q, k, v, np.pad(mod, ((0, 0), (0, pp.max_len - mod.shape[1]))), cfg.seq_lens, cfg.budgets)
+    csp.prune_layer_paged(pp, inpl.q, kp, vp, table, inpl.mod, inpl.lens, inpl.bud, kp, vp, inpl.mod_out, inpl.n_out, inpl.ws,
+                          keep_idx=inpl.idx)
+    assert inpl.status() == 0 and torch.equal(inpl.n_out, dense.n_out) and torch.equal(inpl.idx, dense.idx)
+    tab = table.cpu().numpy()
+    kb, vb = bits(k), bits(v)
+    kpb, vpb = bits(kp), bits(vp)
+    idx = dense.idx.cpu().numpy()
+    for b in range(B):
+        for h in range(H):
+            n = int(dense.n_out[b, h])
+            rows = np.arange(n)
+            pg, r = tab[b, rows // page_rows], rows % page_rows
+            np.testing.assert_array_equal(kpb[pg, h, r], kb[b, h][idx[b, h, :n]])
+            np.testing.assert_array_equal(vpb[pg, h, r], vb[b, h][idx[b, h, :n]])
+    assert torch.equal(inpl.mod_out, dense.mod_out)
+
+
+def test_paged_arguments_are_checked_and_a_bad_page_is_flagged(csp):
+    cfg = synth.small_config("paged", _layouts((300, 200), 5), 2, 2, 128, 32, 32, seed=9)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    k_pool, v_pool, table = _paged_copy(k, v, cfg.seq_lens, 128, seed=1)
+    p = gpu_params(csp, cfg)
+    p.max_len = table.shape[1] * 128
+    run = GpuRun(csp, p, q, k, v, np.pad(cfg.modality(), ((0, 0), (0, p.max_len - cfg.max_len))), cfg.seq_lens, cfg.budgets)
+
+    def call(pool_k, tab, params=p):
+        csp.prune_layer_paged(params, run.q, pool_k, v_pool, tab, run.mod, run.lens, run.bud, run.k_out, run.v_out,
+                              run.mod_out, run.n_out, run.ws)
+    with pytest.raises(csp.CspError) as e:                       # pages must hold whole 128-key tiles
+        call(k_pool[:, :, :64], table)
+    assert e.value.code == csp.ERR_INVALID_ARG
+    with pytest.raises(csp.CspError) as e:                       # the table must cover max_len
+        call(k_pool, table[:, :1].contiguous())
+    assert e.value.code == csp.ERR_INVALID_ARG
+    bad = table.clone()
+    bad[0, 1] = 10 ** 6                                          # a page number outside the pool, inside the sequence
+    call(k_pool, bad)
+    assert run.status() & csp.DEV_BAD_LEN
+    call(k_pool, table)                                          # and the context is still usable
+    assert run.status() == 0
