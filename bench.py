@@ -237,16 +237,11 @@ def run_reference(args, rank, world):
 # ------------------------------------------------------------------------------------ CUDA arm
 
 def kernels_per_call(p, sms) -> int:
-    """Kernels one csp_prune_layer call launches: score, select, compact (the latter two once per chunk), and,
-    for a bf16 cache with more (sequence, head) units than SMs and several sequences, the kernel that orders
-    them by length."""
+    """Kernels one csp_prune_layer call launches: score, select, compact, and, for a bf16 cache with more
+    (sequence, head) units than SMs and several sequences, the kernel that orders them by length."""
     units, tiles = p.batch * p.n_kv_heads, (p.max_len + 127) // 128
     ordered = p.dtype == 1 and 2 <= p.batch <= 4096 and (units > sms or units * min(tiles, 8) > sms * 13 // 16)
-    # with many units the selection and the compaction run as up to four chunks each (overlapped on two streams)
-    chunks = min(4, units // 64, p.n_kv_heads if p.batch == 1 else p.batch)
-    if chunks < 2 or p.max_len > 65536:
-        chunks = 1
-    return (1 if ordered else 0) + 1 + 2 * chunks
+    return 4 if ordered else 3
 
 
 class PathBench:

@@ -21,12 +21,7 @@
  *  - Every pointer is a DEVICE pointer unless its name ends in `_host`.  The caller owns every
  *    buffer.  The library never allocates or frees device memory and, except for
  *    csp_device_status and csp_prune_layer_host, never synchronises: work is enqueued on the
- *    given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).  With many
- *    units csp_prune_layer (and its paged and host forms) runs its selections on a stream of its
- *    own that forks from and rejoins the given stream through events, so that they hide behind the
- *    compaction copies; to the caller the call is ordered like any other work on the given stream,
- *    also under stream capture.  That stream and five events are created on the first such call on
- *    a device and kept; csp_prune_layer_static never does this.
+ *    given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
  *  - Inputs are read-only.  Outputs must not overlap inputs or each other, with one exception:
  *    compaction in place (k_out the very tensor k and v_out the very tensor v), see csp_compact.
  *  - Host threads: entry points may be called from several host threads at once, on the same or on

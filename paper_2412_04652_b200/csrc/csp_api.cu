@@ -1,8 +1,6 @@
 // C interface of libcsp: argument checks, workspace carving and kernel sequencing.
 #include <math.h>
 
-#include <mutex>
-
 #include "csp_internal.cuh"
 
 namespace csp {
@@ -125,139 +123,6 @@ csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor
     return launch_compact(p, a, stream);
 }
 
-// ---- selection and compaction of one call, overlapped -------------------------------------------------
-// The selection is a chain of short dependent phases that leaves the memory system idle; the compaction is
-// pure data movement.  With many units the call is cut into up to four chunks of whole sequences (of heads, when
-// there is one sequence): the selections run back to back on a side stream while each chunk's compaction follows
-// its own selection on the caller's stream, so all but the first selection hide behind copies.  The side stream
-// forks from and joins the caller's stream through events, so the call stays ordered like any other work on that
-// stream (also under stream capture).  Results do not depend on the chunking: units are independent.
-constexpr int kMaxChunks = 4;
-constexpr int kMinUnitsPerChunk = 64;
-struct Overlap {
-    cudaStream_t side = nullptr;
-    cudaEvent_t ev[kMaxChunks + 1] = {};
-    bool ready = false, failed = false;
-};
-std::mutex g_overlap_mutex;           // guards creation and the enqueue sequence (events are shared per device)
-Overlap g_overlap[kMaxDevices];
-
-Overlap* overlap_for_current_device() {           // call with g_overlap_mutex held
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
-    Overlap& o = g_overlap[dev];
-    if (o.failed) return nullptr;
-    if (!o.ready) {
-        bool ok = cudaStreamCreateWithFlags(&o.side, cudaStreamNonBlocking) == cudaSuccess;
-        for (int i = 0; ok && i <= kMaxChunks; ++i)
-            ok = cudaEventCreateWithFlags(&o.ev[i], cudaEventDisableTiming) == cudaSuccess;
-        if (!ok) { cudaGetLastError(); o.failed = true; return nullptr; }
-        o.ready = true;
-    }
-    return &o;
-}
-
-struct TailArgs {      // everything select + compact of a call need
-    const float* ss; const float* sc;
-    const uint8_t* modality; int64_t msb, msh;
-    const int32_t* seq_lens; const int32_t* budgets; const int32_t* total_budget;
-    int32_t* idx; int32_t* n_out;
-    csp_tensor k, v, k_out, v_out;
-    uint8_t* mod_out;
-    void* ws;
-    const csp_pages* pages;
-};
-
-// the same arguments restricted to sequences [b0, b0 + nb) (heads [h0, h0 + nh) of the only sequence when by_head)
-void restrict_to(const csp_params& p, const TailArgs& t, bool by_head, int first, int count, csp_params* pc,
-                 TailArgs* tc, csp_pages* pages_c) {
-    *pc = p;
-    *tc = t;
-    const int64_t es = elem_size(p);
-    const int nbud = p.select_mode == CSP_SELECT_GLOBAL ? 2 : (p.select_mode == CSP_SELECT_OVERALL ? 1 : 4);
-    const int64_t u0 = by_head ? first : int64_t(first) * p.n_kv_heads;
-    if (by_head) pc->n_kv_heads = count, pc->n_q_heads = count * (p.n_q_heads / p.n_kv_heads);
-    else pc->batch = count;
-    tc->ss = t.ss + u0 * p.max_len;
-    tc->sc = t.sc + u0 * p.max_len;
-    tc->idx = t.idx + u0 * p.out_capacity;
-    tc->n_out = t.n_out + u0;
-    if (t.mod_out) tc->mod_out = t.mod_out + u0 * p.out_capacity;
-    auto shift = [&](csp_tensor x, bool pool) {
-        if (pool) { if (by_head) x.ptr = static_cast<char*>(x.ptr) + int64_t(first) * x.stride_h * es; return x; }
-        x.ptr = static_cast<char*>(x.ptr) + int64_t(first) * (by_head ? x.stride_h : x.stride_b) * es;
-        return x;
-    };
-    const bool in_place = t.k.ptr == t.k_out.ptr;
-    tc->k = shift(t.k, t.pages != nullptr);
-    tc->v = shift(t.v, t.pages != nullptr);
-    tc->k_out = shift(t.k_out, t.pages != nullptr && in_place);
-    tc->v_out = shift(t.v_out, t.pages != nullptr && in_place);
-    if (by_head) {
-        tc->modality = t.modality + int64_t(first) * t.msh;
-    } else {
-        tc->modality = t.modality + int64_t(first) * t.msb;
-        tc->seq_lens = t.seq_lens + first;
-        tc->budgets = t.budgets + int64_t(first) * nbud;
-        if (t.total_budget) tc->total_budget = t.total_budget + first;
-        if (t.pages) {
-            *pages_c = *t.pages;
-            pages_c->page_table = t.pages->page_table + int64_t(first) * t.pages->max_pages;
-            tc->pages = pages_c;
-        }
-    }
-}
-
-csp_status select_then_compact(const csp_params& p, const TailArgs& t, cudaStream_t stream) {
-    csp_status st = do_select(p, t.ss, t.sc, t.modality, t.msb, t.msh, t.seq_lens, t.budgets, t.total_budget, t.idx,
-                              t.n_out, t.ws, stream);
-    if (st != CSP_OK) return st;
-    return do_compact(p, t.k, t.v, t.modality, t.msb, t.msh, t.idx, t.n_out, t.k_out, t.v_out, t.mod_out,
-                      static_cast<int32_t*>(t.ws), stream, t.pages);
-}
-
-// Eq. 2-4 of one call.  allow_overlap = false keeps everything on the caller's stream (no stream or event is
-// ever created: the allocation-free entry point).
-csp_status finish_prune(const csp_params& p, const TailArgs& t, cudaStream_t stream, bool allow_overlap) {
-    const int64_t units = int64_t(p.batch) * p.n_kv_heads;
-    const bool by_head = p.batch == 1;
-    const int splittable = by_head ? p.n_kv_heads : p.batch;
-    int chunks = int(units / kMinUnitsPerChunk);
-    if (chunks > kMaxChunks) chunks = kMaxChunks;
-    if (chunks > splittable) chunks = splittable;
-    if (!allow_overlap || chunks < 2 || p.max_len > kSelectClusterMaxLen) return select_then_compact(p, t, stream);
-    std::lock_guard<std::mutex> lock(g_overlap_mutex);
-    Overlap* const o = overlap_for_current_device();
-    if (!o) return select_then_compact(p, t, stream);
-    bool ok = cudaEventRecord(o->ev[kMaxChunks], stream) == cudaSuccess &&          // the scores are complete
-              cudaStreamWaitEvent(o->side, o->ev[kMaxChunks], 0) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return CSP_ERR_CUDA; }
-    csp_params pc[kMaxChunks];
-    TailArgs tc[kMaxChunks];
-    csp_pages pgc[kMaxChunks];
-    csp_status st = CSP_OK;
-    int done = 0;
-    for (int i = 0; i < chunks; ++i) {                    // all selections, in order, on the side stream
-        const int first = int(int64_t(splittable) * i / chunks), last = int(int64_t(splittable) * (i + 1) / chunks);
-        restrict_to(p, t, by_head, first, last - first, &pc[i], &tc[i], &pgc[i]);
-        st = do_select(pc[i], tc[i].ss, tc[i].sc, tc[i].modality, tc[i].msb, tc[i].msh, tc[i].seq_lens, tc[i].budgets,
-                       tc[i].total_budget, tc[i].idx, tc[i].n_out, tc[i].ws, o->side);
-        if (st != CSP_OK) break;
-        if (cudaEventRecord(o->ev[i], o->side) != cudaSuccess) { st = CSP_ERR_CUDA; break; }
-        done = i + 1;
-    }
-    // every recorded event is waited for on the caller's stream (this also rejoins a stream capture), then the
-    // chunk's compaction follows
-    for (int i = 0; i < done; ++i) {
-        if (cudaStreamWaitEvent(stream, o->ev[i], 0) != cudaSuccess) { st = CSP_ERR_CUDA; continue; }
-        if (st != CSP_OK) continue;
-        st = do_compact(pc[i], tc[i].k, tc[i].v, tc[i].modality, tc[i].msb, tc[i].msh, tc[i].idx, tc[i].n_out,
-                        tc[i].k_out, tc[i].v_out, tc[i].mod_out, static_cast<int32_t*>(tc[i].ws), stream, tc[i].pages);
-    }
-    if (st == CSP_ERR_CUDA) cudaGetLastError();
-    return st;
-}
-
 }  // namespace
 
 int sm_count() {
@@ -361,21 +226,6 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes,
                            void* cuda_stream) {
-    return prune_layer_impl(p, q_win, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
-                            lse_or_null, k_out, v_out, mod_out, n_out, score_self_or_null, score_cross_or_null,
-                            keep_idx_or_null, workspace, workspace_bytes, cuda_stream, true);
-}
-
-}  // extern "C"
-
-namespace csp {
-csp_status prune_layer_impl(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
-                            const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
-                            const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget_or_null,
-                            const float* lse_or_null, csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out,
-                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
-                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes,
-                            void* cuda_stream, bool overlap) {
     csp_status st = check_prune_layer_args(p, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, n_out);
     if (st != CSP_OK) return st;
     if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
@@ -388,13 +238,12 @@ csp_status prune_layer_impl(const csp_params* p, csp_tensor q_win, csp_tensor k,
     if ((st = do_score(*p, q_win, k, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null, ss, sc,
                        workspace, stream)) != CSP_OK)
         return st;
-    const TailArgs t = {ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null, idx, n_out,
-                        k, v, k_out, v_out, mod_out, workspace, nullptr};
-    return finish_prune(*p, t, stream, overlap);
+    if ((st = do_select(*p, ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
+                        idx, n_out, workspace, stream)) != CSP_OK)
+        return st;
+    return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
+                      static_cast<int32_t*>(workspace), stream);
 }
-}  // namespace csp
-
-extern "C" {
 
 // A page table must cover max_len positions with pages of whole 128-key tiles.
 static csp_status check_pages(const csp_params& p, const csp_pages* pg) {
@@ -425,9 +274,11 @@ csp_status csp_prune_layer_paged(const csp_params* p, csp_tensor q_win, csp_tens
     if ((st = do_score(*p, q_win, k_pool, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null, ss, sc,
                        workspace, stream, nullptr, pages)) != CSP_OK)
         return st;
-    const TailArgs t = {ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null, idx, n_out,
-                        k_pool, v_pool, k_out, v_out, mod_out, workspace, pages};
-    return finish_prune(*p, t, stream, true);
+    if ((st = do_select(*p, ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
+                        idx, n_out, workspace, stream)) != CSP_OK)
+        return st;
+    return do_compact(*p, k_pool, v_pool, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
+                      static_cast<int32_t*>(workspace), stream, pages);
 }
 
 // staging layout for the host-buffer variant: every block rounded up to 256 bytes

@@ -147,15 +147,6 @@ csp_status check_prune_layer_args(const csp_params* p, const csp_tensor& q_win, 
                                   const uint8_t* modality, const int32_t* seq_lens, const int32_t* budgets,
                                   const csp_tensor& k_out, const csp_tensor& v_out, const int32_t* n_out);
 
-// csp_prune_layer; overlap = false keeps every kernel on the caller's stream and creates no stream or event
-csp_status prune_layer_impl(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
-                            const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
-                            const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget_or_null,
-                            const float* lse_or_null, csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out,
-                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
-                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes,
-                            void* cuda_stream, bool overlap);
-
 // ---- host-side launchers (defined next to their kernels) ----------------------------------
 csp_status launch_score(const csp_params& p, const ScoreArgs& a, const csp_tensor& k, cudaStream_t s,
                         const csp_pages* pages = nullptr);

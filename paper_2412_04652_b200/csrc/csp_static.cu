@@ -61,10 +61,9 @@ csp_status csp_prune_layer_static(const csp_params* p, csp_tensor q_win, csp_ten
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps whatever the previous call left: the status area must start at zero
     if (cudaMemsetAsync(ws, 0, csp::kStatusBytes, stream) != cudaSuccess) { cudaGetLastError(); return CSP_ERR_CUDA; }
-    // all kernels on the caller's stream: the overlapped form of csp_prune_layer would create a stream and events
-    st = csp::prune_layer_impl(p, q_win, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets,
-                               total_budget_or_null, lse_or_null, k_out, v_out, mod_out, n_out, nullptr, nullptr, nullptr,
-                               ws, need, cuda_stream, false);
+    st = csp_prune_layer(p, q_win, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets,
+                         total_budget_or_null, lse_or_null, k_out, v_out, mod_out, n_out, nullptr, nullptr, nullptr,
+                         ws, need, cuda_stream);
     if (st != CSP_OK) return st;
     if (dev_status_out_or_null &&
         cudaMemcpyAsync(dev_status_out_or_null, ws, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
