@@ -34,7 +34,8 @@ __device__ __forceinline__ void cluster_sync_all(uint32_t csize) {
 }
 
 template <int kCsThreads, int E>
-__global__ void __launch_bounds__(kCsThreads, kCsThreads <= 512 ? 2 : 1) select_cluster_kernel(const SelectArgs a) {
+__global__ void __launch_bounds__(kCsThreads, kCsThreads <= 256 ? 4 : (kCsThreads <= 512 ? 2 : 1))
+select_cluster_kernel(const SelectArgs a) {
     constexpr int kCsWarps = kCsThreads / 32;
     __shared__ __align__(16) uint32_t hist[2][4][256];   // ping-pong: a round never zeroes what peers still read
     __shared__ uint32_t chosen[4];                       // digit of the K-th value decided in the last round
@@ -362,6 +363,11 @@ csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaS
     // A CTA covers 4096 keys, or 8192 for caches above 4096 positions: smaller clusters mean fewer cluster
     // barriers per round and, in a ragged batch, fewer CTAs that hold no keys.  With many units the CTAs have
     // 512 threads (8 or 16 keys per thread), two per SM, so that one CTA's barrier phases overlap the other's work.
+    // Short caches (the re-prune rounds of a serving batch: a few hundred rows per head) take small CTAs, so that
+    // a whole batch of units is resident at once instead of queueing in waves of two CTAs per SM.
+    if (p.max_len <= 512) return launch_e<256, 2>(p, a, 1, s);
+    if (p.max_len <= 1024) return launch_e<256, 4>(p, a, 1, s);
+    if (p.max_len <= 2048) return launch_e<512, 4>(p, a, 1, s);
     const int per_cta = p.max_len <= 4096 ? 4096 : 8192;
     int cs = 1;
     while (cs < 8 && cs * per_cta < p.max_len) cs *= 2;

@@ -245,6 +245,18 @@ def test_select_matches_oracle_exactly(csp, oracle, mode):
     _select_case(csp, oracle, 3, 2, lens, 32, budgets, quantise=16, seed=2, **mode)   # heavy ties
 
 
+@pytest.mark.parametrize("lens", [(500, 300, 77), (512, 33), (1000, 513, 64), (1024,), (2048, 1500, 1025), (1300, 40)])
+@pytest.mark.parametrize("mode", [dict(), dict(combine=1), dict(select_mode=1), dict(select_mode=2)])
+def test_select_short_caches(csp, oracle, lens, mode):
+    """Caches of up to 512, 1024 and 2048 positions take smaller CTAs (the re-prune rounds of a serving batch)."""
+    nb = {0: 4, 1: 2, 2: 1}[mode.get("select_mode", 0)]
+    B = len(lens)
+    budgets = np.random.RandomState(len(lens) + lens[0]).randint(0, max(lens) // 4, size=(B, nb))
+    _select_case(csp, oracle, B, 3, lens, 32, budgets, seed=21, **mode)
+    _select_case(csp, oracle, B, 3, lens, 32, budgets, quantise=8, seed=22, **mode)       # heavy ties
+    _select_case(csp, oracle, B, 40, lens, 5, budgets, quantise=64, seed=23, **mode)      # many units
+
+
 def test_select_all_equal_scores_and_extreme_budgets(csp, oracle):
     lens = (2100, 40)
     st, flags = _select_case(csp, oracle, 2, 1, lens, 8, [[5, 7, 0, 0], [0, 0, 0, 0]], quantise=1, seed=3)
