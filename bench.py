@@ -618,7 +618,9 @@ def bench_line(cfg, args, world, config_index, m, e2e, cpu_baseline, parity, n_l
             "warmup": max(args.warmup, 3), "ms_per_step": m["ms_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == torch.bfloat16 else "f32",
             "data": "synthetic",
-            "config": {"workload": f"configs[{config_index}] {cfg.name}", "layers": n_layers,
+            "config": {"workload": f"configs[{config_index}] {cfg.name}" +
+                                   (f", first {n_layers} of {cfg.n_layers} layers only" if n_layers != cfg.n_layers else ""),
+                       "layers": n_layers,
                        "distinct_layer_buffers": n_buf, "batch": cfg.batch, "kv_heads": cfg.n_kv_heads,
                        "q_heads": cfg.n_q_heads, "head_dim": cfg.head_dim, "sum_seq_len": tokens_per_layer,
                        "window": cfg.window, "recent": cfg.recent, "kept_rows_per_layer": m["n_out_total"],
@@ -637,14 +639,12 @@ def bench_line(cfg, args, world, config_index, m, e2e, cpu_baseline, parity, n_l
 def run_config(pb: PathBench, csp, args, config_index, rank, world, dev, budget_pct=None, default_line=True):
     """All measurements of one workload; returns the JSON line(s) as dicts (rank 0 prints)."""
     cfg = synth.config(config_index, budget_pct=budget_pct or args.budget_pct) if config_index == 4 else synth.config(config_index)
-    n_layers = cfg.n_layers
+    n_layers = cfg.n_layers if args.layers <= 0 else min(args.layers, cfg.n_layers)   # --layers: a cache cut to its first layers
     sum_l = int(cfg.seq_lens.sum())
     es = 2 if cfg.dtype == torch.bfloat16 else 4
     kv_bytes = 2 * n_layers * cfg.batch * cfg.n_kv_heads * cfg.max_len * cfg.head_dim * es
     huge = kv_bytes > 40e9                       # cycle four distinct layers when the whole cache is too large
-    n_buf = n_layers if args.layers <= 0 else min(args.layers, n_layers)
-    if huge and args.layers <= 0:
-        n_buf = 4
+    n_buf = 4 if huge else n_layers
     fold = args.fold_layers and n_buf == n_layers
     p, fold_call, layer_calls, (mod, lens, bud, tot) = make_calls(csp, cfg, dev, fold, n_buf, n_layers, args.with_lse)
     wl = f"configs{config_index}" + (f"_{budget_pct or args.budget_pct}pct" if config_index == 4 else "") + \
@@ -941,7 +941,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--layers", type=int, default=0, help="distinct layer buffers (0 = all layers)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="prune only the first N layers of the workload (0 = all): a smaller case of the same kernels, "
+                         "for profiler captures; the workload name in the line says so")
     ap.add_argument("--streams", type=int, default=32, help="concurrent layer chains inside the step graph")
     ap.add_argument("--per-layer-calls", dest="fold_layers", action="store_false",
                     help="time only one csp_prune_layer call per layer (concurrent chains in a CUDA graph); by default "
