@@ -617,7 +617,7 @@ csp_status launch_score(const csp_params& p, const ScoreArgs& a_in, const csp_te
                               4, k.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return CSP_ERR_UNSUPPORTED;
+    if (r != CUDA_SUCCESS) return CSP_ERR_CUDA;      // strides and alignment were checked above: the driver call itself failed
     if (p.dtype == CSP_F32) return launch_t<float>(p, a, tmap, s);
     // several sequences and more CTAs than fit on the GPU at once (up to 8 per unit; clusters of 8 occupy
     // about 13/16 of the SMs, 120 of a B200's 148): take the sequences longest first

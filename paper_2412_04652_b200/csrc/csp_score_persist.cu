@@ -16,8 +16,9 @@
 // uses an mbarrier per CTA that all CTAs of the cluster arrive on remotely, so only the epilogue
 // warps take part and nobody else is held up.  Every wait is bounded.
 //
-// Precondition (checked by the launcher): G = 1, no caller-supplied LSE, and at most 16 tiles per CTA,
-// so that every tile's logits stay in tensor memory between the passes.
+// Precondition (checked by the launcher): G = 1 and at most 16 tiles per CTA, so that every tile's logits stay
+// in tensor memory between the passes.  With a caller-supplied log-sum-exp of the window rows there is no pass 1:
+// the epilogue teams go straight to the weights.
 #include "csp_internal.cuh"
 #include "csp_tc.cuh"
 
@@ -313,6 +314,18 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 if (Lraw < 0 || Lraw > a.max_len) atomicOr(a.status, CSP_DEV_BAD_LEN);
             }
 
+            const int qs = j % kQSets;
+            // With the rows' log-sum-exp supplied by the caller there is no pass 1 and nothing to exchange: the
+            // additive constants follow from it directly and pass 2 consumes the tiles as they arrive.
+            if (a.lse) {
+                if (tw == 0) {
+                    const float m = (lane < W && !x.skip)
+                                        ? a.lse[(int64_t(x.b) * a.n_kv_heads + x.h) * W + lane] * 1.4426950408889634f : 0.f;
+                    const float denom = a.n * ex2f(-m) + 1.f;          // (max, sum) = (lse, 1)
+                    cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
+                    mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
+                }
+            } else {
             // ---------------------------------- pass 1 ----------------------------------
             float m_run[8], z_run[8];
 #pragma unroll
@@ -343,7 +356,6 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 if (lr == 0) wst[tw * 32 + (jj >> 1) * 8 + lq * 2 + (jj & 1)] = make_float2(m_run[jj], z_run[jj]);
             }
             team_sync(team);
-            const int qs = j % kQSets;
             if (tw == 0) {
                 // lane l owns window row l: merge the team's warps, push the result into every peer's
                 // shared memory (slot [p][my rank][l]) and tell the peer; then wait for all peers' pushes
@@ -375,6 +387,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
                 cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
                 mbar_wait(q_ready + 8 * qs, uint32_t(j / kQSets) & 1u, abort_flag);   // label table of this unit
             }
+            }   // pass 1 and the exchange of its statistics
             team_sync(team);
 
             // ---------------------------------- pass 2 ----------------------------------
@@ -385,6 +398,8 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
             uint32_t kmod_next = (group < x.my_cand && t_of(group) < x.N) ? modp[t_of(group)] : 0u;
             for (int i = group; i < kBufs; i += 2) {
                 const int buf = i;
+                // without a pass 1 nobody has waited for this unit's logits yet
+                if (a.lse && i < x.my_all) { mbar_wait(my_full + 8 * buf, ph, abort_flag); tc_fence_after(); }
                 if (i >= x.my_cand) {                                    // nothing to score: just hand the buffer back
                     if (i >= x.my_all) mbar_wait(my_full + 8 * buf, ph, abort_flag);     // keep phases in step
                     tc_fence_before();
@@ -522,7 +537,7 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
 csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s,
                                 bool* taken) {
     *taken = false;
-    if (a.group != 1 || a.lse != nullptr || a.hist != nullptr) return CSP_OK;
+    if (a.group != 1 || a.hist != nullptr) return CSP_OK;
     const int row_bytes = p.head_dim * 2;
     if (row_bytes != 128 && row_bytes != 256) return CSP_OK;
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;

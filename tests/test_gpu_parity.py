@@ -172,6 +172,33 @@ def test_score_with_supplied_lse(csp, oracle):
     assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent)
 
 
+@pytest.mark.parametrize("lens_hi,n_seq,heads,d", [(1000, 40, 8, 128), (2500, 20, 16, 64)])
+def test_score_with_supplied_lse_many_units(csp, oracle, lens_hi, n_seq, heads, d):
+    """Many MHA units with the rows' log-sum-exp supplied: the resident-cluster kernel without its first pass
+    (clusters of 1 and 2).  The oracle computes its own normaliser; the results must agree."""
+    rng = np.random.RandomState(lens_hi + 1)
+    lens = tuple(int(x) for x in rng.randint(90, lens_hi, size=n_seq))
+    cfg = _case(lens, heads, heads, d, 32, 32, seed=19)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    lse = np.zeros((n_seq, heads, 32))
+    for b, L in enumerate(lens):
+        o = torch.einsum("hwd,htd->hwt", q[b].double(), k[b, :, :L].double()) / np.sqrt(d)
+        pos = L - 32 + torch.arange(32, device="cuda")
+        o.masked_fill_((torch.arange(L, device="cuda")[None, :] > pos[:, None])[None], float("-inf"))
+        lse[b] = torch.logsumexp(o, dim=2).cpu().numpy()
+    mod = cfg.modality()
+    for b, L in enumerate(lens):
+        mod[b, L - 32:L] = (rng.rand(32) < (0.5 if b % 3 == 0 else 0.0))          # some mixed windows
+    run = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod, cfg.seq_lens, cfg.budgets, lse=lse).score()
+    assert run.status() == 0
+    s, c = oracle.score(orc_params(oracle, cfg), q.cpu(), k.cpu(), mod, cfg.seq_lens)
+    assert_scores_close(run.ss.cpu().numpy(), s, cfg.seq_lens, cfg.recent, "self")
+    assert_scores_close(run.sc.cpu().numpy(), c, cfg.seq_lens, cfg.recent, "cross")
+    plain = GpuRun(csp, gpu_params(csp, cfg), q, k, v, mod, cfg.seq_lens, cfg.budgets).score()
+    for b, L in enumerate(lens):                         # and against the two-pass run of the same kernel
+        np.testing.assert_allclose(run.ss[b, :, :L - 32].cpu().numpy(), plain.ss[b, :, :L - 32].cpu().numpy(), rtol=1e-4, atol=1e-9)
+
+
 def test_score_mean_over_all_heads(csp, oracle):
     cfg = _case((420, 300), 8, 4, 128, 32, 32, seed=11)
     _run_score(csp, oracle, cfg, gpu_kw=dict(head_reduce=csp.HEADS_MEAN_ALL),
