@@ -239,6 +239,28 @@ def test_decode_steps_carry_the_scores_and_the_reprune_follows(csp, oracle, Hq, 
             np.testing.assert_array_equal(mod_out[b, h, :n].cpu().numpy(), mod[b, h].numpy()[ii])
 
 
+def test_decode_step_bad_row_counts_are_clamped_and_flagged(csp, oracle):
+    q, k, v, rows = _case(71, 2, 4, 2, 128, 90, rows=[[90, 40], [13, 64]])
+    bad = rows.clone()
+    bad[0, 0], bad[1, 0] = 500, -7                    # above the capacity, negative
+    p = csp.Params(2, 4, 2, 128, 1, 0, 90, 90)
+    mod = torch.zeros(2, 2, 90, dtype=torch.uint8, device="cuda")
+    lab = torch.zeros(2, dtype=torch.uint8, device="cuda")
+    acc_s, acc_c = torch.full((2, 2, 90), 3.0, device="cuda"), torch.full((2, 2, 90), 3.0, device="cuda")
+    out = torch.zeros(2, 4, 128, device="cuda")
+    ws = csp.new_decode_step_workspace(p)
+    csp.decode_step(p, q.cuda(), k.cuda(), v.cuda(), bad.cuda(), mod, lab, True, out, acc_s, acc_c, ws)
+    assert csp.device_status(ws) & csp.DEV_BAD_LEN
+    po = oracle.Params(2, 4, 2, 128, 1, 0, 90, 90, dtype=oracle.BF16)
+    clamped = torch.tensor([[90, 40], [0, 64]], dtype=torch.int32)
+    o_s, o_c = np.zeros((2, 2, 90)), np.zeros((2, 2, 90))
+    want = oracle.decode_step(po, q, k, v, clamped.numpy(), mod.cpu().numpy(), lab.cpu().numpy(), o_s, o_c, True)
+    got = out.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want) <= REL * np.abs(want) + ABS * float(v.float().abs().max())).all()
+    _score_tolerance_ok(acc_s.cpu().numpy().reshape(4, 90), o_s.reshape(4, 90), "intra")
+    assert (acc_c == 0).all() and (acc_s[1, 0] == 0).all()       # a unit without rows: its sums are cleared
+
+
 def test_decode_step_rejects_bad_arguments(csp):
     p = csp.Params(1, 2, 2, 128, 1, 0, 64, 64)
     z = torch.zeros(1, 2, 64, 128, dtype=torch.bfloat16, device="cuda")

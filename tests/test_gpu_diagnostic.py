@@ -122,6 +122,32 @@ def test_histograms_with_mixed_windows_per_head_labels_and_sharp_rows(csp, oracl
     assert got[:, :, 1].sum() == 0 and np.isnan(js).all()
 
 
+def test_histograms_with_a_supplied_log_sum_exp(csp, oracle):
+    """The caller's log-sum-exp of the window rows in place of the first pass: the same histograms."""
+    cfg = _case((600, 350), 4, 2, 128, 32, 32, seed=6)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    lse = torch.zeros(2, 4, 32, device="cuda")
+    for b, L in enumerate(cfg.seq_lens):
+        L = int(L)
+        kk = k[b].repeat_interleave(2, dim=0)[:, :L].double()
+        o = torch.einsum("hwd,htd->hwt", q[b].double(), kk) / np.sqrt(128)
+        pos = L - 32 + torch.arange(32, device="cuda")
+        o.masked_fill_((torch.arange(L, device="cuda")[None, :] > pos[:, None])[None], float("-inf"))
+        lse[b] = torch.logsumexp(o, dim=2).float()
+    p = gpu_params(csp, cfg)
+    hists = []
+    for use in (None, lse):
+        hist = torch.zeros((2, 2, 2, csp.HIST_BINS), dtype=torch.int32, device="cuda")
+        ws = csp.new_workspace(p)
+        csp.weight_histogram(p, q, k, torch.from_numpy(cfg.modality()).cuda(), torch.from_numpy(cfg.seq_lens).cuda(), hist, ws, lse=use)
+        assert csp.device_status(ws) == 0
+        hists.append(hist.cpu().numpy().astype(np.int64))
+    assert hists[0].sum() == hists[1].sum()
+    # a weight may cross a bin edge between the two normalisers (they agree to about 1e-6): adjacent-bin moves only
+    moved = np.abs(np.cumsum(hists[0], axis=-1) - np.cumsum(hists[1], axis=-1)).max()
+    assert moved <= max(3, hists[0].sum() // 20000)
+
+
 def test_many_units_take_the_cluster_kernel_not_the_resident_one(csp, oracle):
     """With many MHA units the scores come from the resident-cluster kernel; the diagnostic keeps to the
     one-cluster-per-unit kernel, which carries the histogram code."""

@@ -111,6 +111,37 @@ def test_paged_prune_matches_the_dense_one_and_the_oracle(csp, oracle, lens, n_q
     assert torch.equal(inpl.mod_out, dense.mod_out)
 
 
+def test_paged_cache_below_its_budget_is_passed_through(csp, oracle):
+    """Algorithm 1's early return on a paged cache: a sequence shorter than its total budget is copied whole, through
+    the page table; the other one is pruned.  Supplied log-sum-exp and per-head labels ride along."""
+    cfg = synth.small_config("paged", _layouts((600, 300), 9), 4, 2, 128, 32, 32, seed=13)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    total = np.array([100, 301], np.int32)                        # 600 >= 100: pruned; 300 < 301: kept whole
+    k_pool, v_pool, table = _paged_copy(k, v, cfg.seq_lens, 128, seed=5)
+    p = gpu_params(csp, cfg, cap=300)
+    p.max_len = table.shape[1] * 128
+    rng = np.random.RandomState(1)
+    mod = (rng.rand(2, 2, p.max_len) < 0.4).astype(np.uint8)      # per head
+    for b, L in enumerate(cfg.seq_lens):
+        mod[b, :, L - 32:L] = 0
+    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, cfg.budgets, total_budget=total)
+    csp.prune_layer_paged(p, run.q, k_pool, v_pool, table, run.mod, run.lens, run.bud, run.k_out, run.v_out, run.mod_out,
+                          run.n_out, run.ws, total_budget=run.tot, score_self=run.ss, score_cross=run.sc, keep_idx=run.idx)
+    assert run.status() == 0
+    po = orc_params(oracle, cfg, cap=300)
+    ref = oracle.prune_layer(po, q.cpu(), k.cpu(), v.cpu(), mod[:, :, :cfg.max_len], cfg.seq_lens, cfg.budgets, total)
+    assert (ref["flags"][1] & oracle.FLAG_IDENTITY).all() and not (ref["flags"][0] & oracle.FLAG_IDENTITY).any()
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, mod[:, :, :cfg.max_len], cfg.seq_lens, 32)
+    assert (run.n_out[1] == 300).all()
+    np.testing.assert_array_equal(bits(run.k_out)[1, :, :300], bits(k)[1, :, :300])
+    np.testing.assert_array_equal(bits(run.v_out)[1, :, :300], bits(v)[1, :, :300])
+    idx = run.idx.cpu().numpy()
+    for h in range(2):
+        n = int(run.n_out[0, h])
+        np.testing.assert_array_equal(bits(run.k_out)[0, h, :n], bits(k)[0, h][idx[0, h, :n]])
+        np.testing.assert_array_equal(run.mod_out[0, h, :n].cpu().numpy(), mod[0, h][idx[0, h, :n]])
+
+
 def test_paged_arguments_are_checked_and_a_bad_page_is_flagged(csp):
     cfg = synth.small_config("paged", _layouts((300, 200), 5), 2, 2, 128, 32, 32, seed=9)
     q, k, v = synth.make_layer(cfg, 0, "cuda")
