@@ -263,6 +263,16 @@ csp_status csp_weight_histogram(const csp_params* p, csp_tensor q_win, csp_tenso
                                 uint32_t* hist, float* js_or_null, float* js_all_or_null,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * csp_decode_attn over a paged cache (Section 3.3, Eq. 6-7; only the addressing differs): k_pool, v_pool and pages as
+ * for csp_prune_layer_paged, e.g. the pools a prune in place has just compacted.  p->out_capacity is the logical row
+ * capacity per head (at most max_pages * page_rows); n_rows [B, H_kv] counts logical rows.  A page number outside
+ * the pool is flagged CSP_DEV_BAD_LEN; its rows read as zeros.  Workspace: csp_decode_workspace_bytes.
+ */
+csp_status csp_decode_attn_paged(const csp_params* p, csp_tensor q, csp_tensor k_pool, csp_tensor v_pool,
+                                 const csp_pages* pages, const int32_t* n_rows, float* out,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Bytes of scratch that csp_decode_step needs: those of csp_decode_attn plus one row of logits per query head
  * and unit.  The first 256 bytes must be zero before first use (csp_workspace_reset). */
 size_t csp_decode_step_workspace_bytes(const csp_params* p);

@@ -27,7 +27,8 @@ EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_selec
            "csp_prune_layer", "csp_host_staging_bytes", "csp_prune_layer_host", "csp_device_status",
            "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
            "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step",
-           "csp_weight_histogram", "csp_probe_ex2_rate", "csp_prune_layer_paged")
+           "csp_weight_histogram", "csp_probe_ex2_rate", "csp_prune_layer_paged",
+           "csp_decode_attn_paged")
 HIST_BINS, HIST_LO, HIST_WIDTH = 64, -32.0, 0.5
 
 
@@ -128,6 +129,8 @@ def lib() -> C.CDLL:
         l.csp_prune_layer_paged.restype = C.c_int
         l.csp_prune_layer_paged.argtypes = [P, CTensor, CTensor, CTensor, C.POINTER(CPages), vp, i64, i64, vp, vp, vp, vp,
                                             CTensor, CTensor, vp, vp, vp, vp, vp, vp, sz, vp]
+        l.csp_decode_attn_paged.restype = C.c_int
+        l.csp_decode_attn_paged.argtypes = [P, CTensor, CTensor, CTensor, C.POINTER(CPages), vp, vp, vp, sz, vp]
         l.csp_probe_ex2_rate.restype = C.c_int
         l.csp_probe_ex2_rate.argtypes = [C.c_int32, C.c_int32, vp, sz, C.POINTER(C.c_int64), vp]
         l.csp_weight_histogram.restype = C.c_int
@@ -300,6 +303,17 @@ def prune_layer_paged(p: Params, q_win, k_pool, v_pool, page_table, modality, se
                                        _ptr(lse), tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out),
                                        _ptr(score_self), _ptr(score_cross), _ptr(keep_idx), _ptr(ws), ws.numel(),
                                        _stream()), "csp_prune_layer_paged")
+
+
+def decode_attn_paged(p: Params, q, k_pool, v_pool, page_table, n_rows, out, ws):
+    """csp_decode_attn over pools [n_pages, Hkv, page_rows, d] addressed through page_table int32 [B, max_pages]."""
+    cp = p.c()
+    assert q.dim() == 3 and q.stride(2) == 1 and out.is_contiguous() and out.dtype == torch.float32
+    assert page_table.dtype == torch.int32 and page_table.is_contiguous() and page_table.dim() == 2
+    qt = CTensor(q.data_ptr(), q.stride(0), q.stride(1), q.shape[2])
+    pg = CPages(page_table.data_ptr(), page_table.shape[1], k_pool.shape[2], k_pool.shape[0])
+    _check(lib().csp_decode_attn_paged(C.byref(cp), qt, tensor4(k_pool), tensor4(v_pool), C.byref(pg), _ptr(n_rows),
+                                       _ptr(out), _ptr(ws), ws.numel(), _stream()), "csp_decode_attn_paged")
 
 
 def static_workspace_limit() -> int:

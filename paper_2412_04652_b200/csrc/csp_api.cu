@@ -264,6 +264,8 @@ csp_status csp_prune_layer_paged(const csp_params* p, csp_tensor q_win, csp_tens
     csp_status st = check_prune_layer_args(p, q_win, k_pool, v_pool, modality, seq_lens, budgets, k_out, v_out, n_out);
     if (st != CSP_OK) return st;
     if ((st = check_pages(*p, pages)) != CSP_OK) return st;
+    // in place, the kept rows are addressed through the table as well: it must cover the output capacity
+    if (k_out.ptr == k_pool.ptr && int64_t(pages->max_pages) * pages->page_rows < p->out_capacity) return CSP_ERR_INVALID_ARG;
     if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
     const WorkspaceLayout wl = workspace_layout(*p);
     char* ws = static_cast<char*>(workspace);
@@ -446,6 +448,24 @@ csp_status csp_probe_ex2_rate(int32_t fma_pipe, int32_t iterations, float* sink,
     st = launch_ex2_probe(fma_pipe ? 1 : 0, iterations, sink, sink ? sink_elems : 0, &n, static_cast<cudaStream_t>(cuda_stream));
     *exponentials_host_out = n;
     return st;
+}
+
+csp_status csp_decode_attn_paged(const csp_params* p, csp_tensor q, csp_tensor k_pool, csp_tensor v_pool,
+                                 const csp_pages* pages, const int32_t* n_rows, float* out, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!q.ptr || !k_pool.ptr || !v_pool.ptr || !n_rows || !out) return CSP_ERR_INVALID_ARG;
+    if (p->dtype != CSP_BF16 || (p->head_dim != 64 && p->head_dim != 128)) return CSP_ERR_UNSUPPORTED;
+    if (!tensor_ok(*p, q) || !tensor_ok(*p, k_pool) || !tensor_ok(*p, v_pool)) return CSP_ERR_UNSUPPORTED;
+    if (!pages || !pages->page_table || pages->page_rows <= 0 || pages->page_rows % 128 || pages->max_pages <= 0 ||
+        pages->n_pages <= 0 || int64_t(pages->max_pages) * pages->page_rows < p->out_capacity)
+        return CSP_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < decode_workspace_bytes(*p) || (uintptr_t(workspace) % 256))
+        return CSP_ERR_WORKSPACE;
+    if ((st = check_arch()) != CSP_OK) return st;
+    return launch_decode_attn(*p, q, k_pool, v_pool, n_rows, out, workspace, static_cast<cudaStream_t>(cuda_stream),
+                              nullptr, pages);
 }
 
 size_t csp_decode_step_workspace_bytes(const csp_params* p) {

@@ -48,6 +48,9 @@ struct DecodeArgs {
     const uint8_t* query_label;                    // [B]
     float* acc_self; float* acc_cross;             // [units, capacity]
     int32_t first_step;
+    // paged cache: rows [i page_rows, (i + 1) page_rows) of sequence b are page page_table[b * max_pages + i] of the
+    // pool the tensor maps describe; null for a dense cache
+    const int32_t* page_table; int32_t max_pages, page_rows, n_pages;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -149,11 +152,17 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     if (*abort_flag) break;
                     if (i == 0) item_q[j % kQueue] = w;     // published by the arrive below (release)
                     mbar_expect_tx(full_bar + 8 * s, kStageBytes);
-                    const int row = (x.tile0 + i) * kDecTile;
+                    int row = (x.tile0 + i) * kDecTile, outer = x.b;
+                    if (a.page_table) {
+                        // a page number outside the pool becomes an out-of-range coordinate: zeros arrive, nothing faults
+                        outer = a.page_table[int64_t(x.b) * a.max_pages + row / a.page_rows];
+                        if (outer < 0 || outer >= a.n_pages) { atomicOr(a.status, CSP_DEV_BAD_LEN); outer = a.n_pages; }
+                        row %= a.page_rows;
+                    }
 #pragma unroll
                     for (int hb = 0; hb < NH; ++hb) {
-                        tma_load_4d(base + s * kStageBytes + hb * kDecBlock, &tmap_k, full_bar + 8 * s, hb * 64, row, x.h, x.b);
-                        tma_load_4d(base + s * kStageBytes + kTileBytes + hb * kDecBlock, &tmap_v, full_bar + 8 * s, hb * 64, row, x.h, x.b);
+                        tma_load_4d(base + s * kStageBytes + hb * kDecBlock, &tmap_k, full_bar + 8 * s, hb * 64, row, x.h, outer);
+                        tma_load_4d(base + s * kStageBytes + kTileBytes + hb * kDecBlock, &tmap_v, full_bar + 8 * s, hb * 64, row, x.h, outer);
                     }
                 }
                 ++j;
@@ -419,13 +428,18 @@ size_t decode_step_workspace_bytes(const csp_params& p) {
 }
 
 csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
-                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s, const DecodeStepArgs* step) {
+                              const int32_t* n_rows, float* out, void* ws, cudaStream_t s, const DecodeStepArgs* step,
+                              const csp_pages* pages) {
     if (p.dtype != CSP_BF16 || (p.head_dim != 64 && p.head_dim != 128)) return CSP_ERR_UNSUPPORTED;
     const int units = p.batch * p.n_kv_heads;
     if (units == 0) return CSP_OK;
     DecodeArgs a;
     a.logits = nullptr; a.modality = nullptr; a.mod_sb = a.mod_sh = 0; a.query_label = nullptr;
     a.acc_self = a.acc_cross = nullptr; a.first_step = 0;
+    a.page_table = pages ? pages->page_table : nullptr;
+    a.max_pages = pages ? pages->max_pages : 0;
+    a.page_rows = pages ? pages->page_rows : 1;
+    a.n_pages = pages ? pages->n_pages : 0;
     if (step) {
         a.logits = reinterpret_cast<float*>(static_cast<char*>(ws) + decode_workspace_bytes(p));
         a.modality = step->modality; a.mod_sb = step->mod_sb; a.mod_sh = step->mod_sh;
@@ -447,8 +461,9 @@ csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const cs
     a.scale_log2 = (p.scale > 0.f ? p.scale : 1.0f / sqrtf(float(p.head_dim))) * 1.4426950408889634f;
     if (p.out_capacity > 0) {
         CUtensorMap tk, tv;
-        if (!make_cache_tensor_map(&tk, k, p.dtype, p.head_dim, p.out_capacity, p.n_kv_heads, p.batch, kDecTile) ||
-            !make_cache_tensor_map(&tv, v, p.dtype, p.head_dim, p.out_capacity, p.n_kv_heads, p.batch, kDecTile))
+        const int map_rows = pages ? pages->page_rows : p.out_capacity, map_outer = pages ? pages->n_pages : p.batch;
+        if (!make_cache_tensor_map(&tk, k, p.dtype, p.head_dim, map_rows, p.n_kv_heads, map_outer, kDecTile) ||
+            !make_cache_tensor_map(&tv, v, p.dtype, p.head_dim, map_rows, p.n_kv_heads, map_outer, kDecTile))
             return CSP_ERR_UNSUPPORTED;
         const int NH = p.head_dim / 64;
         const size_t smem = 1024 + size_t(kDecStages) * 2 * NH * kDecBlock + size_t(kDecWarps) * 8 * (p.head_dim + 2) * 4 +

@@ -181,6 +181,6 @@ struct DecodeStepArgs {
 size_t decode_step_workspace_bytes(const csp_params& p);
 csp_status launch_decode_attn(const csp_params& p, const csp_tensor& q, const csp_tensor& k, const csp_tensor& v,
                               const int32_t* n_rows, float* out, void* ws, cudaStream_t s,
-                              const DecodeStepArgs* step = nullptr);
+                              const DecodeStepArgs* step = nullptr, const csp_pages* pages = nullptr);
 
 }  // namespace csp

@@ -142,6 +142,44 @@ def test_paged_cache_below_its_budget_is_passed_through(csp, oracle):
         np.testing.assert_array_equal(run.mod_out[0, h, :n].cpu().numpy(), mod[0, h][idx[0, h, :n]])
 
 
+@pytest.mark.parametrize("G,d,page_rows", [(1, 128, 128), (4, 64, 256), (7, 128, 128)])
+def test_decode_over_the_pages_a_prune_in_place_leaves(csp, oracle, G, d, page_rows):
+    """Prune a paged cache in place, then one decode query per head attends to what is left, through the same page
+    table: compared with the dense decode call on the dense prune's output (bit-identical: the same rows in the same
+    order) and with the oracle."""
+    lens = (900, 517, 1300)
+    cfg = synth.small_config("paged", _layouts(lens, 21), 2 * G, 2, d, 32, 32, seed=30 + G)
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    p = gpu_params(csp, cfg)
+    dense = GpuRun(csp, p, q, k, v, cfg.modality(), cfg.seq_lens, cfg.budgets).prune()
+    k_pool, v_pool, table = _paged_copy(k, v, cfg.seq_lens, page_rows, seed=3)
+    pp = gpu_params(csp, cfg)
+    pp.max_len = table.shape[1] * page_rows
+    inpl = GpuRun(csp, pp, q, k, v, np.pad(cfg.modality(), ((0, 0), (0, pp.max_len - cfg.max_len))), cfg.seq_lens, cfg.budgets)
+    csp.prune_layer_paged(pp, inpl.q, k_pool, v_pool, table, inpl.mod, inpl.lens, inpl.bud, k_pool, v_pool, inpl.mod_out,
+                          inpl.n_out, inpl.ws)
+    assert inpl.status() == 0 and torch.equal(inpl.n_out, dense.n_out)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    q1 = torch.randn(3, 2 * G, d, device="cuda", generator=gen).to(torch.bfloat16)
+    cap = p.out_capacity
+    pd = csp.Params(3, 2 * G, 2, d, 1, 0, cap, cap)
+    out_dense, out_paged = torch.zeros(3, 2 * G, d, device="cuda"), torch.full((3, 2 * G, d), 9.0, device="cuda")
+    wd = csp.new_decode_workspace(pd)
+    csp.decode_attn(pd, q1, dense.k_out, dense.v_out, dense.n_out, out_dense, wd)
+    csp.decode_attn_paged(pd, q1, k_pool, v_pool, table, inpl.n_out, out_paged, wd)
+    assert csp.device_status(wd) == 0
+    assert torch.equal(out_paged, out_dense)
+    po = oracle.Params(3, 2 * G, 2, d, 1, 0, cap, cap, dtype=oracle.BF16)
+    want = oracle.decode_attn(po, q1.cpu(), dense.k_out.cpu(), dense.v_out.cpu(), dense.n_out.cpu().numpy())
+    got = out_paged.cpu().numpy().astype(np.float64)
+    tol = 2e-3 * np.abs(want) + 1e-5 * float(v.float().abs().max())
+    assert (np.abs(got - want) <= tol).all()
+    bad = table.clone()
+    bad[1, 0] = -5
+    csp.decode_attn_paged(pd, q1, k_pool, v_pool, bad, inpl.n_out, out_paged, wd)
+    assert csp.device_status(wd) & csp.DEV_BAD_LEN
+
+
 def test_paged_arguments_are_checked_and_a_bad_page_is_flagged(csp):
     cfg = synth.small_config("paged", _layouts((300, 200), 5), 2, 2, 128, 32, 32, seed=9)
     q, k, v = synth.make_layer(cfg, 0, "cuda")
