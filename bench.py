@@ -325,7 +325,7 @@ class PathBench:
             sink = torch.zeros(2 * self.sms * 1024, device=self.dev)
             res = {}
             with torch.cuda.stream(stream):
-                for name, fma in (("special_function_unit", False), ("fma_pipe_two_wide", True)):
+                for name, fma in (("special_function_unit", 0), ("fma_pipe_two_wide", 1), ("half_precision_pairs", 2)):
                     csp.probe_ex2_rate(fma, 256, sink)
                     stream.synchronize()
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

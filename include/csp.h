@@ -360,8 +360,10 @@ size_t csp_static_workspace_limit(void);
  * registers-only kernel (two CTAs of 1024 threads per SM, eight independent chains per thread) that evaluates
  * *exponentials_host_out base-2 exponentials in total; the caller times it with events on the stream.
  *   fma_pipe    0: ex2.approx.ftz.f32 on the special-function unit (what the scoring kernels issue);
- *               1: the two-wide FMA-pipe evaluation the G >= 3 kernels use for one pair in eight
- *   iterations  1 .. 2^20 loop trips (8 exponentials per thread and trip)
+ *               1: the two-wide FMA-pipe evaluation the G >= 3 kernels use for one pair in eight;
+ *               2: ex2.approx.f16x2, two half-precision exponentials per instruction (measured for comparison; no
+ *                  kernel uses it: a half-precision argument is too coarse for the row sums)
+ *   iterations  1 .. 2^20 loop trips (8 exponentials per thread and trip; 16 in mode 2)
  *   sink        device array that receives one float per thread (keeps the loop alive); may be NULL
  */
 csp_status csp_probe_ex2_rate(int32_t fma_pipe, int32_t iterations, float* sink, size_t sink_elems,

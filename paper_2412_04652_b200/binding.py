@@ -257,7 +257,7 @@ def weight_histogram(p: Params, q_win, k, modality, seq_lens, hist, ws, js=None,
 def probe_ex2_rate(fma_pipe: bool, iterations: int, sink: Optional[torch.Tensor] = None) -> int:
     """Enqueues the exponential-throughput probe on the current stream; returns how many exponentials it evaluates."""
     n = C.c_int64(0)
-    _check(lib().csp_probe_ex2_rate(int(bool(fma_pipe)), int(iterations), _ptr(sink), 0 if sink is None else sink.numel(),
+    _check(lib().csp_probe_ex2_rate(int(fma_pipe), int(iterations), _ptr(sink), 0 if sink is None else sink.numel(),
                                     C.byref(n), _stream()), "csp_probe_ex2_rate")
     return int(n.value)
 

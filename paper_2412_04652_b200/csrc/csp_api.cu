@@ -445,7 +445,7 @@ csp_status csp_probe_ex2_rate(int32_t fma_pipe, int32_t iterations, float* sink,
     csp_status st = check_arch();
     if (st != CSP_OK) return st;
     long long n = 0;
-    st = launch_ex2_probe(fma_pipe ? 1 : 0, iterations, sink, sink ? sink_elems : 0, &n, static_cast<cudaStream_t>(cuda_stream));
+    st = launch_ex2_probe(fma_pipe == 2 ? 2 : (fma_pipe ? 1 : 0), iterations, sink, sink ? sink_elems : 0, &n, static_cast<cudaStream_t>(cuda_stream));
     *exponentials_host_out = n;
     return st;
 }

@@ -564,6 +564,26 @@ __global__ void __launch_bounds__(1024) ex2_probe_kernel(int iters, float* sink,
     if (gtid < sink_elems) sink[gtid] = (x[0].x + x[0].y) + (x[1].x + x[1].y) + (x[2].x + x[2].y) + (x[3].x + x[3].y);
 }
 
+// the same chain on packed half-precision pairs (ex2.approx.f16x2: two exponentials per instruction), eight packed
+// chains per thread
+__global__ void __launch_bounds__(1024) ex2_probe_half2_kernel(int iters, float* sink, size_t sink_elems) {
+    uint32_t x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = 0x38003400u + uint32_t(threadIdx.x & 7) * 0x00100010u + uint32_t(i);   // halves near 0.5
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t neg = x[i] ^ 0x80008000u;               // x <- 2^-x stays in (0.5, 1]
+            asm volatile("ex2.approx.f16x2 %0, %1;" : "=r"(x[i]) : "r"(neg));
+        }
+    }
+    const size_t gtid = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    uint32_t acc = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc ^= x[i];
+    if (gtid < sink_elems) sink[gtid] = __uint_as_float(acc & 0x3fffffffu);
+}
+
 template <int NH>
 csp_status launch_g(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, cudaStream_t s) {
     switch (a.group) {
@@ -583,10 +603,11 @@ csp_status launch_g(const csp_params& p, const ScoreArgs& a, const CUtensorMap& 
 
 csp_status launch_ex2_probe(int fma_pipe, int iters, float* sink, size_t sink_elems, long long* n_exp, cudaStream_t s) {
     const int blocks = 2 * sm_count();
-    if (fma_pipe) ex2_probe_kernel<true><<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
+    if (fma_pipe == 2) ex2_probe_half2_kernel<<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
+    else if (fma_pipe) ex2_probe_kernel<true><<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
     else ex2_probe_kernel<false><<<blocks, 1024, 0, s>>>(iters, sink, sink_elems);
     if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
-    *n_exp = (long long)blocks * 1024LL * 8LL * (long long)iters;
+    *n_exp = (long long)blocks * 1024LL * (fma_pipe == 2 ? 16LL : 8LL) * (long long)iters;
     return CSP_OK;
 }
 
