@@ -8,6 +8,8 @@ second per layer: (sum of sequence lengths) / (time of one layer's prune).
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
     python bench.py --all-configs          one JSON line per workload 1-4 (4: every budget of its sweep)
     python bench.py --decode               the step after the pass: n-softmax decode attention
+    python bench.py --incremental          a re-prune from the sums that decode steps carried, against the rescan
+    python bench.py --diagnostic           per-layer JS divergence between intra- and inter-modality window weights
 
 With N > 1 (launched under torch.distributed.run) every rank prunes its own replica of the
 workload; there is no exchange step on this path, so the job throughput is the sum.
@@ -823,6 +825,49 @@ def run_decode(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_diagnostic(args, rank, world, local_rank):
+    """`--diagnostic`: the measurement behind the method (Section 1: the gap between intra- and inter-modality attention
+    weights) on the synthetic caches: csp_weight_histogram once per layer, the Jensen-Shannon divergence of every
+    layer's pooled intra / inter histograms (64 half-octave bins of log2(weight)), and what the call costs.  Prints its
+    own JSON line; not the default.  The values describe the synthetic generator, not a model."""
+    from paper_2412_04652_b200 import binding as csp
+    csp.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    cfg = synth.config(args.config, budget_pct=args.budget_pct) if args.config == 4 else synth.config(args.config)
+    n_layers = min(cfg.n_layers, 8 if args.config == 4 else cfg.n_layers)
+    p = csp.Params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.recent, cfg.max_len,
+                   cfg.out_capacity())
+    mod = torch.from_numpy(cfg.modality()).to(dev)
+    lens = torch.from_numpy(cfg.seq_lens).to(dev)
+    ws = csp.new_workspace(p, dev)
+    hist = torch.zeros(cfg.batch, cfg.n_kv_heads, 2, csp.HIST_BINS, dtype=torch.int32, device=dev)
+    js_all = torch.zeros(1, device=dev)
+    pb = PathBench(csp, args, dev, local_rank, None)
+    js, totals, ms = [], np.zeros((2, csp.HIST_BINS), np.int64), []
+    with torch.cuda.stream(pb.stream):
+        for layer in range(n_layers):
+            q, k, v = synth.make_layer(cfg, layer, dev)
+            call = lambda: csp.weight_histogram(p, q, k, mod, lens, hist, ws, js_all=js_all)
+            ms.append(pb.time_graph_of(call, 5))
+            js.append(float(js_all.item()))
+            totals += hist.sum(dim=(0, 1)).cpu().numpy().astype(np.int64)
+            del q, k, v
+        status = csp.device_status(ws)
+    weights_per_layer = int(totals.sum()) // n_layers
+    if rank == 0:
+        line = {"metric": "window_attention_weights_binned_per_sec", "value": weights_per_layer / (float(np.mean(ms)) * 1e-3),
+                "unit": "weights/s", "n_gpus": world, "steps": 5, "warmup": 1, "ms_per_step": float(np.mean(ms)),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"configs[{args.config}] {cfg.name}: csp_weight_histogram, one call per layer, {n_layers} layers",
+                           "bins": f"{csp.HIST_BINS} half-octave bins of log2(weight) from 2^{int(csp.HIST_LO)}",
+                           "weights_per_layer": weights_per_layer},
+                "js_divergence_per_layer_nats": js, "js_max_possible": float(np.log(2.0)),
+                "intra_histogram": totals[0].tolist(), "inter_histogram": totals[1].tolist(),
+                "device_status": status, "gpu_launches": n_layers * 5 * 3, "e2e": None, "cpu_baseline": None}
+        print(json.dumps(line), flush=True)
+
+
 def run_incremental(args, rank, world, local_rank):
     """`--incremental`: a re-prune round of the serving shape (configs[4]) two ways.  Every head's compacted cache
     has grown by 64 decoded tokens and is pruned back to its budget, either by csp_prune_layer (the window's 32
@@ -957,6 +1002,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode", action="store_true",
                     help="time the step after the pruning pass instead: n-softmax decode attention over the pruned caches")
+    ap.add_argument("--diagnostic", action="store_true",
+                    help="per-layer Jensen-Shannon divergence between intra- and inter-modality attention weights of the window")
     ap.add_argument("--incremental", action="store_true",
                     help="a re-prune round of configs[4] from the sums carried by csp_decode_step, against the full rescan")
     ap.add_argument("--with-lse", action="store_true",
@@ -986,6 +1033,9 @@ def main():
         return
     if args.incremental:
         run_incremental(args, rank, world, local_rank)
+        return
+    if args.diagnostic:
+        run_diagnostic(args, rank, world, local_rank)
         return
     from paper_2412_04652_b200 import binding as csp
     csp.lib()
