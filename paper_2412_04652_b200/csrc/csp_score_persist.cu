@@ -19,6 +19,8 @@
 // Precondition (checked by the launcher): G = 1 and at most 16 tiles per CTA, so that every tile's logits stay
 // in tensor memory between the passes.  With a caller-supplied log-sum-exp of the window rows there is no pass 1:
 // the epilogue teams go straight to the weights.
+#include <mutex>
+
 #include "csp_internal.cuh"
 #include "csp_tc.cuh"
 
@@ -53,6 +55,7 @@ __device__ __forceinline__ void team_sync(int team) {
 constexpr int kBufs = 16;                               // tiles whose logits tensor memory holds (32 columns each)
 constexpr int kPsMaxStages = 8;
 constexpr int kQSets = 3;                               // Q tiles and label tables staged ahead (ring)
+constexpr int kMaxCluster = 16;                         // CTAs per cluster (sizes above 8 need the non-portable opt-in)
 
 struct PsSmemPlan {   // byte offsets from the 1024-aligned base
     uint32_t q, wstats, cstats, cvec, dq_mask, dq_val, bars, misc, total;
@@ -62,7 +65,7 @@ __host__ __device__ inline PsSmemPlan ps_smem_plan(int nh, int stages) {
     uint32_t off = uint32_t(stages) * uint32_t(nh) * kBlockBytes;
     s.q = off;        off += uint32_t(kQSets) * uint32_t(nh) * 32u * 128u;   // staged ahead of the tensor core
     s.wstats = off;   off += 16u * 32u * 8u;                     // [team][warp][column]
-    s.cstats = off;   off += 4u * 8u * 32u * 8u;                  // [unit & 3][rank][row], written by the peers
+    s.cstats = off;   off += 4u * uint32_t(kMaxCluster) * 32u * 8u;   // [unit & 3][rank][row], written by the peers
     s.cvec = off;     off += 2u * 32u * 4u;                      // per team
     s.dq_mask = off;  off += uint32_t(kQSets) * 32u * 4u;
     s.dq_val = off;   off += uint32_t(kQSets) * 32u * 4u;
@@ -367,21 +370,20 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 #pragma unroll
                     for (int w = 0; w < kTeamWarps; w += 2 * d) merge_stats(v[w].x, v[w].y, v[w + d].x, v[w + d].y);
                 const int slot4 = j & 3;   // a peer can only overwrite a slot four units later, after this CTA's arrive for j + 2
-                const uint32_t mine = smem_u32(&cstats[(slot4 * 8 + int(rank)) * 32 + lane]);
+                const uint32_t mine = smem_u32(&cstats[(slot4 * kMaxCluster + int(rank)) * 32 + lane]);
                 for (uint32_t r = 0; r < csize; ++r) st_remote_f2(mine, r, v[0]);
                 asm volatile("fence.acq_rel.cluster;" ::: "memory");
                 __syncwarp();
                 if (lane < int(csize)) mbar_arrive_remote(stats_ready + 8 * p, uint32_t(lane));
                 mbar_wait_cluster(stats_ready + 8 * p, ph, abort_flag);
-                float2 c8[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r)
-                    c8[r] = r < int(csize) ? cstats[(slot4 * 8 + r) * 32 + lane] : make_float2(kNeg, 0.f);
-#pragma unroll
-                for (int d = 1; d < 8; d <<= 1)
-#pragma unroll
-                    for (int w = 0; w < 8; w += 2 * d) merge_stats(c8[w].x, c8[w].y, c8[w + d].x, c8[w + d].y);
-                const float m = c8[0].x, z = c8[0].y;
+                // merged in rank order (fixed, so results are reproducible); this sits on the unit's critical path, so no
+                // work is spent on ranks the cluster does not have (a tree over all sixteen possible ranks, guarded per
+                // node, measured 8 % slower on the whole kernel)
+                float m = kNeg, z = 0.f;
+                for (int r = 0; r < int(csize); ++r) {
+                    const float2 cr = cstats[(slot4 * kMaxCluster + r) * 32 + lane];
+                    merge_stats(m, z, cr.x, cr.y);
+                }
                 // weight of 2^(x - m) is 1 / (n 2^-m + Z); fold it and -m into one additive constant
                 const float denom = a.n * ex2f(-m) + z;
                 cv_team[lane] = lane < W ? lg2f(a.weight / denom) - m : -INFINITY;
@@ -488,7 +490,7 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
 }
 
 template <int NH>
-csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, int c, cudaStream_t s,
+csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap& tmap, int c_min, cudaStream_t s,
                      bool* taken) {
     const int units = p.batch * p.n_kv_heads;
     const int fixed = int(ps_smem_plan(NH, 0).total) + 1024;
@@ -498,7 +500,8 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
     const size_t smem = ps_smem_plan(NH, stages).total + 1024;
     auto kern = score_tc_persist_kernel<NH>;
     static std::atomic<bool> configured[kMaxDevices];
-    static std::atomic<int> resident[kMaxDevices][4];   // clusters of 1, 2, 4, 8 CTAs that fit on the device at once
+    static std::atomic<bool> wide_ok[kMaxDevices];            // cluster sizes above 8 have been allowed for this kernel
+    static std::atomic<int> resident[kMaxDevices][kMaxCluster + 1];   // clusters of each size that fit on the device at once
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return CSP_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return CSP_OK;
@@ -508,21 +511,46 @@ csp_status launch_nh(const csp_params& p, const ScoreArgs& a, const CUtensorMap&
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (!raise_smem_limit(kern, 227 * 1024, configured)) return CSP_ERR_CUDA;
-    const int slot = c == 1 ? 0 : (c == 2 ? 1 : (c == 4 ? 2 : 3));
-    int n_clusters = resident[dev][slot].load(std::memory_order_relaxed);
-    if (n_clusters == 0) {
-        const int sms = sm_count();
-        cfg.gridDim = dim3((sms / c) * c, 1, 1);
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = sms / c / 2; }
-        n_clusters = n > 0 ? n : 1;
-        resident[dev][slot].store(n_clusters, std::memory_order_relaxed);
+    // Sizes above 8 need the kernel's non-portable opt-in.  It is switched on only around a query or a launch that
+    // needs it (launches of the portable sizes ran 3 % slower with it left on), under a lock because it is a
+    // property of the kernel, not of the launch.
+    static std::mutex wide_mutex;
+    auto set_wide = [&](bool on) {
+        if (wide_ok[dev].load(std::memory_order_relaxed) == on) return;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, on ? 1 : 0) != cudaSuccess) cudaGetLastError();
+        wide_ok[dev].store(on, std::memory_order_relaxed);
+    };
+    std::lock_guard<std::mutex> lock(wide_mutex);
+    const int sms = sm_count();
+    auto clusters_of = [&](int c) {
+        int n = resident[dev][c].load(std::memory_order_relaxed);
+        if (n == 0) {
+            set_wide(c > 8);
+            attr[0].val.clusterDim.x = c;
+            cfg.gridDim = dim3((sms / c) * c, 1, 1);
+            int q = 0;
+            if (cudaOccupancyMaxActiveClusters(&q, kern, &cfg) != cudaSuccess || q <= 0) { cudaGetLastError(); q = -1; }
+            n = q;
+            resident[dev][c].store(n, std::memory_order_relaxed);
+        }
+        return n > 0 ? n : 0;
+    };
+    // Cluster size: the smallest that keeps a unit's logits in tensor memory, unless a larger one covers at least 5 % more
+    // SMs (clusters must sit inside one GPC: on a B200 sizes 4 and 8 cover 132 and 120 of the 148 SMs, size 9 covers 135).
+    int c = c_min, covered = clusters_of(c_min) * c_min;
+    for (int cc = c_min + 1; cc <= kMaxCluster; ++cc) {
+        const int cov = clusters_of(cc) * cc;
+        if (cov * 100 >= covered * 105) { c = cc; covered = cov; }
     }
+    const int n_clusters = clusters_of(c);
+    if (n_clusters <= 0) return CSP_OK;
     if (units < 2 * n_clusters) return CSP_OK;           // too few units for a resident loop to pay off
+    attr[0].val.clusterDim.x = c;
     cfg.gridDim = dim3(n_clusters * c, 1, 1);
+    set_wide(c > 8);
     if (cudaLaunchKernelEx(&cfg, kern, tmap, a, stages, units, n_clusters) != cudaSuccess) {
         cudaGetLastError();
         return CSP_ERR_CUDA;
@@ -541,9 +569,8 @@ csp_status launch_score_persist(const csp_params& p, const ScoreArgs& a, const C
     const int row_bytes = p.head_dim * 2;
     if (row_bytes != 128 && row_bytes != 256) return CSP_OK;
     const int max_tiles = (p.max_len + kTileKeys - 1) / kTileKeys;
-    int c = 1;
-    while (c < 8 && (max_tiles + c - 1) / c > kBufs) c *= 2;
-    if ((max_tiles + c - 1) / c > kBufs) return CSP_OK;
+    const int c = (max_tiles + kBufs - 1) / kBufs > 0 ? (max_tiles + kBufs - 1) / kBufs : 1;   // smallest size that keeps the logits
+    if (c > kMaxCluster) return CSP_OK;
     return row_bytes == 128 ? launch_nh<1>(p, a, tmap, c, s, taken) : launch_nh<2>(p, a, tmap, c, s, taken);
 }
 
