@@ -83,6 +83,37 @@ def test_null_misaligned_and_small_workspace(csp):
                              None, None, None, None, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
 
 
+def test_later_entry_points_reject_bad_arguments_on_the_host(csp):
+    """The decode step, the histogram diagnostic, the paged decode call and the probe check their arguments before
+    any CUDA call, so the refusals are the same with and without a device."""
+    p = csp.Params(1, 8, 4, 128, 1, 0, 512, 512)
+    cp = p.c()
+    good = csp.CTensor(4096, 4 * 512 * 128, 512 * 128, 128)
+    l = csp.lib()
+    # csp_decode_step: a missing label array, then a workspace that is too small
+    assert l.csp_decode_step(C.byref(cp), good, good, good, 256, None, 0, 0, 256, 1, 256, 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    assert l.csp_decode_step(C.byref(cp), good, good, good, 256, 256, 0, 0, 256, 1, 256, 256, 256, 256, 64, None) == csp.ERR_WORKSPACE
+    n = csp.lib().csp_decode_step_workspace_bytes(C.byref(cp))
+    assert n > csp.decode_workspace_bytes(p) > 0
+    # csp_weight_histogram: no histogram array; fp32 caches are not supported
+    ps = csp.Params(1, 8, 4, 128, 32, 32, 512, 128)
+    cps = ps.c()
+    assert l.csp_weight_histogram(C.byref(cps), good, good, 256, 0, 0, 256, None, None, None, None, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    pf = csp.Params(1, 8, 4, 64, 32, 32, 512, 128, dtype=csp.F32)
+    cpf = pf.c()
+    assert l.csp_weight_histogram(C.byref(cpf), good, good, 256, 0, 0, 256, None, 256, None, None, 256, 1 << 30, None) == csp.ERR_UNSUPPORTED
+    # csp_decode_attn_paged: pages that do not hold whole 128-key tiles, a table that does not cover the capacity
+    bad_rows = csp.CPages(256, 8, 64, 16)
+    assert l.csp_decode_attn_paged(C.byref(cp), good, good, good, C.byref(bad_rows), 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    short_table = csp.CPages(256, 2, 128, 16)
+    assert l.csp_decode_attn_paged(C.byref(cp), good, good, good, C.byref(short_table), 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    assert l.csp_decode_attn_paged(C.byref(cp), good, good, good, None, 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    # csp_probe_ex2_rate: iteration count out of range
+    out = C.c_int64(0)
+    assert l.csp_probe_ex2_rate(0, 0, None, 0, C.byref(out), None) == csp.ERR_INVALID_ARG
+    assert l.csp_probe_ex2_rate(0, 1 << 21, None, 0, C.byref(out), None) == csp.ERR_INVALID_ARG
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
 def test_without_a_gpu_the_path_fails_loudly(csp):
     """There is no CPU fallback: with valid arguments and no device the call reports an error."""
