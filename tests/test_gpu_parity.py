@@ -838,3 +838,50 @@ def test_config4_reprune_rounds(csp, oracle, budget_pct):
             assert_scores_close(run.sc[b:b + 1, h:h + 1, :L].cpu().numpy(), ref["score_cross"], [L], R)
             assert_index_sets_match(run.idx[b:b + 1, h:h + 1].cpu().numpy(), run.n_out[b:b + 1, h:h + 1].cpu().numpy(),
                                     ref, mod2[b:b + 1, h:h + 1, :L].cpu().numpy(), [L], R)
+
+
+# ------------------------------------------------------------------ a seeded sweep over shapes and modes
+
+@pytest.mark.parametrize("seed", range(24))
+def test_seeded_sweep_of_shapes_and_modes(csp, oracle, seed):
+    """Random (seeded) combinations of group size, head_dim, window, recent size, batch raggedness, budgets, selection
+    and combination mode, labels shared or per head, mixed-modality windows, n: the whole pass against the oracle."""
+    rng = np.random.RandomState(1000 + seed)
+    G = int(rng.choice([1, 1, 2, 3, 4, 7, 8]))
+    n_kv = int(rng.choice([1, 2, 3]))
+    d = int(rng.choice([64, 128]))
+    W = int(rng.choice([1, 7, 16, 32]))
+    R = int(rng.choice([0, 5, W, 40]))
+    B = int(rng.randint(1, 5))
+    lens = tuple(int(x) for x in rng.randint(max(W, R, 41) + 1, 1400, size=B))
+    cfg = _case(lens, G * n_kv, n_kv, d, W, R, seed=seed, visual_pct=int(rng.randint(5, 90)), text_pct=int(rng.randint(5, 90)))
+    mode = dict(select_mode=int(rng.choice([0, 0, 1, 2])), combine=int(rng.choice([0, 0, 1])))
+    n = float(rng.choice([0.0, 1.0, 1.0, 30.0]))
+    per_head = bool(rng.randint(2))
+    mod = cfg.modality()
+    if per_head:
+        mod = np.repeat(mod[:, None, :], n_kv, axis=1).copy()
+        mod[:, :, :] ^= (rng.rand(B, n_kv, cfg.max_len) < 0.1).astype(np.uint8)     # heads differ in a tenth of the labels
+    if rng.randint(2):                                                              # a mixed-modality window
+        for b, L in enumerate(lens):
+            mod[b, ..., L - W:L] = (rng.rand(W) < 0.4).astype(np.uint8)
+    nb = {0: 4, 1: 2, 2: 1}[mode["select_mode"]]
+    budgets = rng.randint(0, max(2, min(lens) // 3), size=(B, nb)).astype(np.int32)
+    total = rng.randint(0, 1500, size=B).astype(np.int32) if rng.randint(3) == 0 else None
+    cap = int(max(lens))
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    if rng.randint(3) == 0:
+        q = (q.float() * 4.0).to(cfg.dtype)                                         # peaked rows
+    p = gpu_params(csp, cfg, cap=cap, n=n, **mode)
+    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, budgets, total_budget=total).prune()
+    ref = oracle.prune_layer(orc_params(oracle, cfg, cap=cap, n=n, **mode), q.cpu(), k.cpu(), v.cpu(), mod, cfg.seq_lens,
+                             budgets, total)
+    assert run.status() & ~csp.DEV_K_CLAMPED == 0
+    assert_scores_close(run.ss.cpu().numpy(), ref["score_self"], cfg.seq_lens, R, "self")
+    assert_scores_close(run.sc.cpu().numpy(), ref["score_cross"], cfg.seq_lens, R, "cross")
+    assert_index_sets_match(run.idx.cpu().numpy(), run.n_out.cpu().numpy(), ref, mod, cfg.seq_lens, R,
+                            global_mode=mode["select_mode"] == 1, overall=mode["select_mode"] == 2)
+    assert_selection_follows_own_scores(oracle, orc_params(oracle, cfg, cap=cap, n=n, **mode), run.ss.cpu().numpy(),
+                                        run.sc.cpu().numpy(), run.idx.cpu().numpy(), run.n_out.cpu().numpy(), mod,
+                                        cfg.seq_lens, budgets, total)
+    assert_compaction_exact(run, mod)
