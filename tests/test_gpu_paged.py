@@ -1,6 +1,8 @@
 """GPU parity of csp_prune_layer_paged: the pass on a cache whose rows live in pages of a pool.  Paging changes
-addressing only, so the result must be bit-identical to the dense entry point on the same rows, and it is compared
-with the CPU oracle (run on the dense rows) under the tolerances of the pass."""
+addressing only, so the result must be bit-identical to the dense entry point on the same rows whenever both launches
+see the same number of key tiles (the page table pads the logical length to whole pages; a different tile count can
+change the cluster size and with it the order in which row statistics are merged: scores then agree to fp32 rounding,
+about 2e-7 relative).  It is also compared with the CPU oracle (run on the dense rows) under the tolerances of the pass."""
 import numpy as np
 import pytest
 import torch
@@ -77,9 +79,14 @@ def test_paged_prune_matches_the_dense_one_and_the_oracle(csp, oracle, lens, n_q
     assert paged.status() == 0
     assert torch.equal(paged.n_out, dense.n_out) and torch.equal(paged.idx, dense.idx)
     B, H = cfg.batch, cfg.n_kv_heads
+    same_tiles = (pp.max_len + 127) // 128 == (cfg.max_len + 127) // 128
     for b in range(B):
         N = int(cfg.seq_lens[b]) - 32
-        assert torch.equal(paged.ss[b, :, :N], dense.ss[b, :, :N]) and torch.equal(paged.sc[b, :, :N], dense.sc[b, :, :N])
+        if same_tiles:
+            assert torch.equal(paged.ss[b, :, :N], dense.ss[b, :, :N]) and torch.equal(paged.sc[b, :, :N], dense.sc[b, :, :N])
+        else:
+            torch.testing.assert_close(paged.ss[b, :, :N], dense.ss[b, :, :N], rtol=2e-6, atol=0)
+            torch.testing.assert_close(paged.sc[b, :, :N], dense.sc[b, :, :N], rtol=2e-6, atol=0)
         for h in range(H):
             n = int(dense.n_out[b, h])
             assert torch.equal(paged.k_out[b, h, :n], dense.k_out[b, h, :n])
