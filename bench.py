@@ -140,7 +140,8 @@ def algorithmic_bytes(cfg, lens, n_out_total: int, labels_per_head: bool = False
     score = sum_l * Hkv * d * es + len(lens) * Hq * W * d * es + labels + 2 * 4 * sum_n * Hkv
     select = 2 * 4 * sum_n * Hkv + sum_n * Hkv + 4 * n_out_total
     compact = 4 * n_out_total + 2 * 2 * n_out_total * d * es + 2 * n_out_total
-    return {"score": score, "select": select, "compact": compact, "total": score + select + compact}
+    return {"score": score, "select": select, "compact": compact, "select_compact": select + compact,
+            "total": score + select + compact}
 
 
 class LayerBuffers:
@@ -238,12 +239,19 @@ def run_reference(args, rank, world):
 
 # ------------------------------------------------------------------------------------ CUDA arm
 
+def fused_select_compact(p, sms) -> bool:
+    """Whether csp_select_compact runs as one persistent kernel for dense, contiguous outputs in a second buffer (what
+    this file passes): at least two units per SM and caches of 2 K - 8 K positions."""
+    return p.batch * p.n_kv_heads >= 2 * sms and 2048 < p.max_len <= 8192 and p.out_capacity > 0
+
+
 def kernels_per_call(p, sms) -> int:
-    """Kernels one csp_prune_layer call launches: score, select, compact, and, for a bf16 cache with more
-    (sequence, head) units than SMs and several sequences, the kernel that orders them by length."""
+    """Kernels one csp_prune_layer call launches: score, select and compact (one kernel where they are fused), and,
+    for a bf16 cache with more (sequence, head) units than SMs and several sequences, the kernel that orders them by
+    length."""
     units, tiles = p.batch * p.n_kv_heads, (p.max_len + 127) // 128
     ordered = p.dtype == 1 and 2 <= p.batch <= 4096 and (units > sms or units * min(tiles, 8) > sms * 13 // 16)
-    return 4 if ordered else 3
+    return (4 if ordered else 3) - (1 if fused_select_compact(p, sms) else 0)
 
 
 class PathBench:
@@ -389,9 +397,17 @@ class PathBench:
                 for c in calls:
                     csp.compact(c.p, c.lb.k, c.lb.v, c.mod, c.lb.idx, c.lb.n_out, c.lb.k_out, c.lb.v_out, c.lb.mod_out)
 
+            def select_compact_all():
+                for c in calls:
+                    csp.select_compact(c.p, c.lb.ss, c.lb.sc, c.lb.k, c.lb.v, c.mod, c.lens, c.bud, c.lb.k_out, c.lb.v_out,
+                                       c.lb.mod_out, c.lb.n_out, ws, total_budget=c.tot, keep_idx=c.lb.idx)
+
             per = {}
             reps = max(3, min(50, args.steps))
-            for name, fn in (("score", score_all), ("select", select_all), ("compact", compact_all)):
+            stages = [("score", score_all), ("select", select_all), ("compact", compact_all)]
+            if any(fused_select_compact(c.p, self.sms) for c in calls):
+                stages.append(("select_compact", select_compact_all))     # what the step runs instead of the two
+            for name, fn in stages:
                 per[name] = self.time_graph_of(fn, reps) / len(calls)                # ms per launch
             status |= csp.device_status(ws)
 
@@ -1012,7 +1028,7 @@ def main():
     ap.add_argument("--budget-pct", type=int, default=20, help="budget of configs[4]")
     ap.add_argument("--rounds", type=int, default=4, help="re-prune rounds of configs[4] under --all-configs")
     ap.add_argument("--all-configs", action="store_true",
-                    help="one JSON line per workload 1-4; for 4, every budget of {5,10,20,40} % with round 0, "
+                    help="one JSON line per workload 1-4; for 4, every budget of {5,10,20,40} %% with round 0, "
                          "rounds 1-4 and their total (not the default: takes several minutes)")
     args = ap.parse_args()
 

@@ -168,8 +168,25 @@ csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v,
                        csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, void* cuda_stream);
 
 /*
- * Algorithm 1, one invocation for one layer: csp_score, csp_select, csp_compact back to back on
- * one stream.  score_self / score_cross / keep_idx may be NULL, in which case they live in the
+ * csp_select followed by csp_compact on the same stream (Eq. 2-4), for a caller that already has the two score
+ * vectors (from csp_score, or carried along by csp_decode_step).  Same arguments, results and flags as the two
+ * calls; keep_idx may be NULL, in which case the list lives in the workspace.  With several hundred units whose
+ * caches hold 2 K - 8 K positions, a second (not in-place) output buffer and contiguous output rows
+ * (stride_t == head_dim), both steps run in one persistent kernel in which the selection of later units overlaps
+ * the copy of earlier ones; otherwise as two kernels.  The results do not depend on which.
+ */
+csp_status csp_select_compact(const csp_params* p, const float* score_self, const float* score_cross,
+                              csp_tensor k, csp_tensor v,
+                              const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                              const int32_t* seq_lens, const int32_t* budgets,
+                              const int32_t* total_budget_or_null,
+                              csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
+                              int32_t* keep_idx_or_null,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 1, one invocation for one layer: csp_score, then csp_select_compact, on one stream.
+ * score_self / score_cross / keep_idx may be NULL, in which case they live in the
  * workspace; n_out is required.
  */
 csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,

@@ -28,7 +28,7 @@ EXPORTS = ("csp_workspace_bytes", "csp_workspace_reset", "csp_score", "csp_selec
            "csp_status_string", "csp_prune_layer_static", "csp_static_workspace_limit",
            "csp_decode_workspace_bytes", "csp_decode_attn", "csp_decode_step_workspace_bytes", "csp_decode_step",
            "csp_weight_histogram", "csp_probe_ex2_rate", "csp_prune_layer_paged",
-           "csp_decode_attn_paged")
+           "csp_decode_attn_paged", "csp_select_compact")
 HIST_BINS, HIST_LO, HIST_WIDTH = 64, -32.0, 0.5
 
 
@@ -105,6 +105,9 @@ def lib() -> C.CDLL:
         l.csp_select.argtypes = [P, vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         l.csp_compact.restype = C.c_int
         l.csp_compact.argtypes = [P, CTensor, CTensor, vp, i64, i64, vp, vp, CTensor, CTensor, vp, vp]
+        l.csp_select_compact.restype = C.c_int
+        l.csp_select_compact.argtypes = [P, vp, vp, CTensor, CTensor, vp, i64, i64, vp, vp, vp, CTensor, CTensor, vp, vp,
+                                         vp, vp, sz, vp]
         l.csp_prune_layer.restype = C.c_int
         l.csp_prune_layer.argtypes = [P, CTensor, CTensor, CTensor, vp, i64, i64, vp, vp, vp, vp,
                                       CTensor, CTensor, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -277,6 +280,16 @@ def compact(p: Params, k, v, modality, keep_idx, n_out, k_out, v_out, mod_out=No
     _check(lib().csp_compact(C.byref(cp), tensor4(k), tensor4(v), _ptr(modality), sb, sh, _ptr(keep_idx),
                              _ptr(n_out), tensor4(k_out), tensor4(v_out), _ptr(mod_out), _stream()),
            "csp_compact")
+
+
+def select_compact(p: Params, score_self, score_cross, k, v, modality, seq_lens, budgets, k_out, v_out, mod_out, n_out,
+                   ws, total_budget=None, keep_idx=None):
+    cp = p.c()
+    sb, sh = _mod_strides(modality)
+    _check(lib().csp_select_compact(C.byref(cp), _ptr(score_self), _ptr(score_cross), tensor4(k), tensor4(v),
+                                    _ptr(modality), sb, sh, _ptr(seq_lens), _ptr(budgets), _ptr(total_budget),
+                                    tensor4(k_out), tensor4(v_out), _ptr(mod_out), _ptr(n_out), _ptr(keep_idx),
+                                    _ptr(ws), ws.numel(), _stream()), "csp_select_compact")
 
 
 def prune_layer(p: Params, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, mod_out, n_out, ws,

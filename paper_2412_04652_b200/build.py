@@ -12,7 +12,7 @@ INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 LIB = os.path.join(PKG, "libcsp.so")
 OBJ_DIR = os.path.join(PKG, "_build")
 SOURCES = ["csp_api.cu", "csp_score.cu", "csp_score_tc.cu", "csp_score_persist.cu", "csp_select.cu", "csp_select_cluster.cu",
-           "csp_compact.cu", "csp_decode.cu", "csp_static.cu"]
+           "csp_compact.cu", "csp_select_compact.cu", "csp_decode.cu", "csp_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

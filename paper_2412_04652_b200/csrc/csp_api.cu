@@ -82,10 +82,10 @@ csp_status do_score(const csp_params& p, const csp_tensor& q, const csp_tensor& 
     return st;
 }
 
-csp_status do_select(const csp_params& p, const float* score_self, const float* score_cross,
-                     const uint8_t* modality, int64_t msb, int64_t msh, const int32_t* seq_lens,
-                     const int32_t* budgets, const int32_t* total_budget, int32_t* keep_idx, int32_t* n_out,
-                     void* ws, cudaStream_t stream) {
+SelectArgs select_args(const csp_params& p, const float* score_self, const float* score_cross,
+                       const uint8_t* modality, int64_t msb, int64_t msh, const int32_t* seq_lens,
+                       const int32_t* budgets, const int32_t* total_budget, int32_t* keep_idx, int32_t* n_out,
+                       void* ws) {
     SelectArgs a;
     a.score_self = score_self; a.score_cross = score_cross;
     a.modality = modality; a.mod_sb = msb; a.mod_sh = msh;
@@ -97,13 +97,21 @@ csp_status do_select(const csp_params& p, const float* score_self, const float* 
     // OVERALL runs as GLOBAL with both problems on the summed score and the same budget: their union is the one top-K
     a.overall = p.select_mode == CSP_SELECT_OVERALL;
     a.global_mode = p.select_mode == CSP_SELECT_GLOBAL || a.overall;
-    return launch_select(p, a, stream);
+    return a;
 }
 
-csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor& v, const uint8_t* modality,
-                      int64_t msb, int64_t msh, const int32_t* keep_idx, const int32_t* n_out,
-                      const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, int32_t* status,
-                      cudaStream_t stream, const csp_pages* pages = nullptr) {
+csp_status do_select(const csp_params& p, const float* score_self, const float* score_cross,
+                     const uint8_t* modality, int64_t msb, int64_t msh, const int32_t* seq_lens,
+                     const int32_t* budgets, const int32_t* total_budget, int32_t* keep_idx, int32_t* n_out,
+                     void* ws, cudaStream_t stream) {
+    return launch_select(p, select_args(p, score_self, score_cross, modality, msb, msh, seq_lens, budgets, total_budget,
+                                        keep_idx, n_out, ws), stream);
+}
+
+CompactArgs compact_args(const csp_params& p, const csp_tensor& k, const csp_tensor& v, const uint8_t* modality,
+                         int64_t msb, int64_t msh, const int32_t* keep_idx, const int32_t* n_out,
+                         const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, int32_t* status,
+                         const csp_pages* pages) {
     const int64_t es = elem_size(p);
     CompactArgs a;
     a.k = k.ptr; a.v = v.ptr; a.k_out = k_out.ptr; a.v_out = v_out.ptr;
@@ -120,7 +128,34 @@ csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor
     a.max_pages = pages ? pages->max_pages : 0;
     a.page_rows = pages ? pages->page_rows : 1;
     a.n_pages = pages ? pages->n_pages : 0;
-    return launch_compact(p, a, stream);
+    return a;
+}
+
+csp_status do_compact(const csp_params& p, const csp_tensor& k, const csp_tensor& v, const uint8_t* modality,
+                      int64_t msb, int64_t msh, const int32_t* keep_idx, const int32_t* n_out,
+                      const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out, int32_t* status,
+                      cudaStream_t stream, const csp_pages* pages = nullptr) {
+    return launch_compact(p, compact_args(p, k, v, modality, msb, msh, keep_idx, n_out, k_out, v_out, mod_out, status,
+                                          pages), stream);
+}
+
+// Selection and compaction of one call: the fused persistent kernel where the shape qualifies (many units whose
+// selection fits one CTA, dense second output buffers), else the two kernels one after the other.
+csp_status do_select_compact(const csp_params& p, const float* ss, const float* sc, const csp_tensor& k,
+                             const csp_tensor& v, const uint8_t* modality, int64_t msb, int64_t msh,
+                             const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget,
+                             int32_t* idx, int32_t* n_out, const csp_tensor& k_out, const csp_tensor& v_out,
+                             uint8_t* mod_out, void* ws, cudaStream_t stream, bool allow_fused) {
+    const SelectArgs sa = select_args(p, ss, sc, modality, msb, msh, seq_lens, budgets, total_budget, idx, n_out, ws);
+    const CompactArgs ca = compact_args(p, k, v, modality, msb, msh, idx, n_out, k_out, v_out, mod_out,
+                                        static_cast<int32_t*>(ws), nullptr);
+    if (allow_fused) {
+        bool taken = false;
+        const csp_status st = launch_select_compact(p, sa, ca, stream, &taken);
+        if (st != CSP_OK || taken) return st;
+    }
+    const csp_status st = launch_select(p, sa, stream);
+    return st != CSP_OK ? st : launch_compact(p, ca, stream);
 }
 
 }  // namespace
@@ -155,6 +190,34 @@ csp_status check_prune_layer_args(const csp_params* p, const csp_tensor& q_win, 
         return CSP_ERR_UNSUPPORTED;
     return check_arch();
 }
+
+namespace {
+// csp_prune_layer; `v_on_device` is false when V is page-locked host memory read over the bus, which keeps the
+// compaction kernel with many small CTAs (more requests in flight than one resident CTA per SM has)
+csp_status prune_layer_impl(const csp_params* p, const csp_tensor& q_win, const csp_tensor& k, const csp_tensor& v,
+                            const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                            const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget_or_null,
+                            const float* lse_or_null, const csp_tensor& k_out, const csp_tensor& v_out, uint8_t* mod_out,
+                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
+                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                            bool v_on_device) {
+    csp_status st = check_prune_layer_args(p, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, n_out);
+    if (st != CSP_OK) return st;
+    if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
+    const WorkspaceLayout wl = workspace_layout(*p);
+    char* ws = static_cast<char*>(workspace);
+    float* ss = score_self_or_null ? score_self_or_null : reinterpret_cast<float*>(ws + wl.score_self);
+    float* sc = score_cross_or_null ? score_cross_or_null : reinterpret_cast<float*>(ws + wl.score_cross);
+    int32_t* idx = keep_idx_or_null ? keep_idx_or_null : reinterpret_cast<int32_t*>(ws + wl.keep_idx);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if ((st = do_score(*p, q_win, k, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null, ss, sc,
+                       workspace, stream)) != CSP_OK)
+        return st;
+    return do_select_compact(*p, ss, sc, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets,
+                             total_budget_or_null, idx, n_out, k_out, v_out, mod_out, workspace, stream, v_on_device);
+}
+
+}  // namespace
 
 }  // namespace csp
 
@@ -219,6 +282,26 @@ csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v, const ui
                       nullptr, static_cast<cudaStream_t>(cuda_stream));
 }
 
+csp_status csp_select_compact(const csp_params* p, const float* score_self, const float* score_cross, csp_tensor k,
+                              csp_tensor v, const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
+                              const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget_or_null,
+                              csp_tensor k_out, csp_tensor v_out, uint8_t* mod_out, int32_t* n_out,
+                              int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    csp_status st = check_params(p);
+    if (st != CSP_OK) return st;
+    if (!score_self || !score_cross || !modality || !seq_lens || !budgets || !n_out || !k.ptr || !v.ptr || !k_out.ptr ||
+        !v_out.ptr)
+        return CSP_ERR_INVALID_ARG;
+    if (!tensor_ok(*p, k) || !tensor_ok(*p, v) || !tensor_ok(*p, k_out) || !tensor_ok(*p, v_out)) return CSP_ERR_UNSUPPORTED;
+    if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
+    if ((st = check_arch()) != CSP_OK) return st;
+    int32_t* idx = keep_idx_or_null ? keep_idx_or_null
+                                    : reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + workspace_layout(*p).keep_idx);
+    return do_select_compact(*p, score_self, score_cross, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets,
+                             total_budget_or_null, idx, n_out, k_out, v_out, mod_out, workspace,
+                             static_cast<cudaStream_t>(cuda_stream), true);
+}
+
 csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, csp_tensor v,
                            const uint8_t* modality, int64_t mod_stride_b, int64_t mod_stride_h,
                            const int32_t* seq_lens, const int32_t* budgets, const int32_t* total_budget_or_null,
@@ -226,23 +309,9 @@ csp_status csp_prune_layer(const csp_params* p, csp_tensor q_win, csp_tensor k, 
                            int32_t* n_out, float* score_self_or_null, float* score_cross_or_null,
                            int32_t* keep_idx_or_null, void* workspace, size_t workspace_bytes,
                            void* cuda_stream) {
-    csp_status st = check_prune_layer_args(p, q_win, k, v, modality, seq_lens, budgets, k_out, v_out, n_out);
-    if (st != CSP_OK) return st;
-    if ((st = check_workspace(*p, workspace, workspace_bytes)) != CSP_OK) return st;
-    const WorkspaceLayout wl = workspace_layout(*p);
-    char* ws = static_cast<char*>(workspace);
-    float* ss = score_self_or_null ? score_self_or_null : reinterpret_cast<float*>(ws + wl.score_self);
-    float* sc = score_cross_or_null ? score_cross_or_null : reinterpret_cast<float*>(ws + wl.score_cross);
-    int32_t* idx = keep_idx_or_null ? keep_idx_or_null : reinterpret_cast<int32_t*>(ws + wl.keep_idx);
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if ((st = do_score(*p, q_win, k, modality, mod_stride_b, mod_stride_h, seq_lens, lse_or_null, ss, sc,
-                       workspace, stream)) != CSP_OK)
-        return st;
-    if ((st = do_select(*p, ss, sc, modality, mod_stride_b, mod_stride_h, seq_lens, budgets, total_budget_or_null,
-                        idx, n_out, workspace, stream)) != CSP_OK)
-        return st;
-    return do_compact(*p, k, v, modality, mod_stride_b, mod_stride_h, idx, n_out, k_out, v_out, mod_out,
-                      static_cast<int32_t*>(workspace), stream);
+    return prune_layer_impl(p, q_win, k, v, modality, mod_stride_b, mod_stride_h, seq_lens, budgets,
+                            total_budget_or_null, lse_or_null, k_out, v_out, mod_out, n_out, score_self_or_null,
+                            score_cross_or_null, keep_idx_or_null, workspace, workspace_bytes, cuda_stream, true);
 }
 
 // A page table must cover max_len positions with pages of whole 128-key tiles.
@@ -375,11 +444,12 @@ csp_status csp_prune_layer_host(const csp_params* p, const void* q_host, const v
     csp_tensor vo = {d + sl.v_out, ko.stride_b, ko.stride_h, d_};
     const int64_t msb = mod_per_head ? int64_t(p->n_kv_heads) * p->max_len : p->max_len;
     const int64_t msh = mod_per_head ? p->max_len : 0;
-    st = csp_prune_layer(p, q, k, v, reinterpret_cast<uint8_t*>(d + sl.mod), msb, msh,
-                         reinterpret_cast<int32_t*>(d + sl.seq), reinterpret_cast<int32_t*>(d + sl.bud),
-                         total_budget_host_or_null ? reinterpret_cast<int32_t*>(d + sl.tot) : nullptr, nullptr, ko, vo,
-                         reinterpret_cast<uint8_t*>(d + sl.mod_out), reinterpret_cast<int32_t*>(d + sl.n_out),
-                         nullptr, nullptr, nullptr, d + sl.ws, workspace_layout(*p).total, cuda_stream);
+    st = prune_layer_impl(p, q, k, v, reinterpret_cast<uint8_t*>(d + sl.mod), msb, msh,
+                          reinterpret_cast<int32_t*>(d + sl.seq), reinterpret_cast<int32_t*>(d + sl.bud),
+                          total_budget_host_or_null ? reinterpret_cast<int32_t*>(d + sl.tot) : nullptr, nullptr, ko, vo,
+                          reinterpret_cast<uint8_t*>(d + sl.mod_out), reinterpret_cast<int32_t*>(d + sl.n_out),
+                          nullptr, nullptr, nullptr, d + sl.ws, workspace_layout(*p).total, cuda_stream,
+                          v_mapped == nullptr);
     if (st != CSP_OK) return st;
     d2h(k_out_host, sl.k_out, out_bytes);
     d2h(v_out_host, sl.v_out, out_bytes);

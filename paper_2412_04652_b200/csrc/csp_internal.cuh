@@ -162,6 +162,8 @@ csp_status launch_select(const csp_params& p, const SelectArgs& a, cudaStream_t 
 constexpr int kSelectClusterMaxLen = 8 * 1024 * 8;   // longest cache the register-resident cluster select takes
 csp_status launch_select_cluster(const csp_params& p, const SelectArgs& a, cudaStream_t s);
 csp_status launch_compact(const csp_params& p, const CompactArgs& a, cudaStream_t s);
+csp_status launch_select_compact(const csp_params& p, const SelectArgs& sa, const CompactArgs& ca, cudaStream_t s,
+                                 bool* taken);
 
 // 4-D tensor map over a cache [batch, heads, rows, head_dim] with 128-byte swizzle and boxes of 128 bytes x
 // box_rows rows; false if the driver entry point is missing or the strides / alignment do not qualify.

@@ -885,3 +885,104 @@ def test_seeded_sweep_of_shapes_and_modes(csp, oracle, seed):
                                         run.sc.cpu().numpy(), run.idx.cpu().numpy(), run.n_out.cpu().numpy(), mod,
                                         cfg.seq_lens, budgets, total)
     assert_compaction_exact(run, mod)
+
+
+# ------------------------------------------------------------------ many units: selection and compaction in one kernel
+
+def _many_units_case(rng, seed, hi, n_kv, d, dtype=torch.bfloat16, G=1):
+    """A batch with at least 300 (sequence, KV head) units and caches of up to `hi` positions, a few of them short."""
+    B = -(-300 // n_kv) + int(rng.randint(0, 3))
+    lens = [int(x) for x in rng.randint(hi // 2, hi + 1, size=B)]
+    lens[0] = hi
+    lens[1] = int(rng.randint(60, 200))                  # a short cache in the same call
+    return _case(tuple(lens), G * n_kv, n_kv, d, 32, 32, dtype=dtype, seed=seed, visual_pct=int(rng.randint(5, 60)),
+                 text_pct=int(rng.randint(5, 60)))
+
+
+@pytest.mark.parametrize("seed,hi,n_kv,d,dtype", [
+    (0, 2100, 16, 128, torch.bfloat16), (1, 4096, 8, 128, torch.bfloat16), (2, 3000, 16, 64, torch.bfloat16),
+    (3, 8192, 8, 64, torch.bfloat16), (4, 5000, 8, 128, torch.bfloat16), (5, 2500, 8, 128, torch.float32)])
+def test_many_units_mid_length_caches(csp, oracle, seed, hi, n_kv, d, dtype):
+    """Launches that take the fused selection + compaction kernel (hundreds of units, caches of 2-8 K positions): the
+    whole pass against the oracle, and bit-identical to the three stages called one by one."""
+    rng = np.random.RandomState(7000 + seed)
+    cfg = _many_units_case(rng, seed, hi, n_kv, d, dtype)
+    mode = dict(select_mode=int(rng.choice([0, 0, 1, 2])), combine=int(rng.choice([0, 0, 1])))
+    nb = {0: 4, 1: 2, 2: 1}[mode["select_mode"]]
+    B = cfg.batch
+    budgets = rng.randint(0, hi // 6, size=(B, nb)).astype(np.int32)
+    total = rng.randint(0, hi, size=B).astype(np.int32) if seed % 2 else None     # some caches below their budget T
+    cap = int(budgets.sum(axis=1).max()) + 32 if total is None else hi
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    mod = cfg.modality()
+    p = gpu_params(csp, cfg, cap=cap, **mode)
+    run = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, budgets, total_budget=total).prune()
+    assert run.status() & ~csp.DEV_K_CLAMPED == 0
+    # the stages one by one, on the scores of the call above
+    step = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, budgets, total_budget=total)
+    step.ss.copy_(run.ss); step.sc.copy_(run.sc)
+    step.select().compact()
+    assert torch.equal(step.n_out, run.n_out)
+    # and csp_select_compact on those scores, without the optional index list
+    both = GpuRun(csp, p, q, k, v, mod, cfg.seq_lens, budgets, total_budget=total)
+    csp.select_compact(p, run.ss, run.sc, both.k, both.v, both.mod, both.lens, both.bud, both.k_out, both.v_out,
+                       both.mod_out, both.n_out, both.ws, total_budget=both.tot)
+    assert both.status() & ~csp.DEV_K_CLAMPED == 0
+    assert torch.equal(both.n_out, run.n_out) and torch.equal(both.k_out, run.k_out)
+    assert torch.equal(both.v_out, run.v_out) and torch.equal(both.mod_out, run.mod_out)
+    n_out = run.n_out.cpu().numpy()
+    assert (n_out >= 0).all()
+    for b in range(B):
+        for h in range(n_kv):
+            n = int(n_out[b, h])
+            assert torch.equal(step.idx[b, h, :n], run.idx[b, h, :n])
+            assert torch.equal(step.k_out[b, h, :n], run.k_out[b, h, :n])
+            assert torch.equal(step.v_out[b, h, :n], run.v_out[b, h, :n])
+            assert torch.equal(step.mod_out[b, h, :n], run.mod_out[b, h, :n])
+            assert (run.k_out[b, h, n:] == 0).all() and (run.mod_out[b, h, n:] == 0).all()    # nothing beyond the kept rows
+    assert_compaction_exact(run, mod)
+    # against the oracle: a sample of sequences (all their heads), always with the longest and the short one
+    pick = sorted({0, 1, *[int(x) for x in rng.choice(B, size=4, replace=False)]})
+    op = oracle.Params(len(pick), cfg.n_q_heads, n_kv, d, 32, 32, cfg.max_len, cap,
+                       dtype=oracle.F32 if dtype == torch.float32 else oracle.BF16, **mode)
+    pad = lambda t: t[pick].cpu()
+    ref = oracle.prune_layer(op, pad(q), pad(k), pad(v), mod[pick], cfg.seq_lens[pick], budgets[pick],
+                             None if total is None else total[pick])
+    lens = cfg.seq_lens[pick]
+    assert_scores_close(run.ss[pick].cpu().numpy(), ref["score_self"], lens, 32, "self")
+    assert_scores_close(run.sc[pick].cpu().numpy(), ref["score_cross"], lens, 32, "cross")
+    assert_index_sets_match(run.idx[pick].cpu().numpy(), n_out[pick], ref, mod[pick], lens, 32,
+                            global_mode=mode["select_mode"] == 1, overall=mode["select_mode"] == 2)
+    assert_selection_follows_own_scores(oracle, op, run.ss[pick].cpu().numpy(), run.sc[pick].cpu().numpy(),
+                                        run.idx[pick].cpu().numpy(), n_out[pick], mod[pick], lens, budgets[pick],
+                                        None if total is None else total[pick])
+
+
+def test_many_units_bad_length_and_capacity_are_flagged(csp, oracle):
+    """In a launch that takes the fused kernel: a length outside [0, max_len] gives -1 rows and DEV_BAD_LEN, a unit
+    whose kept rows exceed the capacity gives -1 rows and DEV_CAPACITY; the other units are unaffected; no label output."""
+    rng = np.random.RandomState(7100)
+    cfg = _many_units_case(rng, 9, 2600, 16, 128)
+    B = cfg.batch
+    budgets = np.full((B, 4), 40, np.int32)
+    budgets[2] = 400                                     # 1600 + 32 rows do not fit the capacity below
+    cap = 4 * 40 + 32
+    lens = cfg.seq_lens.copy()
+    lens[3] = cfg.max_len + 1
+    lens[4] = -5
+    q, k, v = synth.make_layer(cfg, 0, "cuda")
+    mod = cfg.modality()
+    p = gpu_params(csp, cfg, cap=cap)
+    run = GpuRun(csp, p, q, k, v, mod, lens, budgets)
+    run.csp.prune_layer(p, run.q, run.k, run.v, run.mod, run.lens, run.bud, run.k_out, run.v_out, None, run.n_out,
+                        run.ws, keep_idx=run.idx)
+    st = run.status()
+    assert st & csp.DEV_BAD_LEN and st & csp.DEV_CAPACITY and not st & csp.DEV_TIMEOUT
+    n_out = run.n_out.cpu().numpy()
+    assert (n_out[2] == -1).all() and (n_out[3] == -1).all() and (n_out[4] == -1).all()
+    good = [b for b in range(B) if b not in (2, 3, 4)]
+    assert (n_out[good] > 0).all()
+    assert (run.k_out[[2, 3, 4]] == 0).all()             # nothing written for the flagged units
+    assert (run.mod_out == 0).all()
+    run.n_out[[2, 3, 4]] = 0
+    assert_compaction_exact(run, np.zeros_like(mod))

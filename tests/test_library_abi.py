@@ -108,6 +108,14 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(csp):
     short_table = csp.CPages(256, 2, 128, 16)
     assert l.csp_decode_attn_paged(C.byref(cp), good, good, good, C.byref(short_table), 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
     assert l.csp_decode_attn_paged(C.byref(cp), good, good, good, None, 256, 256, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    # csp_select_compact: no row-count array, a misaligned output, a workspace that is too small
+    odd = csp.CTensor(4096 + 2, 4 * 512 * 128, 512 * 128, 128)
+    assert l.csp_select_compact(C.byref(cps), 256, 256, good, good, 256, 0, 0, 256, 256, None, good, good, None, None,
+                                None, 256, 1 << 30, None) == csp.ERR_INVALID_ARG
+    assert l.csp_select_compact(C.byref(cps), 256, 256, good, good, 256, 0, 0, 256, 256, None, good, odd, None, 256,
+                                None, 256, 1 << 30, None) == csp.ERR_UNSUPPORTED
+    assert l.csp_select_compact(C.byref(cps), 256, 256, good, good, 256, 0, 0, 256, 256, None, good, good, None, 256,
+                                None, 256, 64, None) == csp.ERR_WORKSPACE
     # csp_probe_ex2_rate: iteration count out of range
     out = C.c_int64(0)
     assert l.csp_probe_ex2_rate(0, 0, None, 0, C.byref(out), None) == csp.ERR_INVALID_ARG
