@@ -241,8 +241,8 @@ def run_reference(args, rank, world):
 
 def fused_select_compact(p, sms) -> bool:
     """Whether csp_select_compact runs as one persistent kernel for dense, contiguous outputs in a second buffer (what
-    this file passes): at least two units per SM and caches of 2 K - 8 K positions."""
-    return p.batch * p.n_kv_heads >= 2 * sms and 2048 < p.max_len <= 8192 and p.out_capacity > 0
+    this file passes): at least one unit per SM and caches of 1 K - 4 K positions."""
+    return p.batch * p.n_kv_heads >= sms and 1024 < p.max_len <= 4096 and p.out_capacity > 0
 
 
 def kernels_per_call(p, sms) -> int:
@@ -354,6 +354,9 @@ class PathBench:
         world = 1 if self.dist is None else self.dist.get_world_size()
         wss = [csp.new_workspace(calls[0].p, dev) for _ in range(n_chains)]   # one scratch area per concurrent chain
         out = {}
+        # the inputs and the zeroed workspaces were produced on torch's default stream; the calls below run on a
+        # stream of their own that does not wait for it
+        torch.cuda.synchronize()
         with torch.cuda.stream(stream):
             for _ in range(max(args.warmup, 3)):
                 for c in calls:

@@ -147,7 +147,13 @@ score_tc_persist_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArg
     auto unit_of = [&](int u) {
         Unit x;
         x.b = u / a.n_kv_heads; x.h = u % a.n_kv_heads;
-        if (a.order) x.b = a.order[x.b];
+        if (a.order) {
+            // the order list lives in the caller's workspace: an entry that is not a sequence number (the caller
+            // overwrote the workspace during the call) must not become an address
+            const int ob = a.order[x.b];
+            if (ob >= 0 && ob < n_units / a.n_kv_heads) x.b = ob;
+            else atomicOr(a.status, CSP_DEV_BAD_LEN);
+        }
         int L = a.seq_lens[x.b];
         const bool bad = L < 0 || L > a.max_len;
         x.skip = bad || L < a.window || L < a.recent;

@@ -115,7 +115,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreArgs a, con
     volatile int* const n_dq = reinterpret_cast<volatile int*>(base_ptr + sp.misc + 8);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int h = blockIdx.y, b = a.order ? a.order[blockIdx.z] : int(blockIdx.z);
+    const int h = blockIdx.y;
+    int b = int(blockIdx.z);
+    if (a.order) {
+        // the order list lives in the caller's workspace: an entry that is not a sequence number must not become an address
+        const int ob = a.order[b];
+        if (ob >= 0 && ob < int(gridDim.z)) b = ob;
+        else if (threadIdx.x == 0) atomicOr(a.status, CSP_DEV_BAD_LEN);
+    }
     const uint32_t rank = cluster_rank(), csize = cluster_size();
 
     int L = a.seq_lens[b];

@@ -14,8 +14,8 @@
 // No register staging: what is in flight is bounded by shared memory (six stages of 32 KB), not by the
 // register file.  Stages of 16 KB were 13 % slower on the copy, stages of 64 KB 2 %.  Every wait is bounded.
 //
-// Preconditions (checked by the launcher): one CTA's selection covers the longest cache, the outputs are a
-// second, dense buffer with contiguous rows, the cache is not paged.
+// Preconditions (checked by the launcher): the longest cache has at most 4096 positions (8 keys per selection
+// thread), the outputs are a second, dense buffer with contiguous rows, the cache is not paged.
 #include "csp_select_unit.cuh"
 
 namespace csp {
@@ -77,7 +77,7 @@ __device__ __forceinline__ bool wait_selected(uint32_t counter, int want, volati
     }
 }
 
-template <int E, int CPR>    // keys per selection thread; 16-byte chunks per row (8, 16 or 32)
+template <int E, int CPR>    // keys per selection thread (4 or 8); 16-byte chunks per row (8, 16 or 32)
 __global__ void __launch_bounds__(kScThreads, 1)
 select_compact_kernel(const SelectArgs sa, const CompactArgs ca, const int n_units, const int n_stages) {
     constexpr int kRowsPerStage = kHalfStage / (16 * CPR);
@@ -252,8 +252,11 @@ csp_status launch_select_compact(const csp_params& p, const SelectArgs& sa, cons
     *taken = false;
     const int units = p.batch * p.n_kv_heads;
     const int sms = sm_count();
-    if (units < 2 * sms || p.out_capacity == 0) return CSP_OK;          // too few units for a resident loop to pay off
-    if (p.max_len <= 2048 || p.max_len > 8192) return CSP_OK;            // one 512-thread team per unit, 8 or 16 keys a thread
+    // Measured against the two kernels one after the other (d = 128, a quarter of the rows kept): 4 % faster with 160
+    // units of 4096 positions, 9 % with 256, 15 % with 1024; 11 % faster at 2048 positions, even at 1024, slower at
+    // 512 and, with 16 keys per selection thread, at 8192.
+    if (units < sms || p.out_capacity == 0) return CSP_OK;
+    if (p.max_len <= 1024 || p.max_len > 4096) return CSP_OK;           // one 512-thread team per unit, 4 or 8 keys a thread
     if (ca.page_table || !ca.status) return CSP_OK;
     if (ca.k == ca.k_out || ca.v == ca.v_out) return CSP_OK;
     if (ca.ko_st != ca.chunks_per_row || ca.vo_st != ca.chunks_per_row) return CSP_OK;   // kept rows back to back
@@ -267,11 +270,11 @@ csp_status launch_select_compact(const csp_params& p, const SelectArgs& sa, cons
         return CSP_OK;
     };
     static std::atomic<bool> cfg[6][kMaxDevices];
-    const bool wide = p.max_len > 4096;
+    const bool wide = p.max_len > 2048;
     switch (ca.chunks_per_row) {
-        case 8: return wide ? go(select_compact_kernel<16, 8>, cfg[0]) : go(select_compact_kernel<8, 8>, cfg[1]);
-        case 16: return wide ? go(select_compact_kernel<16, 16>, cfg[2]) : go(select_compact_kernel<8, 16>, cfg[3]);
-        case 32: return wide ? go(select_compact_kernel<16, 32>, cfg[4]) : go(select_compact_kernel<8, 32>, cfg[5]);
+        case 8: return wide ? go(select_compact_kernel<8, 8>, cfg[0]) : go(select_compact_kernel<4, 8>, cfg[1]);
+        case 16: return wide ? go(select_compact_kernel<8, 16>, cfg[2]) : go(select_compact_kernel<4, 16>, cfg[3]);
+        case 32: return wide ? go(select_compact_kernel<8, 32>, cfg[4]) : go(select_compact_kernel<4, 32>, cfg[5]);
         default: return CSP_OK;
     }
 }

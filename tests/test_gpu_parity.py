@@ -889,9 +889,9 @@ def test_seeded_sweep_of_shapes_and_modes(csp, oracle, seed):
 
 # ------------------------------------------------------------------ many units: selection and compaction in one kernel
 
-def _many_units_case(rng, seed, hi, n_kv, d, dtype=torch.bfloat16, G=1):
-    """A batch with at least 300 (sequence, KV head) units and caches of up to `hi` positions, a few of them short."""
-    B = -(-300 // n_kv) + int(rng.randint(0, 3))
+def _many_units_case(rng, seed, hi, n_kv, d, dtype=torch.bfloat16, G=1, min_units=300):
+    """A batch with at least `min_units` (sequence, KV head) units and caches of up to `hi` positions, one of them short."""
+    B = -(-min_units // n_kv) + int(rng.randint(0, 3))
     lens = [int(x) for x in rng.randint(hi // 2, hi + 1, size=B)]
     lens[0] = hi
     lens[1] = int(rng.randint(60, 200))                  # a short cache in the same call
@@ -899,14 +899,17 @@ def _many_units_case(rng, seed, hi, n_kv, d, dtype=torch.bfloat16, G=1):
                  text_pct=int(rng.randint(5, 60)))
 
 
-@pytest.mark.parametrize("seed,hi,n_kv,d,dtype", [
-    (0, 2100, 16, 128, torch.bfloat16), (1, 4096, 8, 128, torch.bfloat16), (2, 3000, 16, 64, torch.bfloat16),
-    (3, 8192, 8, 64, torch.bfloat16), (4, 5000, 8, 128, torch.bfloat16), (5, 2500, 8, 128, torch.float32)])
-def test_many_units_mid_length_caches(csp, oracle, seed, hi, n_kv, d, dtype):
-    """Launches that take the fused selection + compaction kernel (hundreds of units, caches of 2-8 K positions): the
-    whole pass against the oracle, and bit-identical to the three stages called one by one."""
+@pytest.mark.parametrize("seed,hi,n_kv,d,dtype,min_units", [
+    (0, 2100, 16, 128, torch.bfloat16, 300), (1, 4096, 8, 128, torch.bfloat16, 300), (2, 3000, 16, 64, torch.bfloat16, 300),
+    (3, 8192, 8, 64, torch.bfloat16, 300), (4, 5000, 8, 128, torch.bfloat16, 300), (5, 2500, 8, 128, torch.float32, 300),
+    (6, 1100, 16, 128, torch.bfloat16, 300), (7, 2048, 8, 64, torch.bfloat16, 150), (8, 4000, 4, 128, torch.bfloat16, 150),
+    (9, 1500, 8, 128, torch.float32, 200)])
+def test_many_units_mid_length_caches(csp, oracle, seed, hi, n_kv, d, dtype, min_units):
+    """Launches that take the fused selection + compaction kernel (at least one unit per SM, caches of 1 K - 4 K
+    positions, with 4 or 8 keys per selection thread) and, beside them, some just outside that range: the whole pass
+    against the oracle, and bit-identical to the three stages called one by one."""
     rng = np.random.RandomState(7000 + seed)
-    cfg = _many_units_case(rng, seed, hi, n_kv, d, dtype)
+    cfg = _many_units_case(rng, seed, hi, n_kv, d, dtype, min_units=min_units)
     mode = dict(select_mode=int(rng.choice([0, 0, 1, 2])), combine=int(rng.choice([0, 0, 1])))
     nb = {0: 4, 1: 2, 2: 1}[mode["select_mode"]]
     B = cfg.batch
