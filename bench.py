@@ -373,17 +373,6 @@ class PathBench:
             n_out_total = int(first.lb.n_out.clamp(min=0).sum().item()) // first.layers      # kept rows per layer
             ms_step, clocks = self.time_replays(graph, args.steps)
 
-            # ---- sustained: the same graph replayed for about args.sustain_s seconds; the SM clock is sampled
-            # throughout, and time x clock shows how much of a difference to the short run is the clock's
-            sustained = None
-            if want_extras and args.sustain_s > 0:
-                n_rep = max(args.steps, int(args.sustain_s * 1e3 / max(ms_step, 1e-3)) + 1)
-                ms_sus, clk_sus = self.time_replays(graph, n_rep)
-                sustained = {"seconds": ms_sus * n_rep * 1e-3, "steps": n_rep, "ms_per_step": ms_sus,
-                             "value": job_throughput(world, tokens_per_layer, n_layers, ms_sus), "clocks": clk_sus,
-                             "ms_x_ghz": None if not clk_sus or not clk_sus.get("sm_mhz") else ms_sus * clk_sus["sm_mhz"] * 1e-3,
-                             "short_run_ms_x_ghz": None if not clocks or not clocks.get("sm_mhz") else ms_step * clocks["sm_mhz"] * 1e-3}
-
             # ---- per-kernel durations, live: one CUDA graph per kernel holding that kernel's launch for
             # every call of a step, replayed back to back and timed with events on the launching stream
             ws = wss[0]
@@ -413,6 +402,18 @@ class PathBench:
             for name, fn in stages:
                 per[name] = self.time_graph_of(fn, reps) / len(calls)                # ms per launch
             status |= csp.device_status(ws)
+
+            # ---- sustained: the same graph replayed for about args.sustain_s seconds; the SM clock is sampled
+            # throughout, and time x clock shows how much of a difference to the short run is the clock's.  Last,
+            # so that the per-kernel durations above are taken at the clocks of the short run
+            sustained = None
+            if want_extras and args.sustain_s > 0:
+                n_rep = max(args.steps, int(args.sustain_s * 1e3 / max(ms_step, 1e-3)) + 1)
+                ms_sus, clk_sus = self.time_replays(graph, n_rep)
+                sustained = {"seconds": ms_sus * n_rep * 1e-3, "steps": n_rep, "ms_per_step": ms_sus,
+                             "value": job_throughput(world, tokens_per_layer, n_layers, ms_sus), "clocks": clk_sus,
+                             "ms_x_ghz": None if not clk_sus or not clk_sus.get("sm_mhz") else ms_sus * clk_sus["sm_mhz"] * 1e-3,
+                             "short_run_ms_x_ghz": None if not clocks or not clocks.get("sm_mhz") else ms_step * clocks["sm_mhz"] * 1e-3}
 
         peak, peak_kind = measured_peaks()
         lens = lens_per_layer if lens_per_layer is not None else cfg.seq_lens
