@@ -892,7 +892,7 @@ def run_incremental(args, rank, world, local_rank):
     """`--incremental`: a re-prune round of the serving shape (configs[4]) two ways.  Every head's compacted cache
     has grown by 64 decoded tokens and is pruned back to its budget, either by csp_prune_layer (the window's 32
     queries rescan the whole cache) or from the intra / inter sums that the last 32 decode steps carried along
-    (csp_decode_step), which leaves csp_select + csp_compact.  Four distinct layers folded into one call each;
+    (csp_decode_step), which leaves csp_select_compact.  Four distinct layers folded into one call each;
     decode calls are timed at the final cache length.  Prints its own JSON line; not the default."""
     from paper_2412_04652_b200 import binding as csp
     csp.lib()
@@ -966,8 +966,8 @@ def run_incremental(args, rank, world, local_rank):
         n_full = n_o.clone()
 
         def from_sums():
-            csp.select(p2, acc_s, acc_c, mod_c, lens2, bud2, idx, n_o, ws2, total_budget=tot2)
-            csp.compact(p2, k_c, v_c, mod_c, idx, n_o, k_o, v_o, mod_o)
+            csp.select_compact(p2, acc_s, acc_c, k_c, v_c, mod_c, lens2, bud2, k_o, v_o, mod_o, n_o, ws2, total_budget=tot2,
+                               keep_idx=idx)
         t_inc = pb.time_graph_of(from_sums, reps)
         status |= csp.device_status(ws2) | csp.device_status(wd) | csp.device_status(wst)
         same_rows = bool(torch.equal(n_full, n_o))
@@ -994,7 +994,10 @@ def run_incremental(args, rank, world, local_rank):
                 "full_rescan": {"value": world * tokens_per_layer / (per_layer(t_full) * 1e-3), "unit": UNIT},
                 "decode": {"achieved_gbs": dec_bytes / (t_dec * 1e-3) / 1e9, "with_sums_gbs": dec_bytes / (t_step * 1e-3) / 1e9,
                            "peak": peak, "peak_kind": f"of {peak_kind}"},
-                "same_row_counts_both_ways": same_rows, "device_status": status, "gpu_launches": reps * 9, "e2e": None,
+                "same_row_counts_both_ways": same_rows, "device_status": status,
+                # decode attention + merge, decode step + merge, the rescan's kernels, selection + compaction from the sums
+                "gpu_launches": reps * (2 + 2 + kernels_per_call(p2, pb.sms) + (1 if fused_select_compact(p2, pb.sms) else 2)),
+                "e2e": None,
                 "cpu_baseline": None}
         print(json.dumps(line), flush=True)
 
