@@ -989,3 +989,63 @@ def test_many_units_bad_length_and_capacity_are_flagged(csp, oracle):
     assert (run.mod_out == 0).all()
     run.n_out[[2, 3, 4]] = 0
     assert_compaction_exact(run, np.zeros_like(mod))
+
+
+def test_select_compact_randomized_against_the_two_calls(csp):
+    """Seeded random launches inside the fused kernel's range (148-420 units, 1 K - 4 K positions; head_dim, element type,
+    window, recent size, selection and combination mode, shared or per-head labels, tied scores, budgets above the
+    candidates, caches too short to prune, capacities that do not hold every unit): csp_select_compact must leave exactly what
+    csp_select followed by csp_compact leaves, untouched rows included, and raise the same flags."""
+    for it in range(60):
+        rng = np.random.RandomState(50000 + it)
+        H = int(rng.choice([4, 8, 16, 32]))
+        B = int(rng.randint(-(-148 // H), -(-420 // H) + 1))
+        d, dt = [(128, torch.bfloat16), (64, torch.bfloat16), (128, torch.float32), (64, torch.float32)][rng.randint(4)]
+        hi = int(rng.randint(1025, 4097))
+        R, W = int(rng.choice([0, 7, 32, 64])), int(rng.choice([1, 16, 32]))
+        lens = rng.randint(max(W, R, 2), hi + 1, size=B).astype(np.int32)
+        lens[0] = hi
+        if rng.randint(3) == 0:
+            lens[rng.randint(B)] = int(rng.randint(0, max(W, R) + 1))
+        mode, comb = int(rng.choice([0, 0, 1, 2])), int(rng.choice([0, 0, 1]))
+        bud = rng.randint(0, hi // 5, size=(B, {0: 4, 1: 2, 2: 1}[mode])).astype(np.int32)
+        if rng.randint(4) == 0:
+            bud[rng.randint(B)] = hi
+        tot = rng.randint(0, hi, size=B).astype(np.int32) if rng.randint(3) == 0 else None
+        most = int(bud.sum(axis=1).max()) + R
+        cap = max(1, int(rng.choice([hi, most, most - int(rng.randint(1, 50))])))
+        g = torch.Generator(device="cuda")
+        g.manual_seed(it)
+        k = torch.randn(B, H, hi, d, device="cuda", generator=g).to(dt)
+        v = torch.randn(B, H, hi, d, device="cuda", generator=g).to(dt)
+        ss = torch.rand(B, H, hi, device="cuda", generator=g)
+        sc = torch.rand(B, H, hi, device="cuda", generator=g)
+        if rng.randint(3) == 0:
+            ss, sc = (ss * 8).floor() / 8, (sc * 4).floor() / 4
+        mod = (torch.rand((B, H, hi) if rng.randint(2) else (B, hi), device="cuda", generator=g) < 0.6).to(torch.uint8)
+        p = csp.Params(B, H, H, d, W, R, hi, cap, dtype=csp.F32 if dt == torch.float32 else csp.BF16, select_mode=mode,
+                       combine=comb)
+        lens_t, bud_t = torch.from_numpy(lens).cuda(), torch.from_numpy(bud).cuda()
+        tot_t = None if tot is None else torch.from_numpy(tot).cuda()
+        outs = []
+        for fused in (True, False):
+            ko = torch.full((B, H, cap, d), 3.0, device="cuda").to(dt)
+            vo = torch.full((B, H, cap, d), 5.0, device="cuda").to(dt)
+            mo = torch.full((B, H, cap), 9, dtype=torch.uint8, device="cuda")
+            no = torch.full((B, H), -7, dtype=torch.int32, device="cuda")
+            idx = torch.full((B, H, cap), -1, dtype=torch.int32, device="cuda")
+            ws = csp.new_workspace(p)
+            torch.cuda.synchronize()
+            if fused:
+                csp.select_compact(p, ss, sc, k, v, mod, lens_t, bud_t, ko, vo, mo, no, ws, total_budget=tot_t, keep_idx=idx)
+            else:
+                csp.select(p, ss, sc, mod, lens_t, bud_t, idx, no, ws, total_budget=tot_t)
+                csp.compact(p, k, v, mod, idx, no, ko, vo, mo)
+            outs.append((ko, vo, mo, no, idx, csp.device_status(ws)))
+        a, b = outs
+        what = f"iteration {it}: B={B} H={H} d={d} {dt} max_len={hi} R={R} W={W} mode={mode} combine={comb} cap={cap}"
+        assert a[5] == b[5] and not a[5] & csp.DEV_TIMEOUT, what
+        assert torch.equal(a[3], b[3]), what
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and torch.equal(a[2], b[2]), what
+        kept = torch.arange(cap, device="cuda")[None, None, :] < a[3].clamp(min=0)[:, :, None]
+        assert torch.equal(a[4][kept], b[4][kept]), what
