@@ -5,16 +5,19 @@
 // of the second's time.  Here one CTA per SM walks over units blockIdx.x, blockIdx.x + gridDim.x, ... with
 // its warps split by role, so that the selection of later units hides under the copy of earlier ones:
 //   warps 0-15   selection team: sel::select_unit on one unit after the other, as far ahead as it likes (its
-//                results go to global memory: keep_idx, n_out); after each unit it publishes a counter
-//   warps 16-23  gather team: for every kept row, 16-byte asynchronous copies (cp.async) from the row's place in
+//                results go to global memory: keep_idx, n_out, and the labels of the kept positions, which it holds
+//                in registers); after each unit it publishes a counter
+//   next 4 (3)   gather team: for every kept row, 16-byte asynchronous copies (cp.async) from the row's place in
 //                K and V into a stage of shared memory, where the kept rows of a unit lie back to back
-//   warp  24     store: one bulk copy (cp.async.bulk) per tensor and stage from shared memory to the output,
+//   last warp    store: one bulk copy (cp.async.bulk) per tensor and stage from shared memory to the output,
 //                where kept rows are contiguous as well
-//   warp  25     labels of the kept rows (two dependent loads per row: kept off the gather team's path)
-// No register staging: what is in flight is bounded by shared memory (six stages of 32 KB), not by the
-// register file.  Stages of 16 KB were 13 % slower on the copy, stages of 64 KB 2 %.  Every wait is bounded.
+// No register staging: what is in flight is bounded by shared memory (six stages of 32 KB, or eight of 24 KB with
+// three gather warps), not by the register file.  Stages of 16 KB were 13 % slower on the copy, stages of 64 KB 2 %;
+// 24 and 32 KB are level, and so are 3, 4 and 8 gather warps.  A warp of its own for the labels (two dependent loads per
+// kept row) cost registers the selection needs, and fetching them in the gather team held every stage up (the copy took
+// twice as long): the selection team has them in registers.  Every wait is bounded.
 //
-// Preconditions (checked by the launcher): the longest cache has at most 4096 positions (8 keys per selection
+// Preconditions (checked by the launcher): the longest cache has at most 8192 positions (16 keys per selection
 // thread), the outputs are a second, dense buffer with contiguous rows, the cache is not paged.
 #include "csp_select_unit.cuh"
 
@@ -24,20 +27,29 @@ using namespace dev;
 
 constexpr int kSelThreads = 512;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kGatherWarps = 8;
-constexpr int kGatherThreads = 32 * kGatherWarps;
-constexpr int kStoreWarp = kSelWarps + kGatherWarps;
-constexpr int kLabelWarp = kStoreWarp + 1;
-constexpr int kScThreads = kSelThreads + kGatherThreads + 64;
-constexpr int kHalfStage = 16384;                         // bytes of K (and of V) per stage
-constexpr int kStageBytes = 2 * kHalfStage;
-constexpr int kChunksPerThread = kHalfStage / 16 / kGatherThreads;   // 16-byte chunks of one tensor per gather thread and stage
-constexpr int kMaxStages = 6;
-constexpr int kDepth = 3;                                // stages a gather thread keeps in flight
 constexpr int kAhead = 2;                                // stages between the fetch of a row's position and its use
 constexpr int kStoresPending = 2;                        // bulk stores that may still be reading shared memory
-static_assert(kMaxStages >= kDepth + kStoresPending + 1, "ring too short for the copies in flight");
-static_assert(kChunksPerThread * kGatherThreads * 16 == kHalfStage, "stage must divide among the gather threads");
+constexpr int kMaxStages = 8;
+
+// The CTA's shape follows from the registers the selection needs.  The register file is four partitions of 16384
+// registers, each holding a quarter of the CTA's warps: 21 warps (four of them gathering) may use 80 registers a thread,
+// which 4 or 8 keys per selection thread fit; 16 keys need 96, which leaves room for 20 warps (three gathering).
+template <int E>
+struct Shape {
+    static constexpr int kGatherWarps = E > 8 ? 3 : 4;
+    static constexpr int kGatherThreads = 32 * kGatherWarps;
+    static constexpr int kStoreWarp = kSelWarps + kGatherWarps;
+    static constexpr int kThreads = kSelThreads + kGatherThreads + 32;
+    static constexpr int kRegisters = E > 8 ? 96 : 80;
+    static constexpr int kHalfStage = E > 8 ? 12288 : 16384;          // bytes of K (and of V) per stage
+    static constexpr int kStageBytes = 2 * kHalfStage;
+    static constexpr int kChunksPerThread = kHalfStage / 16 / kGatherThreads;   // 16-byte chunks of one tensor per gather thread and stage
+    static constexpr int kStages = E > 8 ? 8 : 6;
+    static constexpr int kDepth = E > 8 ? 4 : 3;                      // stages a gather thread keeps in flight
+    static_assert((kThreads / 32 + 3) / 4 * (kRegisters * 32) <= 16384, "the CTA must fit the register file");
+    static_assert(kStages >= kDepth + kStoresPending + 1 && kStages <= kMaxStages, "ring too short for the copies in flight");
+    static_assert(kChunksPerThread * kGatherThreads * 16 == kHalfStage, "stage must divide among the gather threads");
+};
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -77,11 +89,16 @@ __device__ __forceinline__ bool wait_selected(uint32_t counter, int want, volati
     }
 }
 
-template <int E, int CPR>    // keys per selection thread (4 or 8); 16-byte chunks per row (8, 16 or 32)
-__global__ void __launch_bounds__(kScThreads, 1)
-select_compact_kernel(const SelectArgs sa, const CompactArgs ca, const int n_units, const int n_stages) {
+template <int E, int CPR>    // keys per selection thread (4, 8 or 16); 16-byte chunks per row (8, 16 or 32)
+__global__ void __maxnreg__(Shape<E>::kRegisters)
+select_compact_kernel(const SelectArgs sa, const CompactArgs ca, const int n_units) {
+    using S = Shape<E>;
+    constexpr int kGatherThreads = S::kGatherThreads, kStoreWarp = S::kStoreWarp, kHalfStage = S::kHalfStage;
+    constexpr int kStageBytes = S::kStageBytes, kChunksPerThread = S::kChunksPerThread, kDepth = S::kDepth;
+    constexpr int n_stages = S::kStages;
     constexpr int kRowsPerStage = kHalfStage / (16 * CPR);
     constexpr int kRowStep = kGatherThreads / CPR;       // rows between two chunks of one gather thread
+    static_assert(kGatherThreads % CPR == 0, "whole rows per pass of the gather team");
     __shared__ sel::SelectSmem<kSelWarps> sm;
     __shared__ __align__(8) uint64_t bars[2 * kMaxStages];
     __shared__ int selected;                             // units the selection team has finished
@@ -105,7 +122,7 @@ select_compact_kernel(const SelectArgs sa, const CompactArgs ca, const int n_uni
         // =============================== selection team ===============================
         int done = 0;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-            sel::select_unit<kSelThreads, E, true>(sa, u, sm);
+            sel::select_unit<kSelThreads, E, true>(sa, u, sm, (ca.mod_out && ca.modality) ? ca.mod_out : nullptr);
             // keep_idx and n_out of this unit are written: order them before the counter, and keep the next
             // unit's writes to the team's shared memory behind this unit's last reads
             __threadfence();
@@ -183,30 +200,6 @@ select_compact_kernel(const SelectArgs sa, const CompactArgs ca, const int n_uni
         }
         cp_async_wait<0>();                              // also on the way out after a timeout: nothing may land later
         signal_upto(issued);
-    } else if (warp == kLabelWarp) {
-        // =============================== labels ===============================
-        if (ca.mod_out && ca.modality) {
-            int j = 0;
-            for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++j) {
-                if (!wait_selected(counter, j + 1, abort_flag)) break;
-                const int b = u / ca.n_kv_heads, h = u % ca.n_kv_heads;
-                const int n = min(__ldcg(ca.n_out + u), ca.out_capacity);
-                const int32_t* const idx = ca.keep_idx + int64_t(u) * ca.out_capacity;
-                const uint8_t* const mod = ca.modality + int64_t(b) * ca.mod_sb + int64_t(h) * ca.mod_sh;
-                uint8_t* const mod_out = ca.mod_out + int64_t(u) * ca.out_capacity;
-                for (int r0 = 0; r0 < n; r0 += 4 * 32) {
-                    int t[4];
-                    uint8_t lab[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) { const int r = r0 + q * 32 + lane; t[q] = r < n ? __ldcg(idx + r) : -1; }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) lab[q] = (t[q] >= 0 && t[q] < ca.max_len) ? mod[t[q]] : 0;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (t[q] >= 0 && t[q] < ca.max_len) mod_out[r0 + q * 32 + lane] = lab[q];
-                }
-            }
-        }
     } else if (lane == 0) {
         // =============================== store ===============================
         uint8_t* const kout = static_cast<uint8_t*>(ca.k_out);
@@ -253,28 +246,36 @@ csp_status launch_select_compact(const csp_params& p, const SelectArgs& sa, cons
     const int units = p.batch * p.n_kv_heads;
     const int sms = sm_count();
     // Measured against the two kernels one after the other (d = 128, a quarter of the rows kept): 4 % faster with 160
-    // units of 4096 positions, 9 % with 256, 15 % with 1024; 11 % faster at 2048 positions, even at 1024, slower at
-    // 512 and, with 16 keys per selection thread, at 8192.
+    // units of 4096 positions, 9 % with 256, 15 % with 1024; 13 % faster at 2048 positions, 9 % at 1500, even at 1024,
+    // slower at 512.  With 16 keys per selection thread (above 4096 positions): 10 % faster with 1024 units of 8192
+    // positions, 6 % with 512, even with 320, 2 % slower with 256.
     if (units < sms || p.out_capacity == 0) return CSP_OK;
-    if (p.max_len <= 1024 || p.max_len > 4096) return CSP_OK;           // one 512-thread team per unit, 4 or 8 keys a thread
+    if (p.max_len <= 1024 || p.max_len > 8192) return CSP_OK;           // one 512-thread team per unit, 4, 8 or 16 keys a thread
+    if (p.max_len > 4096 && units < 2 * sms) return CSP_OK;
     if (ca.page_table || !ca.status) return CSP_OK;
     if (ca.k == ca.k_out || ca.v == ca.v_out) return CSP_OK;
     if (ca.ko_st != ca.chunks_per_row || ca.vo_st != ca.chunks_per_row) return CSP_OK;   // kept rows back to back
-    const int stages = kMaxStages;
-    const size_t smem = size_t(stages) * kStageBytes + 128;
-    auto go = [&](auto kern, std::atomic<bool> (&configured)[kMaxDevices]) {
+    auto go = [&](auto kern, auto shape, std::atomic<bool> (&configured)[kMaxDevices]) {
+        using S = decltype(shape);
+        const size_t smem = size_t(S::kStages) * S::kStageBytes + 128;
         if (!raise_smem_limit(kern, int(smem), configured)) return CSP_ERR_CUDA;
-        kern<<<sms, kScThreads, smem, s>>>(sa, ca, units, stages);
+        kern<<<sms, S::kThreads, smem, s>>>(sa, ca, units);
         if (cudaGetLastError() != cudaSuccess) return CSP_ERR_CUDA;
         *taken = true;
         return CSP_OK;
     };
-    static std::atomic<bool> cfg[6][kMaxDevices];
-    const bool wide = p.max_len > 2048;
+    static std::atomic<bool> cfg[9][kMaxDevices];
+    const int e = p.max_len > 4096 ? 16 : (p.max_len > 2048 ? 8 : 4);
     switch (ca.chunks_per_row) {
-        case 8: return wide ? go(select_compact_kernel<8, 8>, cfg[0]) : go(select_compact_kernel<4, 8>, cfg[1]);
-        case 16: return wide ? go(select_compact_kernel<8, 16>, cfg[2]) : go(select_compact_kernel<4, 16>, cfg[3]);
-        case 32: return wide ? go(select_compact_kernel<8, 32>, cfg[4]) : go(select_compact_kernel<4, 32>, cfg[5]);
+        case 8:
+            return e == 16 ? go(select_compact_kernel<16, 8>, Shape<16>(), cfg[0])
+                 : e == 8  ? go(select_compact_kernel<8, 8>, Shape<8>(), cfg[1]) : go(select_compact_kernel<4, 8>, Shape<4>(), cfg[2]);
+        case 16:
+            return e == 16 ? go(select_compact_kernel<16, 16>, Shape<16>(), cfg[3])
+                 : e == 8  ? go(select_compact_kernel<8, 16>, Shape<8>(), cfg[4]) : go(select_compact_kernel<4, 16>, Shape<4>(), cfg[5]);
+        case 32:
+            return e == 16 ? go(select_compact_kernel<16, 32>, Shape<16>(), cfg[6])
+                 : e == 8  ? go(select_compact_kernel<8, 32>, Shape<8>(), cfg[7]) : go(select_compact_kernel<4, 32>, Shape<4>(), cfg[8]);
         default: return CSP_OK;
     }
 }

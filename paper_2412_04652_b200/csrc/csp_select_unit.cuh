@@ -60,9 +60,12 @@ __device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
 
 // kTeam = false: the calling CTA (all kCsThreads threads of it) is one of the cluster that owns unit u.
 // kTeam = true: the first kCsThreads threads of a larger CTA own unit u alone (no cluster); they synchronise
-// on a named barrier, and the caller puts such a barrier between two units because `sm` is reused.
+// on a named barrier, and the caller puts such a barrier between two units because `sm` is reused.  In this mode the team
+// also writes the labels of the kept positions (label side of Eq. 4) to labels_out [B, H_kv, out_capacity] when that is
+// not null: it holds every key's label in registers anyway.
 template <int kCsThreads, int E, bool kTeam>
-__device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit, SelectSmem<kCsThreads / 32>& sm) {
+__device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit, SelectSmem<kCsThreads / 32>& sm,
+                                            uint8_t* const labels_out = nullptr) {
     const int u = kTeam ? unit : int(blockIdx.y);       // the stand-alone kernel's grid row (a special register, not a live value)
     constexpr int kCsWarps = kCsThreads / 32;
     uint32_t (&hist)[2][4][256] = sm.hist;
@@ -100,6 +103,12 @@ __device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit,
             return;
         }
         for (int t = int(rank) * kCsThreads + tid; t < L; t += int(csize) * kCsThreads) idx[t] = t;
+        if constexpr (kTeam) {
+            if (labels_out) {
+                const uint8_t* const mod_u = a.modality + int64_t(b) * a.mod_sb + int64_t(h) * a.mod_sh;
+                for (int t = tid; t < L; t += kCsThreads) labels_out[int64_t(u) * a.out_capacity + t] = mod_u[t];
+            }
+        }
         if (tid == 0 && rank == 0) a.n_out[u] = L;
         return;
     }
@@ -117,6 +126,10 @@ __device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit,
     const int warp_base = (int(rank) * kCsWarps + warp) * (32 * E);
     uint32_t ks[E], kc[E];
     uint32_t valid = 0u, vis = 0u;                       // bit e: position in range / visual key
+    // team mode: the keys' label bytes, four to a register; with 16 keys per thread the registers are needed
+    // elsewhere and the labels of the kept keys are read again at the end
+    constexpr bool kKeepLabels = kTeam && E <= 8;
+    uint32_t labels[kKeepLabels ? (E + 3) / 4 : 1] = {};
     {
         // all loads are issued before any is used (positions past the end re-read position 0)
         float fs[E], fc[E];
@@ -137,6 +150,7 @@ __device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit,
             kc[e] = ok ? order_key(fc[e]) : 0u;
             if (ok) valid |= 1u << e;
             if (ok && !a.global_mode && lab[e] != 0) vis |= 1u << e;
+            if constexpr (kKeepLabels) labels[e >> 2] |= uint32_t(lab[e]) << (8 * (e & 3));
         }
     }
     if (tid < 4) {
@@ -363,11 +377,22 @@ __device__ __forceinline__ void select_unit(const SelectArgs& a, const int unit,
         for (int e = 0; e < E; ++e) {
             const bool keep = (keep_bits >> e) & 1u;
             const uint32_t m = __ballot_sync(kFull, keep);
-            if (keep) idx[pos + __popc(m & lt_mask)] = warp_base + e * 32 + lane;
+            if (keep) {
+                idx[pos + __popc(m & lt_mask)] = warp_base + e * 32 + lane;
+                if constexpr (kTeam) {
+                    if (labels_out)
+                        labels_out[int64_t(u) * a.out_capacity + pos + __popc(m & lt_mask)] =
+                            kKeepLabels ? uint8_t(labels[e >> 2] >> (8 * (e & 3))) : mod[warp_base + e * 32 + lane];
+                }
+            }
             pos += __popc(m);
         }
         if (rank == 0) {
             for (int j = tid; j < a.recent; j += kCsThreads) idx[int(n_keep) + j] = N + j;   // (+) the last R positions
+            if constexpr (kTeam) {
+                if (labels_out)
+                    for (int j = tid; j < a.recent; j += kCsThreads) labels_out[int64_t(u) * a.out_capacity + int(n_keep) + j] = mod[N + j];
+            }
             if (tid == 0) a.n_out[u] = int(n_keep) + a.recent;
         }
     }

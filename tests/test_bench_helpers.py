@@ -40,14 +40,15 @@ def test_algorithmic_bytes_of_the_headline_workload():
 
 def test_launch_count_of_a_call():
     """Kernels per csp_prune_layer call as the bench line claims them: the ordering kernel for batches of sequences, one
-    kernel for selection and compaction where at least an SM's worth of units hold 1 K - 4 K positions each."""
+    kernel for selection and compaction where at least an SM's worth of units hold 1 K - 4 K positions each (two per SM up to 8 K)."""
     class P:
         def __init__(self, batch, n_kv_heads, max_len, out_capacity=100, dtype=1):
             self.batch, self.n_kv_heads, self.max_len, self.out_capacity, self.dtype = batch, n_kv_heads, max_len, out_capacity, dtype
     assert bench.kernels_per_call(P(32, 32, 4096), 148) == 3        # order, score, selection + compaction
     assert bench.kernels_per_call(P(1, 32, 4096), 148) == 3         # one sequence: score, select, compact
     assert bench.kernels_per_call(P(32, 32, 16384), 148) == 4       # too long for one CTA's selection
-    assert bench.kernels_per_call(P(32, 8, 8109), 148) == 4         # more than 4096 positions
+    assert bench.kernels_per_call(P(32, 8, 8109), 148) == 4         # more than 4096 positions and fewer than two units per SM
+    assert bench.kernels_per_call(P(32, 32, 8109), 148) == 3        # 1024 units of up to 8109 positions
     assert bench.kernels_per_call(P(4, 32, 4096), 148) == 4         # 128 units: fewer than one per SM
     assert not bench.fused_select_compact(P(32, 32, 1024), 148) and bench.fused_select_compact(P(37, 4, 1025), 148)
 

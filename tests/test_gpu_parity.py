@@ -992,16 +992,17 @@ def test_many_units_bad_length_and_capacity_are_flagged(csp, oracle):
 
 
 def test_select_compact_randomized_against_the_two_calls(csp):
-    """Seeded random launches inside the fused kernel's range (148-420 units, 1 K - 4 K positions; head_dim, element type,
+    """Seeded random launches inside the fused kernel's range (148-420 units, 1 K - 4 K positions, every fourth one 300 units
+    or more of up to 8 K positions; head_dim, element type,
     window, recent size, selection and combination mode, shared or per-head labels, tied scores, budgets above the
     candidates, caches too short to prune, capacities that do not hold every unit): csp_select_compact must leave exactly what
     csp_select followed by csp_compact leaves, untouched rows included, and raise the same flags."""
     for it in range(60):
         rng = np.random.RandomState(50000 + it)
         H = int(rng.choice([4, 8, 16, 32]))
-        B = int(rng.randint(-(-148 // H), -(-420 // H) + 1))
+        B = int(rng.randint(-(-148 // H), -(-420 // H) + 1)) if it % 4 else -(-300 // H) + int(rng.randint(0, 3))
         d, dt = [(128, torch.bfloat16), (64, torch.bfloat16), (128, torch.float32), (64, torch.float32)][rng.randint(4)]
-        hi = int(rng.randint(1025, 4097))
+        hi = int(rng.randint(1025, 4097)) if it % 4 else int(rng.randint(4097, 8193))
         R, W = int(rng.choice([0, 7, 32, 64])), int(rng.choice([1, 16, 32]))
         lens = rng.randint(max(W, R, 2), hi + 1, size=B).astype(np.int32)
         lens[0] = hi
