@@ -241,9 +241,11 @@ def run_reference(args, rank, world):
 
 def fused_select_compact(p, sms) -> bool:
     """Whether csp_select_compact runs as one persistent kernel for dense, contiguous outputs in a second buffer (what
-    this file passes): at least one unit per SM and caches of 1 K - 4 K positions, or two per SM up to 8 K."""
+    this file passes): at least one unit per SM and caches of 1 K - 4 K positions, or two per SM up to 8 K when at least a
+    twelfth of the rows can be kept."""
     units = p.batch * p.n_kv_heads
-    return p.out_capacity > 0 and ((units >= sms and 1024 < p.max_len <= 4096) or (units >= 2 * sms and 4096 < p.max_len <= 8192))
+    return p.out_capacity > 0 and ((units >= sms and 1024 < p.max_len <= 4096) or
+                                   (units >= 2 * sms and 4096 < p.max_len <= 8192 and p.out_capacity * 12 >= p.max_len))
 
 
 def kernels_per_call(p, sms) -> int:

@@ -171,7 +171,7 @@ csp_status csp_compact(const csp_params* p, csp_tensor k, csp_tensor v,
  * csp_select followed by csp_compact on the same stream (Eq. 2-4), for a caller that already has the two score
  * vectors (from csp_score, or carried along by csp_decode_step).  Same arguments, results and flags as the two
  * calls; keep_idx may be NULL, in which case the list lives in the workspace.  With at least one unit per SM
- * and max_len in (1024, 4096] (two units per SM up to 8192), a second (not in-place) output buffer and contiguous output rows
+ * and max_len in (1024, 4096] (up to 8192 with two units per SM and out_capacity >= max_len / 12), a second (not in-place) output buffer and contiguous output rows
  * (stride_t == head_dim), both steps run in one persistent kernel in which the selection of later units overlaps
  * the copy of earlier ones; otherwise as two kernels.  The results do not depend on which.
  */

@@ -248,10 +248,13 @@ csp_status launch_select_compact(const csp_params& p, const SelectArgs& sa, cons
     // Measured against the two kernels one after the other (d = 128, a quarter of the rows kept): 4 % faster with 160
     // units of 4096 positions, 9 % with 256, 15 % with 1024; 13 % faster at 2048 positions, 9 % at 1500, even at 1024,
     // slower at 512.  With 16 keys per selection thread (above 4096 positions): 10 % faster with 1024 units of 8192
-    // positions, 6 % with 512, even with 320, 2 % slower with 256.
+    // positions (2080 rows kept), 6 % with 512, even with 320, 2 % slower with 256.
     if (units < sms || p.out_capacity == 0) return CSP_OK;
     if (p.max_len <= 1024 || p.max_len > 8192) return CSP_OK;           // one 512-thread team per unit, 4, 8 or 16 keys a thread
-    if (p.max_len > 4096 && units < 2 * sms) return CSP_OK;
+    // with 16 keys per thread one team selects a unit in about 22 us: the copy of a unit must be at least as long for the
+    // selection to hide (a ragged batch of 1024 units of up to 8109 positions: 5 % slower when 405 rows are kept per unit,
+    // 5 % faster with 811, 12 % with 1622 and 3244)
+    if (p.max_len > 4096 && (units < 2 * sms || int64_t(p.out_capacity) * 12 < p.max_len)) return CSP_OK;
     if (ca.page_table || !ca.status) return CSP_OK;
     if (ca.k == ca.k_out || ca.v == ca.v_out) return CSP_OK;
     if (ca.ko_st != ca.chunks_per_row || ca.vo_st != ca.chunks_per_row) return CSP_OK;   // kept rows back to back

@@ -48,7 +48,8 @@ def test_launch_count_of_a_call():
     assert bench.kernels_per_call(P(1, 32, 4096), 148) == 3         # one sequence: score, select, compact
     assert bench.kernels_per_call(P(32, 32, 16384), 148) == 4       # too long for one CTA's selection
     assert bench.kernels_per_call(P(32, 8, 8109), 148) == 4         # more than 4096 positions and fewer than two units per SM
-    assert bench.kernels_per_call(P(32, 32, 8109), 148) == 3        # 1024 units of up to 8109 positions
+    assert bench.kernels_per_call(P(32, 32, 8109, 811), 148) == 3   # 1024 units of up to 8109 positions, a tenth kept
+    assert bench.kernels_per_call(P(32, 32, 8109, 405), 148) == 4   # too few rows to copy for the selection to hide
     assert bench.kernels_per_call(P(4, 32, 4096), 148) == 4         # 128 units: fewer than one per SM
     assert not bench.fused_select_compact(P(32, 32, 1024), 148) and bench.fused_select_compact(P(37, 4, 1025), 148)
 
